@@ -1,0 +1,144 @@
+/*
+ * dass.h -- C ABI of the B200 (sm_100a) hot path of DaSS, Dependency-aware
+ * Semi-structured Sparsity for GLU-based MLPs (arXiv 2405.01943).
+ *
+ * Two stages:
+ *   (a) calibration: for every intermediate neuron i accumulate, over the
+ *       calibration tokens, the squared l2 norm of the GLU intermediate
+ *       activation  y = sigma(x W1) (*) x W2  (Eq. 2; norm as group importance,
+ *       Section 3 "Incorporating Dependency into Weight Importance").
+ *   (b) pruning: score every weight with |W| * ||y||^alpha (Eq. 4, gate / up)
+ *       or |W| * ||y|| (Eq. 5, down), keep the best n of every m consecutive
+ *       weights of a comparison line (Section 3, "Extension to N:M Sparsity"),
+ *       emit mask, pruned weights and a compressed values + metadata form.
+ *
+ * Conventions for every call
+ *   - Matrices are row-major with a leading dimension `ld` counted in elements.
+ *     The paper's transposed projections are used as stored by common
+ *     checkpoints: Wg = W(1)^T and Wu = W(2)^T are [I x d], Wd = W(3)^T is
+ *     [d x I]  (I = d_int, d = d_hidden), X is [T x d] (T tokens).
+ *   - Unless a parameter is documented as HOST, every pointer is DEVICE memory of
+ *     the current CUDA device, owned by the caller before, during and after the
+ *     call.  The library allocates no device memory and frees nothing.
+ *   - Calls only enqueue work on `cuda_stream` (a cudaStream_t passed as void*,
+ *     NULL = the default stream) and return without waiting for it.
+ *   - Base pointers of matrices must be 16-byte aligned and `ld` a multiple of
+ *     8 elements (bf16) or 4 elements (f32), else DASS_ERR_ALIGN.  A matrix
+ *     buffer must span rows * ld elements (vector loads may touch the padding
+ *     between `cols` and `ld`; it is never written).
+ *   - Errors are reported by the return code only: nothing aborts, throws or
+ *     prints, and on a non-OK return no output has been touched.
+ *   - Non-finite inputs are not diagnosed; results for them are unspecified.
+ */
+#ifndef DASS_H
+#define DASS_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    DASS_OK = 0,
+    DASS_ERR_NULL = 1,         /* a required pointer is NULL */
+    DASS_ERR_SHAPE = 2,        /* non-positive size, extent not divisible by m, bad n_keep */
+    DASS_ERR_ALIGN = 3,        /* pointer or leading dimension not aligned as required */
+    DASS_ERR_DTYPE = 4,        /* unknown dass_dtype / dass_act / dass_axis value */
+    DASS_ERR_UNSUPPORTED = 5,  /* a valid request this build has no kernel for */
+    DASS_ERR_WORKSPACE = 6,    /* workspace NULL or smaller than the query says */
+    DASS_ERR_CUDA = 7,         /* a CUDA runtime / driver call failed */
+    DASS_ERR_TIMEOUT = 8       /* a bounded device-side wait ran out (reported by dass_calib_status) */
+} dass_status;
+
+typedef enum { DASS_BF16 = 0, DASS_F32 = 1 } dass_dtype;
+typedef enum { DASS_ACT_SILU = 0, DASS_ACT_GELU_TANH = 1, DASS_ACT_RELU = 2 } dass_act;
+/* Which matrix axis an index runs along: ROWS = the row index varies, COLS = the column index varies. */
+typedef enum { DASS_AXIS_ROWS = 0, DASS_AXIS_COLS = 1 } dass_axis;
+
+/* ------------------------------------------------------------------ stage (a)
+ * Eq. 2 and the per-neuron squared norm:
+ *     sumsq[i] += sum_{t < T} ( act(X[t,:] . Wg[i,:]) * (X[t,:] . Wu[i,:]) )^2     for i in [0, I)
+ * act = SiLU (SwiGLU), tanh-form GeLU (GeGLU) or ReLU (ReGLU) -- Section 2.2.
+ * The intermediate H is never written to memory.
+ *
+ * X [T x d, ldx], Wg and Wu [I x d, ldw] in `dt`.  bf16: tensor-core path
+ * (fp32 accumulation, activation and square in fp32).  f32: plain fp32 FMA path.
+ * sumsq [I] doubles, in/out: the call ADDS this batch's contribution, so a
+ * calibration set may be fed in any number of batches; the caller zeroes it
+ * before the first batch.  The per-batch contribution is reduced in a fixed
+ * order, so equal inputs give bit-equal results.
+ * workspace: scratch of at least dass_calib_workspace_bytes(...) bytes, 256-byte
+ * aligned, contents irrelevant on entry; it must not be shared by calls that
+ * may overlap on the device.  Its first word receives a device status that
+ * dass_calib_status reads.
+ * Errors: NULL / SHAPE (T, d, I < 1) / ALIGN / DTYPE / WORKSPACE / CUDA. */
+dass_status dass_calib_workspace_bytes(int64_t T, int64_t d, int64_t I, dass_dtype dt, size_t *bytes /* HOST */);
+dass_status dass_calib_accumulate(const void *X, int64_t T, int64_t ldx,
+                                  const void *Wg, const void *Wu, int64_t I, int64_t d, int64_t ldw,
+                                  dass_dtype dt, dass_act act,
+                                  double *sumsq,
+                                  void *workspace, size_t workspace_bytes, void *cuda_stream);
+/* Waits for `cuda_stream`, then reports what the last dass_calib_accumulate that used
+ * `workspace` left in its status word: DASS_OK, or DASS_ERR_TIMEOUT if a bounded wait inside
+ * the kernel gave up (the results of that call are then invalid; the context stays usable). */
+dass_status dass_calib_status(const void *workspace, void *cuda_stream);
+
+/* norm[i] = (float) sqrt(sumsq[i]): the l2 norm ||y_i||_2 handed to stage (b).
+ * Both operations are correctly rounded, so the value is reproducible bit for bit. */
+dass_status dass_norm_finalize(const double *sumsq, int64_t I, float *norm, void *cuda_stream);
+
+/* ------------------------------------------------------------------ stage (b)
+ * Eq. 4 / Eq. 5 score and N:M selection.
+ *     score(r,c) = |W[r,c]| * scale(norm[k], alpha),   k = r if norm_axis == ROWS, c if COLS
+ *     scale(n, alpha) = (float) n^alpha, rounded once: 1 for alpha = 0 (also when n = 0), n for
+ *     alpha = 1, sqrt / sqrt(sqrt) / sqrt*sqrt(sqrt) evaluated in double for 1/2, 1/4, 3/4,
+ *     pow in double otherwise.  Scores are compared as exact products (no rounding).
+ * Groups are m consecutive elements along group_axis (ROWS: rows r..r+m-1 of one column; COLS:
+ * columns c..c+m-1 of one row).  In each group the n_keep highest scores are kept; among equal
+ * scores the lower index wins.
+ *     gate / up, Eq. 4:  W = Wg or Wu [I x d], norm_axis = ROWS, group_axis = ROWS  (input-balanced:
+ *                        the weights of one input column are compared across neurons), alpha = 0.5
+ *     down, Eq. 5:       W = Wd [d x I],       norm_axis = COLS, group_axis = COLS  (output-balanced),
+ *                        alpha = 1
+ *     Wanda, Eq. 1:      any W [out x in] with input-feature norms: norm_axis = COLS, group_axis = COLS
+ * norm: rows (ROWS) or cols (COLS) floats.  alpha: finite, >= 0.
+ * Supported patterns: m in {4, 8}, 1 <= n_keep < m; the group-axis extent must be a multiple of m,
+ * and for group_axis = ROWS with bf16 data `cols` ... any value; see alignment rules above.
+ * mask_bits (nullable): rows * ceil(cols/32) words; bit (c % 32) of word r * ceil(cols/32) + c / 32
+ *     is 1 iff W[r,c] is kept; padding bits are written as 0.
+ * W_pruned (nullable): same dtype and ld as W; survivors are copied bit for bit, the others become +0
+ *     ("no weight update").  May be W itself (in place).
+ * At least one of the two outputs must be given.
+ * Errors: NULL / SHAPE / ALIGN / DTYPE / UNSUPPORTED (alpha < 0 or not finite, m not 4 or 8). */
+dass_status dass_score_nm(const void *W, int64_t rows, int64_t cols, int64_t ld, dass_dtype dt,
+                          const float *norm, dass_axis norm_axis, float alpha,
+                          int n_keep, int m, dass_axis group_axis,
+                          uint32_t *mask_bits, void *W_pruned, void *cuda_stream);
+
+/* Compressed N:M form of W under a mask produced by dass_score_nm with the same n_keep, m, group_axis.
+ * The paper gives no storage format (it only points to N:M hardware support, Section 2.3); this is a
+ * plain, un-swizzled one:
+ * values: the n_keep survivors of every group in index order, dtype of W, densely packed:
+ *     group_axis = COLS: [rows x cols*n_keep/m];  ROWS: [rows*n_keep/m x cols].
+ * meta: one field per group.  2:4: a nibble pos_lo | pos_hi << 2 (positions 0..3 of the two survivors,
+ *     pos_lo < pos_hi).  Any other pattern: the m-bit keep mask of the group.  Fields are packed LSB
+ *     first along the columns; a line of fields (COLS: one row, cols/m fields; ROWS: one row group,
+ *     cols fields) is padded with zeros to whole 32-bit words.
+ *     Sizes: COLS: rows * ceil(cols/m / F) words, ROWS: (rows/m) * ceil(cols / F), F = 32 / field bits.
+ * A mask that does not hold exactly n_keep survivors in some group gives unspecified output.
+ * Errors: NULL / SHAPE / ALIGN / DTYPE / UNSUPPORTED as for dass_score_nm. */
+dass_status dass_compress_nm(const void *W, const uint32_t *mask_bits,
+                             int64_t rows, int64_t cols, int64_t ld, dass_dtype dt,
+                             int n_keep, int m, dass_axis group_axis,
+                             void *values, uint32_t *meta, void *cuda_stream);
+
+/* ------------------------------------------------------------------ misc */
+const char *dass_status_string(dass_status s);   /* static string, never NULL */
+int dass_version(void);                          /* major * 10000 + minor * 100 + patch */
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DASS_H */

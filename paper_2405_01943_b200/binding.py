@@ -1,0 +1,224 @@
+"""ctypes binding over libdass.so -- argument marshalling only.
+
+Every function here has the name of the C entry point it forwards to (minus the ``dass_`` prefix
+where that reads better) and does nothing but check tensor devices/dtypes, allocate requested
+outputs with torch, and pass raw pointers, sizes and the current CUDA stream across the C ABI
+(``include/dass.h``).  There is no CPU or PyTorch fallback: if the library is missing or a call
+fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Tuple
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libdass.so")
+
+OK = 0
+BF16, F32 = 0, 1
+ACT_SILU, ACT_GELU_TANH, ACT_RELU = 0, 1, 2
+AXIS_ROWS, AXIS_COLS = 0, 1
+ACT_BY_NAME = {"silu": ACT_SILU, "gelu_tanh": ACT_GELU_TANH, "relu": ACT_RELU}
+
+EXPORTS = (
+    "dass_calib_workspace_bytes", "dass_calib_accumulate", "dass_calib_status", "dass_norm_finalize",
+    "dass_score_nm", "dass_compress_nm", "dass_status_string", "dass_version",
+)
+
+
+class DassError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = int(code)
+        super().__init__(f"{where}: {status_string(code)} (dass_status {int(code)})")
+
+
+_lib = None
+
+
+def load() -> ctypes.CDLL:
+    """Loads libdass.so (built in-tree by ``python -m paper_2405_01943_b200.build``)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError(f"{LIB_PATH} is missing: build it with `python -m paper_2405_01943_b200.build` "
+                           "(there is no fallback implementation)")
+    lib = ctypes.CDLL(LIB_PATH)
+    i64, vp, sz = ctypes.c_int64, ctypes.c_void_p, ctypes.c_size_t
+    lib.dass_calib_workspace_bytes.restype = ctypes.c_int
+    lib.dass_calib_workspace_bytes.argtypes = [i64, i64, i64, ctypes.c_int, ctypes.POINTER(sz)]
+    lib.dass_calib_accumulate.restype = ctypes.c_int
+    lib.dass_calib_accumulate.argtypes = [vp, i64, i64, vp, vp, i64, i64, i64, ctypes.c_int, ctypes.c_int,
+                                          vp, vp, sz, vp]
+    lib.dass_calib_status.restype = ctypes.c_int
+    lib.dass_calib_status.argtypes = [vp, vp]
+    lib.dass_norm_finalize.restype = ctypes.c_int
+    lib.dass_norm_finalize.argtypes = [vp, i64, vp, vp]
+    lib.dass_score_nm.restype = ctypes.c_int
+    lib.dass_score_nm.argtypes = [vp, i64, i64, i64, ctypes.c_int, vp, ctypes.c_int, ctypes.c_float,
+                                  ctypes.c_int, ctypes.c_int, ctypes.c_int, vp, vp, vp]
+    lib.dass_compress_nm.restype = ctypes.c_int
+    lib.dass_compress_nm.argtypes = [vp, vp, i64, i64, i64, ctypes.c_int, ctypes.c_int, ctypes.c_int,
+                                     ctypes.c_int, vp, vp, vp]
+    lib.dass_status_string.restype = ctypes.c_char_p
+    lib.dass_status_string.argtypes = [ctypes.c_int]
+    lib.dass_version.restype = ctypes.c_int
+    lib.dass_version.argtypes = []
+    _lib = lib
+    return lib
+
+
+def status_string(code: int) -> str:
+    return load().dass_status_string(int(code)).decode()
+
+
+def version() -> int:
+    return int(load().dass_version())
+
+
+def _check(code: int, where: str) -> None:
+    if code != OK:
+        raise DassError(code, where)
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.bfloat16:
+        return BF16
+    if t.dtype == torch.float32:
+        return F32
+    raise TypeError(f"unsupported dtype {t.dtype}: the library takes bfloat16 or float32")
+
+
+def _matrix(t: torch.Tensor, name: str) -> Tuple[int, int, int]:
+    if not t.is_cuda:
+        raise ValueError(f"{name} must be a CUDA tensor")
+    if t.dim() != 2 or t.stride(1) != 1:
+        raise ValueError(f"{name} must be a 2-D row-major tensor (unit stride along columns)")
+    return t.shape[0], t.shape[1], t.stride(0) if t.shape[0] > 1 else max(t.stride(0), t.shape[1])
+
+
+def _stream(stream: Optional[torch.cuda.Stream]) -> int:
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return int(s.cuda_stream)
+
+
+def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
+    return None if t is None else t.data_ptr()
+
+
+# ----------------------------------------------------------------------------- stage (a)
+
+def calib_workspace_bytes(T: int, d: int, I: int, dtype: torch.dtype) -> int:
+    out = ctypes.c_size_t(0)
+    code = load().dass_calib_workspace_bytes(int(T), int(d), int(I), BF16 if dtype == torch.bfloat16 else F32,
+                                             ctypes.byref(out))
+    _check(code, "dass_calib_workspace_bytes")
+    return int(out.value)
+
+
+def calib_workspace(T: int, d: int, I: int, dtype: torch.dtype, device="cuda") -> torch.Tensor:
+    """A uint8 tensor large (and aligned) enough to serve as workspace of calib_accumulate."""
+    n = calib_workspace_bytes(T, d, I, dtype)
+    buf = torch.empty(n + 256, dtype=torch.uint8, device=device)
+    off = (-buf.data_ptr()) % 256
+    return buf[off:off + n]
+
+
+def calib_accumulate(X: torch.Tensor, Wg: torch.Tensor, Wu: torch.Tensor, act: int, sumsq: torch.Tensor,
+                     workspace: torch.Tensor, stream: Optional[torch.cuda.Stream] = None) -> None:
+    """sumsq[i] += sum_t (act(X Wg^T) * (X Wu^T))[t, i]^2 on the given (or current) stream."""
+    T, d, ldx = _matrix(X, "X")
+    I, d2, ldw = _matrix(Wg, "Wg")
+    I3, d3, ldw3 = _matrix(Wu, "Wu")
+    if (d2, I3, d3, ldw3) != (d, I, d, ldw) or Wg.dtype != X.dtype or Wu.dtype != X.dtype:
+        raise ValueError("X [T x d], Wg [I x d], Wu [I x d] must agree in d, I, dtype and row pitch")
+    if sumsq.dtype != torch.float64 or not sumsq.is_cuda or sumsq.numel() != I or not sumsq.is_contiguous():
+        raise ValueError("sumsq must be a contiguous CUDA float64 tensor of I elements")
+    if not workspace.is_cuda or workspace.dtype != torch.uint8:
+        raise ValueError("workspace must be a CUDA uint8 tensor (see calib_workspace)")
+    code = load().dass_calib_accumulate(X.data_ptr(), T, ldx, Wg.data_ptr(), Wu.data_ptr(), I, d, ldw,
+                                        _dtype_code(X), int(act), sumsq.data_ptr(),
+                                        workspace.data_ptr(), workspace.numel(), _stream(stream))
+    _check(code, "dass_calib_accumulate")
+
+
+def calib_status(workspace: torch.Tensor, stream: Optional[torch.cuda.Stream] = None) -> None:
+    """Waits for the stream and raises if the last calibration kernel reported a timed-out wait."""
+    _check(load().dass_calib_status(workspace.data_ptr(), _stream(stream)), "dass_calib_status")
+
+
+def norm_finalize(sumsq: torch.Tensor, norm: Optional[torch.Tensor] = None,
+                  stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
+    """norm = float32(sqrt(sumsq))."""
+    if norm is None:
+        norm = torch.empty(sumsq.numel(), dtype=torch.float32, device=sumsq.device)
+    code = load().dass_norm_finalize(sumsq.data_ptr(), sumsq.numel(), norm.data_ptr(), _stream(stream))
+    _check(code, "dass_norm_finalize")
+    return norm
+
+
+# ----------------------------------------------------------------------------- stage (b)
+
+def mask_words_per_row(cols: int) -> int:
+    return (cols + 31) // 32
+
+
+def score_nm(W: torch.Tensor, norm: torch.Tensor, norm_axis: int, alpha: float, n_keep: int, m: int,
+             group_axis: int, mask_bits: Optional[torch.Tensor] = None, W_pruned: Optional[torch.Tensor] = None,
+             want_mask: bool = True, want_pruned: bool = True,
+             stream: Optional[torch.cuda.Stream] = None):
+    """Eq. 4 / Eq. 5 score + N:M selection. Returns (mask_bits or None, W_pruned or None)."""
+    rows, cols, ld = _matrix(W, "W")
+    if norm.dtype != torch.float32 or not norm.is_cuda or not norm.is_contiguous():
+        raise ValueError("norm must be a contiguous CUDA float32 tensor")
+    if norm.numel() != (rows if norm_axis == AXIS_ROWS else cols):
+        raise ValueError("norm has the wrong length for norm_axis")
+    if mask_bits is None and want_mask:
+        mask_bits = torch.empty((rows, mask_words_per_row(cols)), dtype=torch.int32, device=W.device)
+    if W_pruned is None and want_pruned:
+        W_pruned = torch.empty_strided((rows, cols), (ld, 1), dtype=W.dtype, device=W.device)
+    if W_pruned is not None:
+        prow, pcol, pld = _matrix(W_pruned, "W_pruned")
+        if (prow, pcol, pld) != (rows, cols, ld) or W_pruned.dtype != W.dtype:
+            raise ValueError("W_pruned must have W's shape, dtype and row pitch")
+    code = load().dass_score_nm(W.data_ptr(), rows, cols, ld, _dtype_code(W), norm.data_ptr(), int(norm_axis),
+                                float(alpha), int(n_keep), int(m), int(group_axis),
+                                _ptr(mask_bits), _ptr(W_pruned), _stream(stream))
+    _check(code, "dass_score_nm")
+    return mask_bits, W_pruned
+
+
+def compress_shapes(rows: int, cols: int, n_keep: int, m: int, group_axis: int):
+    """((value rows, value cols), (meta lines, meta words per line))."""
+    bits = 4 if (n_keep == 2 and m == 4) else m
+    fpw = 32 // bits
+    if group_axis == AXIS_COLS:
+        return (rows, cols // m * n_keep), (rows, (cols // m + fpw - 1) // fpw)
+    return (rows // m * n_keep, cols), (rows // m, (cols + fpw - 1) // fpw)
+
+
+def compress_nm(W: torch.Tensor, mask_bits: torch.Tensor, n_keep: int, m: int, group_axis: int,
+                values: Optional[torch.Tensor] = None, meta: Optional[torch.Tensor] = None,
+                stream: Optional[torch.cuda.Stream] = None):
+    """Compressed values + metadata of W under mask_bits. Returns (values, meta)."""
+    rows, cols, ld = _matrix(W, "W")
+    vshape, mshape = compress_shapes(rows, cols, n_keep, m, group_axis)
+    if values is None:
+        values = torch.empty(vshape, dtype=W.dtype, device=W.device)
+    if meta is None:
+        meta = torch.empty(mshape, dtype=torch.int32, device=W.device)
+    if tuple(values.shape) != vshape or not values.is_contiguous() or values.dtype != W.dtype:
+        raise ValueError(f"values must be a contiguous {vshape} tensor of W's dtype")
+    if tuple(meta.shape) != mshape or not meta.is_contiguous() or meta.dtype != torch.int32:
+        raise ValueError(f"meta must be a contiguous int32 {mshape} tensor")
+    if mask_bits.dtype != torch.int32 or not mask_bits.is_contiguous() or \
+            tuple(mask_bits.shape) != (rows, mask_words_per_row(cols)):
+        raise ValueError("mask_bits must be the contiguous int32 [rows x ceil(cols/32)] tensor score_nm produced")
+    code = load().dass_compress_nm(W.data_ptr(), mask_bits.data_ptr(), rows, cols, ld, _dtype_code(W),
+                                   int(n_keep), int(m), int(group_axis), values.data_ptr(), meta.data_ptr(),
+                                   _stream(stream))
+    _check(code, "dass_compress_nm")
+    return values, meta

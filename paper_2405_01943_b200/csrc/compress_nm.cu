@@ -1,0 +1,293 @@
+// Stage (b), last step: N:M compressed values + metadata from the weights and the packed mask.
+//
+// Same tiling as the scoring pass (a warp owns 32 rows x 256 columns, a lane 8 consecutive columns),
+// so weight loads and value stores stay 128-bit and coalesced for either group axis.  Metadata
+// fields are produced in registers and packed into 32-bit words with warp shuffles (groups along the
+// columns: four lanes share a word) or directly per lane (groups along the rows: a lane's 8 columns
+// fill whole words).  Bandwidth-bound: reads W and one mask bit per weight, writes n_keep/m of W plus
+// the fields.
+#include "dass_device.cuh"
+
+namespace dass {
+
+struct CompressParams {
+    const void *W;
+    const uint32_t *mask;
+    void *values;
+    uint32_t *meta;
+    int64_t rows, cols, ld;
+    int64_t wpr;          // mask words per row
+    int64_t vcols;        // columns of the values matrix
+    int64_t mwpl;         // metadata words per line
+    int64_t col_blocks, row_blocks;
+    int n_keep;
+    int vec_ok;           // values rows are 16-byte aligned: vector stores allowed
+};
+
+constexpr int C_TILE_ROWS = 32;
+constexpr int C_TILE_COLS = 256;
+constexpr int C_THREADS = 256;
+
+// Raw bits of element j of a chunk, j only known at run time (select chain, no local memory).
+template <bool BF16>
+__device__ __forceinline__ uint32_t chunk_bits_dyn(const Chunk<BF16> &c, int j)
+{
+    if constexpr (BF16) {
+        const uint32_t a = (j & 2) ? c.w[1] : c.w[0];
+        const uint32_t b = (j & 2) ? c.w[3] : c.w[2];
+        const uint32_t w = (j & 4) ? b : a;
+        return (j & 1) ? (w >> 16) : (w & 0xffffu);
+    } else {
+        const uint32_t a = (j & 1) ? c.w[1] : c.w[0];
+        const uint32_t b = (j & 1) ? c.w[3] : c.w[2];
+        const uint32_t d = (j & 1) ? c.w[5] : c.w[4];
+        const uint32_t e = (j & 1) ? c.w[7] : c.w[6];
+        const uint32_t ab = (j & 2) ? b : a;
+        const uint32_t de = (j & 2) ? e : d;
+        return (j & 4) ? de : ab;
+    }
+}
+
+template <bool BF16>
+__device__ __forceinline__ void chunk_set(Chunk<BF16> &c, int j /* compile-time after unrolling */, uint32_t bits)
+{
+    if constexpr (BF16) {
+        if (j & 1) c.w[j >> 1] = (c.w[j >> 1] & 0x0000ffffu) | (bits << 16);
+        else c.w[j >> 1] = (c.w[j >> 1] & 0xffff0000u) | (bits & 0xffffu);
+    } else {
+        c.w[j] = bits;
+    }
+}
+
+// Stores the first n elements of a chunk at element offset `off`; vector stores only if the
+// destination is known to be 16-byte aligned (vec) and the piece is a whole vector.
+template <bool BF16>
+__device__ __forceinline__ void chunk_store_n(const Chunk<BF16> &c, void *base, int64_t off, int n, bool vec)
+{
+    if constexpr (BF16) {
+        uint16_t *p = static_cast<uint16_t *>(base) + off;
+        if (vec && n == 8) {
+            __stcs(reinterpret_cast<uint4 *>(p), make_uint4(c.w[0], c.w[1], c.w[2], c.w[3]));
+        } else if (vec && n == 4) {
+            __stcs(reinterpret_cast<uint2 *>(p), make_uint2(c.w[0], c.w[1]));
+        } else {
+            for (int j = 0; j < n; ++j) p[j] = (uint16_t)chunk_bits_dyn<true>(c, j);
+        }
+    } else {
+        uint32_t *p = static_cast<uint32_t *>(base) + off;
+        if (vec && n == 8) {
+            __stcs(reinterpret_cast<uint4 *>(p), make_uint4(c.w[0], c.w[1], c.w[2], c.w[3]));
+            __stcs(reinterpret_cast<uint4 *>(p) + 1, make_uint4(c.w[4], c.w[5], c.w[6], c.w[7]));
+        } else if (vec && n == 4) {
+            __stcs(reinterpret_cast<uint4 *>(p), make_uint4(c.w[0], c.w[1], c.w[2], c.w[3]));
+        } else {
+            for (int j = 0; j < n; ++j) p[j] = chunk_bits_dyn<false>(c, j);
+        }
+    }
+}
+
+// Position (0-based) of the k-th (0-based) set bit of x; x has more than k bits set.
+__device__ __forceinline__ int nth_set_bit(uint32_t x, int k)
+{
+    for (int i = 0; i < k; ++i) x &= x - 1;
+    return __ffs(x) - 1;
+}
+
+// ---------------------------------------------------------------- groups along the columns
+template <bool BF16, int M, bool TWO_FOUR>
+__global__ void __launch_bounds__(C_THREADS) compress_group_cols_kernel(const CompressParams p)
+{
+    const int lane = threadIdx.x & 31;
+    const int64_t warp = (int64_t)blockIdx.x * (C_THREADS / 32) + (threadIdx.x >> 5);
+    const int64_t nwarps = (int64_t)gridDim.x * (C_THREADS / 32);
+    const int64_t ntasks = p.col_blocks * p.row_blocks;
+    constexpr int UNROLL = 4;
+
+    for (int64_t task = warp; task < ntasks; task += nwarps) {
+        const int64_t cb = task % p.col_blocks;
+        const int64_t rb = task / p.col_blocks;
+        const int64_t c0 = cb * C_TILE_COLS + lane * 8;
+        const int64_t left = p.cols - c0;
+        const int nvalid = left >= 8 ? 8 : (left > 0 ? (int)left : 0);   // a multiple of M
+        const int nout = nvalid / M * p.n_keep;                           // values this lane emits per row
+
+        for (int i = 0; i < C_TILE_ROWS; i += UNROLL) {
+            const int64_t rbase = rb * C_TILE_ROWS + i;
+            if (rbase >= p.rows) break;
+            Chunk<BF16> ch[UNROLL];
+            uint32_t mbyte[UNROLL];
+#pragma unroll
+            for (int u = 0; u < UNROLL; ++u) {
+                if (rbase + u < p.rows && nvalid > 0) {
+                    chunk_load<BF16>(ch[u], p.W, (rbase + u) * p.ld + c0, nvalid);
+                    mbyte[u] = (__ldg(p.mask + (rbase + u) * p.wpr + (c0 >> 5)) >> (8 * (lane & 3))) & 0xffu;
+                } else {
+                    chunk_zero<BF16>(ch[u]);
+                    mbyte[u] = 0u;
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < UNROLL; ++u) {
+                const int64_t r = rbase + u;
+                Chunk<BF16> out;
+                chunk_zero<BF16>(out);
+                uint32_t field_byte;
+                if constexpr (TWO_FOUR) {
+                    field_byte = 0u;
+#pragma unroll
+                    for (int g = 0; g < 2; ++g) {
+                        const uint32_t nib = (mbyte[u] >> (4 * g)) & 0xfu;
+                        const int lo = nib ? __ffs(nib) - 1 : 0;
+                        const int hi = nib ? 31 - __clz(nib) : 0;
+                        chunk_set<BF16>(out, 2 * g, chunk_bits_dyn<BF16>(ch[u], 4 * g + lo));
+                        chunk_set<BF16>(out, 2 * g + 1, chunk_bits_dyn<BF16>(ch[u], 4 * g + hi));
+                        field_byte |= (uint32_t)(lo | (hi << 2)) << (4 * g);
+                    }
+                } else {
+                    field_byte = mbyte[u];   // the m-bit keep masks, already in place
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) {
+                        if (k < nout) {
+                            const int g = k / p.n_keep, q = k % p.n_keep;
+                            const uint32_t gm = (mbyte[u] >> (g * M)) & ((1u << M) - 1u);
+                            chunk_set<BF16>(out, k, chunk_bits_dyn<BF16>(ch[u], g * M + nth_set_bit(gm, q)));
+                        }
+                    }
+                }
+                const uint32_t word = quad_pack_bytes(field_byte, lane);
+                if (r < p.rows && nvalid > 0) {
+                    if ((lane & 3) == 0) p.meta[r * p.mwpl + (c0 >> 5)] = word;
+                    chunk_store_n<BF16>(out, p.values, r * p.vcols + c0 / M * p.n_keep, nout, p.vec_ok != 0);
+                }
+            }
+        }
+    }
+}
+
+// ---------------------------------------------------------------- groups along the rows
+template <bool BF16, int M, bool TWO_FOUR>
+__global__ void __launch_bounds__(C_THREADS) compress_group_rows_kernel(const CompressParams p)
+{
+    const int lane = threadIdx.x & 31;
+    const int64_t warp = (int64_t)blockIdx.x * (C_THREADS / 32) + (threadIdx.x >> 5);
+    const int64_t nwarps = (int64_t)gridDim.x * (C_THREADS / 32);
+    const int64_t ntasks = p.col_blocks * p.row_blocks;
+    constexpr int MAXK = TWO_FOUR ? 2 : M - 1;   // survivors per group that can occur
+
+    for (int64_t task = warp; task < ntasks; task += nwarps) {
+        const int64_t cb = task % p.col_blocks;
+        const int64_t rb = task / p.col_blocks;
+        const int64_t c0 = cb * C_TILE_COLS + lane * 8;
+        const int64_t left = p.cols - c0;
+        const int nvalid = left >= 8 ? 8 : (left > 0 ? (int)left : 0);
+        if (nvalid == 0) continue;   // no shuffles in this kernel: lanes are independent
+
+        for (int g = 0; g < C_TILE_ROWS / M; ++g) {
+            const int64_t r0 = rb * C_TILE_ROWS + g * M;
+            if (r0 >= p.rows) break;
+            const int64_t line = r0 / M;
+            Chunk<BF16> ch[M];
+            uint32_t mbyte[M];
+#pragma unroll
+            for (int q = 0; q < M; ++q) {
+                chunk_load<BF16>(ch[q], p.W, (r0 + q) * p.ld + c0, nvalid);
+                mbyte[q] = (__ldg(p.mask + (r0 + q) * p.wpr + (c0 >> 5)) >> (8 * (lane & 3))) & 0xffu;
+            }
+            Chunk<BF16> out[MAXK];
+#pragma unroll
+            for (int k = 0; k < MAXK; ++k) chunk_zero<BF16>(out[k]);
+            uint32_t fields_lo = 0u, fields_hi = 0u;   // packed fields of columns 0..3 / 4..7 (or all 8 in lo)
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                uint32_t colmask = 0u;   // bit q: row r0+q kept at column c0+j
+#pragma unroll
+                for (int q = 0; q < M; ++q) colmask |= ((mbyte[q] >> j) & 1u) << q;
+                if constexpr (TWO_FOUR) {
+                    const int lo = colmask ? __ffs(colmask) - 1 : 0;
+                    const int hi = colmask ? 31 - __clz(colmask) : 0;
+                    const uint32_t v_lo = lo == 0 ? chunk_bits<BF16>(ch[0], j) : lo == 1 ? chunk_bits<BF16>(ch[1], j)
+                                        : lo == 2 ? chunk_bits<BF16>(ch[2], j) : chunk_bits<BF16>(ch[3], j);
+                    const uint32_t v_hi = hi == 0 ? chunk_bits<BF16>(ch[0], j) : hi == 1 ? chunk_bits<BF16>(ch[1], j)
+                                        : hi == 2 ? chunk_bits<BF16>(ch[2], j) : chunk_bits<BF16>(ch[3], j);
+                    chunk_set<BF16>(out[0], j, v_lo);
+                    chunk_set<BF16>(out[1], j, v_hi);
+                    fields_lo |= (uint32_t)(lo | (hi << 2)) << (4 * j);
+                } else {
+#pragma unroll
+                    for (int k = 0; k < MAXK; ++k) {
+                        if (k < p.n_keep) {
+                            const int pos = nth_set_bit(colmask, k);
+                            uint32_t v = 0u;
+#pragma unroll
+                            for (int q = 0; q < M; ++q) v = pos == q ? chunk_bits<BF16>(ch[q], j) : v;
+                            chunk_set<BF16>(out[k], j, v);
+                        }
+                    }
+                    if constexpr (M == 4) fields_lo |= colmask << (4 * j);
+                    else if (j < 4) fields_lo |= colmask << (8 * j);
+                    else fields_hi |= colmask << (8 * (j - 4));
+                }
+            }
+            if constexpr (TWO_FOUR || M == 4) {
+                p.meta[line * p.mwpl + (c0 >> 3)] = fields_lo;
+            } else {
+                p.meta[line * p.mwpl + (c0 >> 2)] = fields_lo;
+                if (nvalid > 4) p.meta[line * p.mwpl + (c0 >> 2) + 1] = fields_hi;
+            }
+#pragma unroll
+            for (int k = 0; k < MAXK; ++k)
+                if (k < p.n_keep)
+                    chunk_store_n<BF16>(out[k], p.values, (line * p.n_keep + k) * p.vcols + c0, nvalid, p.vec_ok != 0);
+        }
+    }
+}
+
+template <bool BF16, int M, bool TWO_FOUR>
+static cudaError_t launch_compress(const CompressParams &p, bool group_cols, int grid, cudaStream_t st)
+{
+    if (group_cols) compress_group_cols_kernel<BF16, M, TWO_FOUR><<<grid, C_THREADS, 0, st>>>(p);
+    else compress_group_rows_kernel<BF16, M, TWO_FOUR><<<grid, C_THREADS, 0, st>>>(p);
+    return cudaGetLastError();
+}
+
+int device_sm_count();   // dass_abi.cu
+
+cudaError_t compress_nm_launch(const void *W, const uint32_t *mask_bits, int64_t rows, int64_t cols, int64_t ld,
+                               bool bf16, int n_keep, int m, bool group_cols,
+                               void *values, uint32_t *meta, cudaStream_t st)
+{
+    CompressParams p;
+    p.W = W; p.mask = mask_bits; p.values = values; p.meta = meta;
+    p.rows = rows; p.cols = cols; p.ld = ld;
+    p.wpr = (cols + 31) / 32;
+    const bool two_four = (n_keep == 2 && m == 4);
+    const int field_bits = two_four ? 4 : m;
+    const int fpw = 32 / field_bits;
+    if (group_cols) {
+        p.vcols = cols / m * n_keep;
+        p.mwpl = (cols / m + fpw - 1) / fpw;
+    } else {
+        p.vcols = cols;
+        p.mwpl = (cols + fpw - 1) / fpw;
+    }
+    const int esz = bf16 ? 2 : 4;
+    p.vec_ok = ((p.vcols * esz) % 16 == 0) && ((reinterpret_cast<uintptr_t>(values) & 15u) == 0);
+    p.col_blocks = (cols + C_TILE_COLS - 1) / C_TILE_COLS;
+    p.row_blocks = (rows + C_TILE_ROWS - 1) / C_TILE_ROWS;
+    p.n_keep = n_keep;
+    const int64_t ntasks = p.col_blocks * p.row_blocks;
+    const int64_t wpb = C_THREADS / 32;
+    const int64_t want = (ntasks + wpb - 1) / wpb;
+    const int64_t cap = (int64_t)device_sm_count() * 8;
+    const int grid = (int)(want < cap ? want : cap);
+    if (bf16) {
+        if (two_four) return launch_compress<true, 4, true>(p, group_cols, grid, st);
+        return m == 4 ? launch_compress<true, 4, false>(p, group_cols, grid, st)
+                      : launch_compress<true, 8, false>(p, group_cols, grid, st);
+    }
+    if (two_four) return launch_compress<false, 4, true>(p, group_cols, grid, st);
+    return m == 4 ? launch_compress<false, 4, false>(p, group_cols, grid, st)
+                  : launch_compress<false, 8, false>(p, group_cols, grid, st);
+}
+
+}  // namespace dass

@@ -1,0 +1,184 @@
+// C ABI of the DaSS CUDA library: argument validation and dispatch only.  See include/dass.h.
+#include <cmath>
+#include <cstdint>
+
+#include "dass_device.cuh"
+
+namespace dass {
+
+// kernels' host launchers (defined beside the kernels)
+cudaError_t score_nm_launch(const void *W, int64_t rows, int64_t cols, int64_t ld, bool bf16,
+                            const float *norm, bool norm_cols, float alpha, int n_keep, int m, bool group_cols,
+                            uint32_t *mask_bits, void *W_pruned, cudaStream_t st);
+cudaError_t compress_nm_launch(const void *W, const uint32_t *mask_bits, int64_t rows, int64_t cols, int64_t ld,
+                               bool bf16, int n_keep, int m, bool group_cols,
+                               void *values, uint32_t *meta, cudaStream_t st);
+int64_t calib_simt_parts(int64_t T);
+cudaError_t calib_simt_launch(const float *X, int64_t T, int64_t ldx, const float *Wg, const float *Wu,
+                              int64_t I, int64_t d, int64_t ldw, int act, double *partial, cudaStream_t st);
+cudaError_t calib_reduce_launch(const double *partial, int64_t parts, int64_t I, double *sumsq, cudaStream_t st);
+cudaError_t norm_finalize_launch(const double *sumsq, int64_t I, float *norm, cudaStream_t st);
+cudaError_t status_clear_launch(int *status, cudaStream_t st);
+int64_t calib_tc_parts(int64_t T, int64_t I);
+dass_status calib_tc_launch(const void *X, int64_t T, int64_t ldx, const void *Wg, const void *Wu,
+                            int64_t I, int64_t d, int64_t ldw, int act, double *partial, int *status,
+                            cudaStream_t st);
+
+int device_sm_count()
+{
+    static int cached_dev = -1, cached_sms = 0;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 148;
+    if (dev != cached_dev) {
+        int sms = 0;
+        if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) sms = 148;
+        cached_sms = sms;
+        cached_dev = dev;
+    }
+    return cached_sms;
+}
+
+constexpr size_t WS_HEADER = 256;   // status word + padding; partial sums start here
+
+static inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+static inline bool ld_ok(int64_t ld, bool bf16) { return ld % (bf16 ? 8 : 4) == 0; }
+
+static dass_status check_nm(int64_t rows, int64_t cols, int64_t ld, int dt, int n_keep, int m, int group_axis)
+{
+    if (dt != DASS_BF16 && dt != DASS_F32) return DASS_ERR_DTYPE;
+    if (group_axis != DASS_AXIS_ROWS && group_axis != DASS_AXIS_COLS) return DASS_ERR_DTYPE;
+    if (rows < 1 || cols < 1 || ld < cols) return DASS_ERR_SHAPE;
+    if (m != 4 && m != 8) return (m >= 2 && m <= 64) ? DASS_ERR_UNSUPPORTED : DASS_ERR_SHAPE;
+    if (n_keep < 1 || n_keep >= m) return DASS_ERR_SHAPE;
+    const int64_t extent = group_axis == DASS_AXIS_ROWS ? rows : cols;
+    if (extent % m != 0) return DASS_ERR_SHAPE;
+    if (!ld_ok(ld, dt == DASS_BF16)) return DASS_ERR_ALIGN;
+    return DASS_OK;
+}
+
+}  // namespace dass
+
+using namespace dass;
+
+extern "C" {
+
+const char *dass_status_string(dass_status s)
+{
+    switch (s) {
+    case DASS_OK: return "ok";
+    case DASS_ERR_NULL: return "null pointer";
+    case DASS_ERR_SHAPE: return "bad shape";
+    case DASS_ERR_ALIGN: return "bad alignment";
+    case DASS_ERR_DTYPE: return "bad enum value";
+    case DASS_ERR_UNSUPPORTED: return "unsupported";
+    case DASS_ERR_WORKSPACE: return "workspace too small";
+    case DASS_ERR_CUDA: return "CUDA error";
+    case DASS_ERR_TIMEOUT: return "device-side wait timed out";
+    }
+    return "unknown status";
+}
+
+int dass_version(void) { return 100; }
+
+dass_status dass_calib_workspace_bytes(int64_t T, int64_t d, int64_t I, dass_dtype dt, size_t *bytes)
+{
+    if (!bytes) return DASS_ERR_NULL;
+    if (dt != DASS_BF16 && dt != DASS_F32) return DASS_ERR_DTYPE;
+    if (T < 1 || d < 1 || I < 1) return DASS_ERR_SHAPE;
+    const int64_t parts = dt == DASS_BF16 ? calib_tc_parts(T, I) : calib_simt_parts(T);
+    *bytes = WS_HEADER + (size_t)parts * (size_t)I * sizeof(double);
+    return DASS_OK;
+}
+
+dass_status dass_calib_accumulate(const void *X, int64_t T, int64_t ldx,
+                                  const void *Wg, const void *Wu, int64_t I, int64_t d, int64_t ldw,
+                                  dass_dtype dt, dass_act act, double *sumsq,
+                                  void *workspace, size_t workspace_bytes, void *cuda_stream)
+{
+    if (!X || !Wg || !Wu || !sumsq) return DASS_ERR_NULL;
+    if (dt != DASS_BF16 && dt != DASS_F32) return DASS_ERR_DTYPE;
+    if (act != DASS_ACT_SILU && act != DASS_ACT_GELU_TANH && act != DASS_ACT_RELU) return DASS_ERR_DTYPE;
+    if (T < 1 || d < 1 || I < 1 || ldx < d || ldw < d) return DASS_ERR_SHAPE;
+    const bool bf16 = dt == DASS_BF16;
+    if (!aligned16(X) || !aligned16(Wg) || !aligned16(Wu) || !ld_ok(ldx, bf16) || !ld_ok(ldw, bf16)) return DASS_ERR_ALIGN;
+    if ((reinterpret_cast<uintptr_t>(sumsq) & 7u) != 0) return DASS_ERR_ALIGN;
+    size_t need = 0;
+    const dass_status qs = dass_calib_workspace_bytes(T, d, I, dt, &need);
+    if (qs != DASS_OK) return qs;
+    if (!workspace || workspace_bytes < need) return DASS_ERR_WORKSPACE;
+    if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return DASS_ERR_ALIGN;
+
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    int *status = static_cast<int *>(workspace);
+    double *partial = reinterpret_cast<double *>(static_cast<char *>(workspace) + WS_HEADER);
+    if (status_clear_launch(status, st) != cudaSuccess) return DASS_ERR_CUDA;
+    int64_t parts;
+    if (bf16) {
+        parts = calib_tc_parts(T, I);
+        const dass_status ts = calib_tc_launch(X, T, ldx, Wg, Wu, I, d, ldw, (int)act, partial, status, st);
+        if (ts != DASS_OK) return ts;
+    } else {
+        parts = calib_simt_parts(T);
+        if (calib_simt_launch(static_cast<const float *>(X), T, ldx, static_cast<const float *>(Wg),
+                              static_cast<const float *>(Wu), I, d, ldw, (int)act, partial, st) != cudaSuccess)
+            return DASS_ERR_CUDA;
+    }
+    if (calib_reduce_launch(partial, parts, I, sumsq, st) != cudaSuccess) return DASS_ERR_CUDA;
+    return DASS_OK;
+}
+
+dass_status dass_calib_status(const void *workspace, void *cuda_stream)
+{
+    if (!workspace) return DASS_ERR_NULL;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    int host = 0;
+    if (cudaMemcpyAsync(&host, workspace, sizeof(int), cudaMemcpyDeviceToHost, st) != cudaSuccess) return DASS_ERR_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return DASS_ERR_CUDA;
+    return host == 0 ? DASS_OK : DASS_ERR_TIMEOUT;
+}
+
+dass_status dass_norm_finalize(const double *sumsq, int64_t I, float *norm, void *cuda_stream)
+{
+    if (!sumsq || !norm) return DASS_ERR_NULL;
+    if (I < 1) return DASS_ERR_SHAPE;
+    if (norm_finalize_launch(sumsq, I, norm, static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) return DASS_ERR_CUDA;
+    return DASS_OK;
+}
+
+dass_status dass_score_nm(const void *W, int64_t rows, int64_t cols, int64_t ld, dass_dtype dt,
+                          const float *norm, dass_axis norm_axis, float alpha,
+                          int n_keep, int m, dass_axis group_axis,
+                          uint32_t *mask_bits, void *W_pruned, void *cuda_stream)
+{
+    if (!W || !norm || (!mask_bits && !W_pruned)) return DASS_ERR_NULL;
+    if (norm_axis != DASS_AXIS_ROWS && norm_axis != DASS_AXIS_COLS) return DASS_ERR_DTYPE;
+    const dass_status cs = check_nm(rows, cols, ld, (int)dt, n_keep, m, (int)group_axis);
+    if (cs != DASS_OK) return cs;
+    if (!std::isfinite(alpha) || alpha < 0.0f) return DASS_ERR_UNSUPPORTED;
+    if (!aligned16(W) || (W_pruned && !aligned16(W_pruned))) return DASS_ERR_ALIGN;
+    if ((reinterpret_cast<uintptr_t>(norm) & 3u) || (reinterpret_cast<uintptr_t>(mask_bits) & 3u)) return DASS_ERR_ALIGN;
+    if (score_nm_launch(W, rows, cols, ld, dt == DASS_BF16, norm, norm_axis == DASS_AXIS_COLS, alpha, n_keep, m,
+                        group_axis == DASS_AXIS_COLS, mask_bits, W_pruned,
+                        static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
+        return DASS_ERR_CUDA;
+    return DASS_OK;
+}
+
+dass_status dass_compress_nm(const void *W, const uint32_t *mask_bits,
+                             int64_t rows, int64_t cols, int64_t ld, dass_dtype dt,
+                             int n_keep, int m, dass_axis group_axis,
+                             void *values, uint32_t *meta, void *cuda_stream)
+{
+    if (!W || !mask_bits || !values || !meta) return DASS_ERR_NULL;
+    const dass_status cs = check_nm(rows, cols, ld, (int)dt, n_keep, m, (int)group_axis);
+    if (cs != DASS_OK) return cs;
+    if (!aligned16(W)) return DASS_ERR_ALIGN;
+    if ((reinterpret_cast<uintptr_t>(mask_bits) & 3u) || (reinterpret_cast<uintptr_t>(meta) & 3u)) return DASS_ERR_ALIGN;
+    if (reinterpret_cast<uintptr_t>(values) & (dt == DASS_BF16 ? 1u : 3u)) return DASS_ERR_ALIGN;
+    if (compress_nm_launch(W, mask_bits, rows, cols, ld, dt == DASS_BF16, n_keep, m, group_axis == DASS_AXIS_COLS,
+                           values, meta, static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
+        return DASS_ERR_CUDA;
+    return DASS_OK;
+}
+
+}  // extern "C"
