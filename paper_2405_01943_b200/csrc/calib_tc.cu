@@ -1,7 +1,418 @@
-// placeholder until the tensor-core kernel lands
+// Stage (a) for bf16 inputs: Eq. 2 and the per-neuron sum of squares on the sm_100a tensor cores.
+//
+//   G = Wg_tile . X_tile^T,  U = Wu_tile . X_tile^T      (tcgen05.mma, bf16 x bf16 -> fp32 in TMEM)
+//   sumsq[neuron] += sum over the tile's tokens of ( act(G) * U )^2                (fused epilogue)
+//
+// Neurons are the MMA M dimension (128 per tile = the 128 TMEM lanes), tokens the N dimension (256
+// per tile), so one epilogue thread owns one neuron and adds up its tokens serially in registers --
+// no shuffles, no atomics -- and the intermediate activation H never reaches memory.  The gate and up
+// tiles are two A operands that share one B operand (the X tile).
+//
+// One persistent CTA per SM, warp-specialised:
+//   warp 0      TMA producer: X / Wg / Wu k-slices into a 3-stage, 128B-swizzled shared-memory ring
+//   warp 1      allocates TMEM, issues the MMAs (one lane), commits ring slots and accumulators
+//   warps 2..5  epilogue: tcgen05.ld the two accumulators, activation, gating product, square, sum
+// A work item is (neuron tile, band of up to 16 token tiles); items are ordered so that the CTAs
+// running at the same moment share a few X tiles and a few W tiles through L2.  Every item writes one
+// partial per neuron to partial[band][neuron]; a second tiny kernel adds the bands in a fixed order.
+//
+// Every wait on an mbarrier is bounded: when a wait runs out the CTA raises an abort flag, records
+// DASS_ERR_TIMEOUT in the status word, lets its roles drain and frees its TMEM before returning.
+#include <cuda.h>
+
 #include "dass_device.cuh"
+
 namespace dass {
-int64_t calib_tc_parts(int64_t T, int64_t I) { (void)I; (void)T; return 1; }
-dass_status calib_tc_launch(const void *, int64_t, int64_t, const void *, const void *, int64_t, int64_t, int64_t, int,
-                            double *, int *, cudaStream_t) { return DASS_ERR_UNSUPPORTED; }
+
+constexpr int TC_BM = 128;         // neurons per tile (MMA M, TMEM lanes)
+constexpr int TC_BN = 256;         // tokens per tile (MMA N)
+constexpr int TC_BK = 64;          // k per ring slot: 64 bf16 = one 128-byte swizzle row
+constexpr int TC_UMMA_K = 16;      // k per tcgen05.mma for 16-bit inputs
+constexpr int TC_STAGES = 3;
+constexpr int TC_BAND_TILES = 16;  // token tiles per band (one partial per band and neuron)
+constexpr int TC_SUPER_BANDS = 16; // bands interleaved in the item order for L2 sharing
+constexpr int TC_THREADS = 192;
+constexpr uint32_t TC_W_BYTES = TC_BM * TC_BK * 2;                 // 16 KB
+constexpr uint32_t TC_X_BYTES = TC_BN * TC_BK * 2;                 // 32 KB
+constexpr uint32_t TC_STAGE_BYTES = 2 * TC_W_BYTES + TC_X_BYTES;   // 64 KB
+constexpr uint32_t TC_TMEM_COLS = 512;                             // G: columns 0..255, U: 256..511
+constexpr uint32_t TC_SMEM_BYTES = TC_STAGES * TC_STAGE_BYTES + 1024 /* alignment slack */ + 256 /* barriers */;
+constexpr unsigned long long TC_WAIT_NS = 2000000000ull;           // a wait gives up after 2 s
+
+// ------------------------------------------------------------------ PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
 }
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile("{\n\t.reg .pred p;\n\t"
+                 "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+                 "selp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ unsigned long long global_ns()
+{
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
+// Bounded wait: true when the phase completed, false after TC_WAIT_NS (or when another role aborted).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    const unsigned long long t0 = global_ns();
+    for (uint32_t spin = 1; spin < (1u << 30); ++spin) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((spin & 255u) == 0) {
+            if (*abort_flag) return false;
+            if (global_ns() - t0 > TC_WAIT_NS) return false;
+        }
+    }
+    return false;
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int x, int y)
+{
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+                 ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(x), "r"(y) : "memory");
+}
+__device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t ncols)
+{
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish()
+{
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols)
+{
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile("{\n\t.reg .pred p;\n\t"
+                 "setp.ne.b32 p, %4, 0;\n\t"
+                 "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+                 ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld_32(uint32_t taddr, uint32_t (&r)[32])
+{
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+                 "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+                 "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+                   "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+                   "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+                   "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+                 : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor of a K-major tile whose rows are 128 bytes (64 bf16) and which was
+// written by TMA with the 128-byte swizzle: 8-row groups 1024 bytes apart, descriptor version 1.
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr)
+{
+    return (uint64_t)((addr & 0x3ffffu) >> 4) | (1ull << 16) | ((uint64_t)(1024 >> 4) << 32) | (1ull << 46) | (2ull << 61);
+}
+// tcgen05 instruction descriptor: D = fp32, A = B = bf16, both K-major, shape M x N.
+__host__ __device__ constexpr uint32_t idesc_bf16_f32(int m, int n)
+{
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
+}
+
+template <int ACT>
+__device__ __forceinline__ float glu_h(float g, float u)
+{
+    if constexpr (ACT == DASS_ACT_SILU) {
+        // g * sigmoid(g) * u
+        return __fdividef(g * u, 1.0f + __expf(-g));
+    } else if constexpr (ACT == DASS_ACT_GELU_TANH) {
+        // 0.5 (1 + tanh z) = sigmoid(2 z),  z = sqrt(2/pi) (g + 0.044715 g^3)
+        const float z2 = 1.5957691216057308f * g * fmaf(0.044715f * g, g, 1.0f);
+        return __fdividef(g * u, 1.0f + __expf(-z2));
+    } else {
+        return fmaxf(g, 0.0f) * u;
+    }
+}
+
+struct TcParams {
+    double *partial;     // [bands][I]
+    int *status;
+    int64_t T, I, d;
+    int64_t neuron_tiles, token_tiles, bands, items, k_blocks;
+};
+
+struct ItemCoord { int64_t nt, band; };
+
+__device__ __forceinline__ ItemCoord decode_item(const TcParams &p, int64_t idx)
+{
+    const int64_t per_super = p.neuron_tiles * TC_SUPER_BANDS;
+    const int64_t sb = idx / per_super;
+    const int64_t rem = idx - sb * per_super;
+    const int64_t left = p.bands - sb * TC_SUPER_BANDS;
+    const int64_t nb = left < TC_SUPER_BANDS ? left : TC_SUPER_BANDS;
+    ItemCoord c;
+    c.nt = rem / nb;
+    c.band = sb * TC_SUPER_BANDS + (rem - c.nt * nb);
+    return c;
+}
+
+template <int ACT>
+__global__ void __launch_bounds__(TC_THREADS, 1)
+calib_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_wg,
+                const __grid_constant__ CUtensorMap map_wu, const TcParams p)
+{
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;                 // swizzled tiles need 1024-byte alignment
+    uint8_t *aligned = smem_raw + (base - raw);
+    uint64_t *bars = reinterpret_cast<uint64_t *>(aligned + TC_STAGES * TC_STAGE_BYTES);
+    const uint32_t bar_full = smem_u32(bars);                     // [TC_STAGES]
+    const uint32_t bar_empty = bar_full + 8 * TC_STAGES;          // [TC_STAGES]
+    const uint32_t bar_acc_full = bar_empty + 8 * TC_STAGES;
+    const uint32_t bar_acc_empty = bar_acc_full + 8;
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * TC_STAGES + 2);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < TC_STAGES; ++s) {
+            mbar_init(bar_full + 8 * s, 1);
+            mbar_init(bar_empty + 8 * s, 1);
+        }
+        mbar_init(bar_acc_full, 1);
+        mbar_init(bar_acc_empty, 4);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) {
+        tmem_alloc(smem_u32(tmem_slot), TC_TMEM_COLS);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            uint32_t stage = 0, phase = 0;
+            bool ok = true;
+            for (int64_t idx = blockIdx.x; idx < p.items && ok; idx += gridDim.x) {
+                const ItemCoord c = decode_item(p, idx);
+                const int64_t tt0 = c.band * TC_BAND_TILES;
+                const int64_t tt1 = tt0 + TC_BAND_TILES < p.token_tiles ? tt0 + TC_BAND_TILES : p.token_tiles;
+                for (int64_t tt = tt0; tt < tt1 && ok; ++tt) {
+                    for (int64_t kb = 0; kb < p.k_blocks; ++kb) {
+                        if (!mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
+                        const uint32_t sbase = base + stage * TC_STAGE_BYTES;
+                        const uint32_t fb = bar_full + 8 * stage;
+                        mbar_arrive_expect_tx(fb, TC_STAGE_BYTES);
+                        tma_load_2d(sbase, &map_wg, fb, (int)(kb * TC_BK), (int)(c.nt * TC_BM));
+                        tma_load_2d(sbase + TC_W_BYTES, &map_wu, fb, (int)(kb * TC_BK), (int)(c.nt * TC_BM));
+                        tma_load_2d(sbase + 2 * TC_W_BYTES, &map_x, fb, (int)(kb * TC_BK), (int)(tt * TC_BN));
+                        if (++stage == TC_STAGES) { stage = 0; phase ^= 1u; }
+                    }
+                }
+            }
+            if (!ok) { *abort_flag = 1; atomicExch(p.status, (int)DASS_ERR_TIMEOUT); }
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        // ------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            constexpr uint32_t idesc = idesc_bf16_f32(TC_BM, TC_BN);
+            uint32_t stage = 0, phase = 0, tile = 0;
+            bool ok = true;
+            for (int64_t idx = blockIdx.x; idx < p.items && ok; idx += gridDim.x) {
+                const ItemCoord c = decode_item(p, idx);
+                const int64_t tt0 = c.band * TC_BAND_TILES;
+                const int64_t tt1 = tt0 + TC_BAND_TILES < p.token_tiles ? tt0 + TC_BAND_TILES : p.token_tiles;
+                for (int64_t tt = tt0; tt < tt1 && ok; ++tt, ++tile) {
+                    // the epilogue must have drained the previous tile's accumulators
+                    if (!mbar_wait(bar_acc_empty, (tile & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+                    tc_fence_after();
+                    for (int64_t kb = 0; kb < p.k_blocks; ++kb) {
+                        if (!mbar_wait(bar_full + 8 * stage, phase, abort_flag)) { ok = false; break; }
+                        tc_fence_after();
+                        const uint32_t sbase = base + stage * TC_STAGE_BYTES;
+                        const uint64_t dg = smem_desc_sw128(sbase);
+                        const uint64_t du = smem_desc_sw128(sbase + TC_W_BYTES);
+                        const uint64_t dx = smem_desc_sw128(sbase + 2 * TC_W_BYTES);
+#pragma unroll
+                        for (int k = 0; k < TC_BK / TC_UMMA_K; ++k) {
+                            const uint32_t acc = (kb > 0 || k > 0) ? 1u : 0u;
+                            const uint64_t koff = (uint64_t)(k * TC_UMMA_K * 2 / 16);   // 32 bytes per k step
+                            umma_bf16(tmem_base, dg + koff, dx + koff, idesc, acc);
+                            umma_bf16(tmem_base + TC_BN, du + koff, dx + koff, idesc, acc);
+                        }
+                        umma_commit(bar_empty + 8 * stage);      // slot reusable once these MMAs have read it
+                        if (++stage == TC_STAGES) { stage = 0; phase ^= 1u; }
+                    }
+                    if (ok) umma_commit(bar_acc_full);            // accumulators complete
+                }
+            }
+            if (!ok) { *abort_flag = 1; atomicExch(p.status, (int)DASS_ERR_TIMEOUT); }
+        }
+        __syncwarp();
+    } else {
+        // ------------------------------------------------------------ epilogue (4 warps, 128 neurons)
+        const int quad = warp & 3;                               // TMEM lanes 32*quad .. 32*quad+31
+        const uint32_t lane_addr = tmem_base + ((uint32_t)(quad * 32) << 16);
+        uint32_t tile = 0;
+        bool ok = true;
+        for (int64_t idx = blockIdx.x; idx < p.items && ok; idx += gridDim.x) {
+            const ItemCoord c = decode_item(p, idx);
+            const int64_t tt0 = c.band * TC_BAND_TILES;
+            const int64_t tt1 = tt0 + TC_BAND_TILES < p.token_tiles ? tt0 + TC_BAND_TILES : p.token_tiles;
+            double acc = 0.0;
+            for (int64_t tt = tt0; tt < tt1 && ok; ++tt, ++tile) {
+                if (!mbar_wait(bar_acc_full, tile & 1u, abort_flag)) { ok = false; break; }
+                tc_fence_after();
+                float s = 0.0f;
+#pragma unroll 1
+                for (int col = 0; col < TC_BN; col += 32) {
+                    uint32_t g[32], u[32];
+                    tmem_ld_32(lane_addr + col, g);
+                    tmem_ld_32(lane_addr + TC_BN + col, u);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) {
+                        const float h = glu_h<ACT>(__uint_as_float(g[j]), __uint_as_float(u[j]));
+                        s = fmaf(h, h, s);
+                    }
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_acc_empty);
+                acc += (double)s;       // tokens past T are zero rows of X: act(0) * 0 adds nothing
+            }
+            const int64_t neuron = c.nt * TC_BM + quad * 32 + lane;
+            if (ok && neuron < p.I) p.partial[c.band * p.I + neuron] = acc;
+        }
+        if (!ok && lane == 0) { *abort_flag = 1; atomicExch(p.status, (int)DASS_ERR_TIMEOUT); }
+    }
+
+    // ---------------------------------------------------------------- teardown
+    tc_fence_before();
+    __syncthreads();
+    if (*abort_flag) {
+        // failure path only: give copies and MMAs that were already issued time to land before the
+        // shared memory and the TMEM columns are handed back
+        for (int i = 0; i < 20; ++i) __nanosleep(1000000);
+        __syncthreads();
+    }
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, TC_TMEM_COLS);
+    }
+}
+
+// ------------------------------------------------------------------ host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_tiled_fn()
+{
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void *ptr = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) != cudaSuccess ||
+            qres != cudaDriverEntryPointSuccess)
+            return nullptr;
+        fn = reinterpret_cast<EncodeTiledFn>(ptr);
+    }
+    return fn;
+}
+
+// Row-major bf16 matrix [rows x cols] with pitch ld: dimension 0 = the contiguous k axis.  Boxes are
+// 64 x box_rows elements with the 128-byte swizzle; out-of-range elements read as zero.
+static bool make_map(CUtensorMap *map, const void *ptr, int64_t rows, int64_t cols, int64_t ld, int box_rows)
+{
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)TC_BK, (cuuint32_t)box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(ptr), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+int64_t calib_tc_parts(int64_t T, int64_t I)
+{
+    (void)I;
+    const int64_t token_tiles = (T + TC_BN - 1) / TC_BN;
+    return (token_tiles + TC_BAND_TILES - 1) / TC_BAND_TILES;
+}
+
+int device_sm_count();   // dass_abi.cu
+
+template <int ACT>
+static cudaError_t launch_tc(const CUtensorMap &mx, const CUtensorMap &mg, const CUtensorMap &mu, const TcParams &p,
+                             int grid, cudaStream_t st)
+{
+    static bool configured = false;
+    if (!configured) {
+        const cudaError_t e = cudaFuncSetAttribute(calib_tc_kernel<ACT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                   (int)TC_SMEM_BYTES);
+        if (e != cudaSuccess) return e;
+        configured = true;
+    }
+    calib_tc_kernel<ACT><<<grid, TC_THREADS, TC_SMEM_BYTES, st>>>(mx, mg, mu, p);
+    return cudaGetLastError();
+}
+
+dass_status calib_tc_launch(const void *X, int64_t T, int64_t ldx, const void *Wg, const void *Wu,
+                            int64_t I, int64_t d, int64_t ldw, int act, double *partial, int *status,
+                            cudaStream_t st)
+{
+    if (d > 0x7fffffffll - TC_BK || T > 0x7fffffffll - TC_BN || I > 0x7fffffffll - TC_BM) return DASS_ERR_UNSUPPORTED;
+    CUtensorMap mx, mg, mu;
+    if (!make_map(&mx, X, T, d, ldx, TC_BN) || !make_map(&mg, Wg, I, d, ldw, TC_BM) || !make_map(&mu, Wu, I, d, ldw, TC_BM))
+        return DASS_ERR_CUDA;
+    TcParams p;
+    p.partial = partial; p.status = status;
+    p.T = T; p.I = I; p.d = d;
+    p.neuron_tiles = (I + TC_BM - 1) / TC_BM;
+    p.token_tiles = (T + TC_BN - 1) / TC_BN;
+    p.bands = calib_tc_parts(T, I);
+    p.items = p.neuron_tiles * p.bands;
+    p.k_blocks = (d + TC_BK - 1) / TC_BK;
+    const int sms = device_sm_count();
+    const int grid = (int)(p.items < sms ? p.items : sms);
+    cudaError_t e;
+    switch (act) {
+    case DASS_ACT_SILU: e = launch_tc<DASS_ACT_SILU>(mx, mg, mu, p, grid, st); break;
+    case DASS_ACT_GELU_TANH: e = launch_tc<DASS_ACT_GELU_TANH>(mx, mg, mu, p, grid, st); break;
+    default: e = launch_tc<DASS_ACT_RELU>(mx, mg, mu, p, grid, st); break;
+    }
+    return e == cudaSuccess ? DASS_OK : DASS_ERR_CUDA;
+}
+
+}  // namespace dass
