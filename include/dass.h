@@ -85,6 +85,31 @@ dass_status dass_calib_accumulate(const void *X, int64_t T, int64_t ldx,
  * the kernel gave up (the results of that call are then invalid; the context stays usable). */
 dass_status dass_calib_status(const void *workspace, void *cuda_stream);
 
+/* The paper has no counterpart for this entry point: it exists for callers that cannot allocate.
+ * Some users of this library may not call cudaMalloc where they calibrate -- code inside a framework's
+ * memory-planned region or allocator callback, plugins that own nothing but the tensors they are
+ * handed, processes with a device-memory budget fixed at start-up, loops where an allocation's implicit
+ * device synchronisation is not acceptable.  dass_calib_accumulate makes them supply the workspace; this
+ * variant needs none.  It computes exactly what dass_calib_accumulate computes (same kernels, same
+ * fixed reduction order, same arguments and error codes), but its scratch is a fixed array of
+ * DASS_STATIC_SCRATCH_BYTES inside the library's device image, which every GPU that loads the library
+ * holds until the process exits.  It calls no cudaMalloc / cudaFree and no allocating routine.
+ *  - Limit: a problem whose dass_calib_workspace_bytes(T, d, I, dt) exceeds DASS_STATIC_SCRATCH_BYTES is
+ *    refused with DASS_ERR_WORKSPACE and nothing is touched (16 MiB covers a 28672-neuron bf16 layer
+ *    at 262144 tokens per call; feed larger token counts in several calls).
+ *  - The first call on each device (made with that device current) looks up the scratch's device
+ *    address once; make that first call before any stream capture begins.
+ *  - All calls on a device share the one array, which keeps the previous call's contents; the call
+ *    clears the status word itself and overwrites every partial sum it later reads.  Two calls that may
+ *    overlap on the GPU (different streams, no ordering between them) race on it: order them.
+ *  - scratch_address (HOST pointer, nullable) receives the array's device address, which may be handed
+ *    to dass_calib_status to learn whether a bounded device-side wait timed out. */
+#define DASS_STATIC_SCRATCH_BYTES (16u << 20)
+dass_status dass_calib_accumulate_static(const void *X, int64_t T, int64_t ldx,
+                                         const void *Wg, const void *Wu, int64_t I, int64_t d, int64_t ldw,
+                                         dass_dtype dt, dass_act act, double *sumsq,
+                                         void **scratch_address /* HOST, nullable */, void *cuda_stream);
+
 /* norm[i] = (float) sqrt(sumsq[i]): the l2 norm ||y_i||_2 handed to stage (b).
  * Both operations are correctly rounded, so the value is reproducible bit for bit. */
 dass_status dass_norm_finalize(const double *sumsq, int64_t I, float *norm, void *cuda_stream);

@@ -24,7 +24,8 @@ AXIS_ROWS, AXIS_COLS = 0, 1
 ACT_BY_NAME = {"silu": ACT_SILU, "gelu_tanh": ACT_GELU_TANH, "relu": ACT_RELU}
 
 EXPORTS = (
-    "dass_calib_workspace_bytes", "dass_calib_accumulate", "dass_calib_status", "dass_norm_finalize",
+    "dass_calib_workspace_bytes", "dass_calib_accumulate", "dass_calib_accumulate_static", "dass_calib_status",
+    "dass_norm_finalize",
     "dass_score_nm", "dass_compress_nm", "dass_status_string", "dass_version",
 )
 
@@ -53,6 +54,9 @@ def load() -> ctypes.CDLL:
     lib.dass_calib_accumulate.restype = ctypes.c_int
     lib.dass_calib_accumulate.argtypes = [vp, i64, i64, vp, vp, i64, i64, i64, ctypes.c_int, ctypes.c_int,
                                           vp, vp, sz, vp]
+    lib.dass_calib_accumulate_static.restype = ctypes.c_int
+    lib.dass_calib_accumulate_static.argtypes = [vp, i64, i64, vp, vp, i64, i64, i64, ctypes.c_int, ctypes.c_int,
+                                                 vp, ctypes.POINTER(ctypes.c_void_p), vp]
     lib.dass_calib_status.restype = ctypes.c_int
     lib.dass_calib_status.argtypes = [vp, vp]
     lib.dass_norm_finalize.restype = ctypes.c_int
@@ -143,6 +147,34 @@ def calib_accumulate(X: torch.Tensor, Wg: torch.Tensor, Wu: torch.Tensor, act: i
                                         _dtype_code(X), int(act), sumsq.data_ptr(),
                                         workspace.data_ptr(), workspace.numel(), _stream(stream))
     _check(code, "dass_calib_accumulate")
+
+
+STATIC_SCRATCH_BYTES = 16 << 20
+
+
+def calib_accumulate_static(X: torch.Tensor, Wg: torch.Tensor, Wu: torch.Tensor, act: int, sumsq: torch.Tensor,
+                            stream: Optional[torch.cuda.Stream] = None) -> int:
+    """calib_accumulate for callers that must not allocate: the scratch is a fixed array inside the
+    library (at most STATIC_SCRATCH_BYTES, shared by all calls on the device -- do not overlap calls).
+    Returns the scratch's device address, which calib_status_at() accepts."""
+    T, d, ldx = _matrix(X, "X")
+    I, d2, ldw = _matrix(Wg, "Wg")
+    I3, d3, ldw3 = _matrix(Wu, "Wu")
+    if (d2, I3, d3, ldw3) != (d, I, d, ldw) or Wg.dtype != X.dtype or Wu.dtype != X.dtype:
+        raise ValueError("X [T x d], Wg [I x d], Wu [I x d] must agree in d, I, dtype and row pitch")
+    if sumsq.dtype != torch.float64 or not sumsq.is_cuda or sumsq.numel() != I or not sumsq.is_contiguous():
+        raise ValueError("sumsq must be a contiguous CUDA float64 tensor of I elements")
+    addr = ctypes.c_void_p(0)
+    code = load().dass_calib_accumulate_static(X.data_ptr(), T, ldx, Wg.data_ptr(), Wu.data_ptr(), I, d, ldw,
+                                               _dtype_code(X), int(act), sumsq.data_ptr(), ctypes.byref(addr),
+                                               _stream(stream))
+    _check(code, "dass_calib_accumulate_static")
+    return int(addr.value)
+
+
+def calib_status_at(address: int, stream: Optional[torch.cuda.Stream] = None) -> None:
+    """calib_status for a raw device address (the one calib_accumulate_static returned)."""
+    _check(load().dass_calib_status(int(address), _stream(stream)), "dass_calib_status")
 
 
 def calib_status(workspace: torch.Tensor, stream: Optional[torch.cuda.Stream] = None) -> None:
