@@ -243,7 +243,7 @@ def run_ours(args):
 
     # end to end: pinned host inputs -> device -> path -> results back to the host, every step
     e2e = None
-    if rank == 0 or world > 1:
+    if args.e2e_steps > 0:
         e2e = run_e2e(cfg, path, X, pool[0], alpha, args.e2e_steps, world, device)
 
     out = None

@@ -1,4 +1,6 @@
-// Stage (b): Eq. 4 / Eq. 5 score and N:M selection in one streaming pass.
+// Stage (b): Eq. 4 / Eq. 5 score and N:M selection in one streaming pass -- the plain formulation with
+// exact double products, used for fp32 weights (bf16 weights take the tuned kernels of score_nm_bf16.cu,
+// which fall back to the same exact selection on ties).
 //
 // Bandwidth-bound: every weight is read once (128-bit loads), the pruned copy and one mask bit per
 // weight are written once; no score matrix and no sort exist.  A warp owns a tile of 32 rows by 256
@@ -180,12 +182,17 @@ static cudaError_t launch_score(const ScoreParams &p, bool norm_cols, bool group
 }
 
 int device_sm_count();   // dass_abi.cu
+cudaError_t score_nm_bf16_launch(const void *W, int64_t rows, int64_t cols, int64_t ld,
+                                 const float *norm, bool norm_cols, float alpha, int n_keep, int m, bool group_cols,
+                                 uint32_t *mask_bits, void *W_pruned, cudaStream_t st);   // score_nm_bf16.cu
 
 // Host entry used by the C ABI (arguments already validated there).
 cudaError_t score_nm_launch(const void *W, int64_t rows, int64_t cols, int64_t ld, bool bf16,
                             const float *norm, bool norm_cols, float alpha, int n_keep, int m, bool group_cols,
                             uint32_t *mask_bits, void *W_pruned, cudaStream_t st)
 {
+    if (bf16)   // bf16 weights take the integer / bit-sliced kernels of score_nm_bf16.cu
+        return score_nm_bf16_launch(W, rows, cols, ld, norm, norm_cols, alpha, n_keep, m, group_cols, mask_bits, W_pruned, st);
     ScoreParams p;
     p.W = W; p.Wp = W_pruned; p.mask = mask_bits; p.norm = norm;
     p.rows = rows; p.cols = cols; p.ld = ld;
@@ -200,8 +207,6 @@ cudaError_t score_nm_launch(const void *W, int64_t rows, int64_t cols, int64_t l
     const int64_t want = (ntasks + warps_per_block - 1) / warps_per_block;
     const int64_t cap = (int64_t)device_sm_count() * 8;   // 8 blocks of 256 threads fill an SM
     const int grid = (int)(want < cap ? want : cap);
-    if (bf16) return m == 4 ? launch_score<true, 4>(p, norm_cols, group_cols, grid, st)
-                            : launch_score<true, 8>(p, norm_cols, group_cols, grid, st);
     return m == 4 ? launch_score<false, 4>(p, norm_cols, group_cols, grid, st)
                   : launch_score<false, 8>(p, norm_cols, group_cols, grid, st);
 }
