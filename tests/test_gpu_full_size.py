@@ -1,0 +1,113 @@
+"""Parity at the full sizes of the four large layer shapes (LLaMA2-7B, Mistral-7B, Gemma-7B, LLaMA2-70B),
+in the launch configuration the benchmark times (whole 262144-token calibration batch in one call).
+
+The oracle cannot redo 10^13..10^14 flops, so stage (a) is checked on outputs it can compute one by one:
+ (i)  sampled neurons (strided through every part of the matrix plus the largest-norm ones) over ALL tokens;
+ (ii) all neurons on a token prefix (a separate GPU call).
+Stage (b) is checked in full: every mask word, pruned weight, compressed value and metadata word of the
+gate and down matrices, bit for bit, with the oracle's norm vector.  Finally the end-to-end rule: masks from
+GPU norms may differ from masks from oracle norms only in groups whose oracle score gap is below 1e-3."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from helpers import assert_stage_b_equal, gpu_stage_b, oracle_stage_b, to_np32, u32, unpack_mask
+from paper_2405_01943_b200 import binding, synth
+from paper_2405_01943_b200.binding import AXIS_COLS, AXIS_ROWS
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+NAMES = ["llama2_7b", "mistral_7b", "gemma_7b", "llama2_70b"]
+ORACLE_ACT = {"silu": oracle.ACT_SILU, "gelu_tanh": oracle.ACT_GELU_TANH}
+T_PREFIX = 300
+N_SAMPLED = 64
+
+
+@pytest.fixture(scope="module", params=NAMES)
+def layer(request):
+    cfg = synth.CONFIGS[request.param]
+    X = synth.make_x(cfg, DEV)
+    Wg, Wu, Wd = synth.make_weights(cfg, DEV, layer=0)
+    yield cfg, X, Wg, Wu, Wd
+    del X, Wg, Wu, Wd
+    torch.cuda.empty_cache()
+
+
+def _gpu_sumsq(cfg, X, Wg, Wu):
+    sumsq = torch.zeros(cfg.I, dtype=torch.float64, device=DEV)
+    ws = binding.calib_workspace(X.shape[0], cfg.d, cfg.I, X.dtype, DEV)
+    binding.calib_accumulate(X, Wg, Wu, binding.ACT_BY_NAME[cfg.act], sumsq, ws)
+    binding.calib_status(ws)
+    return sumsq
+
+
+def test_stage_a_sampled_neurons_over_all_tokens(layer):
+    cfg, X, Wg, Wu, _ = layer
+    got = _gpu_sumsq(cfg, X, Wg, Wu).cpu().numpy()
+    assert np.all(np.isfinite(got)) and np.all(got > 0)
+    top = np.argsort(-got)[: N_SAMPLED // 4]
+    strided = np.linspace(0, cfg.I - 1, N_SAMPLED - len(top)).astype(np.int64)    # includes first and last neuron
+    idx = np.unique(np.concatenate([top, strided]))
+    sel = torch.from_numpy(idx).to(DEV)
+    wg, wu = to_np32(Wg[sel]), to_np32(Wu[sel])
+    ref = np.zeros(len(idx), dtype=np.float64)
+    step = 32768
+    for t0 in range(0, cfg.T, step):                       # the oracle accumulates batch by batch
+        oracle.calib_sumsq(to_np32(X[t0:t0 + step]), wg, wu, ORACLE_ACT[cfg.act], ref)
+    rel = np.abs(np.sqrt(got[idx]) - np.sqrt(ref)) / np.sqrt(ref)
+    assert rel.max() <= 2e-3, f"{cfg.name}: sampled-neuron norm error {rel.max():.3e}"
+
+
+def test_stage_a_all_neurons_on_a_token_prefix_then_end_to_end_masks(layer):
+    cfg, X, Wg, Wu, Wd = layer
+    Xp = X[:T_PREFIX]
+    sumsq = _gpu_sumsq(cfg, Xp, Wg, Wu)
+    ref = oracle.calib_sumsq(to_np32(Xp), to_np32(Wg), to_np32(Wu), ORACLE_ACT[cfg.act])
+    rel = np.abs(np.sqrt(sumsq.cpu().numpy()) - np.sqrt(ref)) / np.sqrt(ref)
+    assert rel.max() <= 2e-3, f"{cfg.name}: prefix norm error {rel.max():.3e}"
+
+    # end to end on a slice of the down projection and of the gate projection
+    norm_gpu = binding.norm_finalize(sumsq)
+    norm_ref = oracle.norm_from_sumsq(ref)
+    rows = 256
+    for W, na, alpha, ga in ((Wd[:rows], AXIS_COLS, 1.0, AXIS_COLS), (Wg[:, :rows].contiguous(), AXIS_ROWS, 0.5, AXIS_ROWS)):
+        mask_gpu, _ = binding.score_nm(W, norm_gpu, na, alpha, cfg.n_keep, cfg.m, ga, want_pruned=False)
+        torch.cuda.synchronize()
+        got = unpack_mask(u32(mask_gpu), W.shape[1])
+        Wn = to_np32(W)
+        want, _ = oracle.score_nm(Wn, norm_ref, na, alpha, cfg.n_keep, cfg.m, ga, want_pruned=False)
+        diff = np.argwhere(got != want)
+        scale = np.array([oracle.scale(float(v), alpha) for v in norm_ref], dtype=np.float64)
+        score = np.abs(Wn.astype(np.float64)) * (scale[None, :] if na == AXIS_COLS else scale[:, None])
+        seen = set()
+        for r, c in diff:
+            key = (r, c // cfg.m) if ga == AXIS_COLS else (r // cfg.m, c)
+            if key in seen:
+                continue
+            seen.add(key)
+            grp = score[r, key[1] * cfg.m:(key[1] + 1) * cfg.m] if ga == AXIS_COLS else score[key[0] * cfg.m:(key[0] + 1) * cfg.m, c]
+            s = np.sort(grp)[::-1]
+            gap = (s[cfg.n_keep - 1] - s[cfg.n_keep]) / s[cfg.n_keep - 1]
+            assert gap < 1e-3, f"{cfg.name}: group {key} differs although the oracle gap is {gap:.3e}"
+        assert len(seen) <= 1e-3 * got.size / cfg.m                     # and such near-ties are rare
+
+
+def test_stage_b_full_matrices_bit_exact(layer):
+    cfg, X, Wg, Wu, Wd = layer
+    gen = torch.Generator(device=DEV)
+    gen.manual_seed(cfg.seed + 77)
+    # a norm vector with the spread real intermediate norms have (a few neurons far above the rest)
+    norm = (torch.randn(cfg.I, generator=gen, device=DEV).abs() * 40 + 0.5)
+    norm[torch.randperm(cfg.I, generator=gen, device=DEV)[: cfg.I // 100]] *= 30
+    norm = norm.float().contiguous()
+    norm32 = to_np32(norm)
+    for alpha in cfg.alphas:
+        ref = oracle_stage_b(Wg, norm32, AXIS_ROWS, alpha, cfg.n_keep, cfg.m, AXIS_ROWS)
+        assert_stage_b_equal(gpu_stage_b(Wg, norm, AXIS_ROWS, alpha, cfg.n_keep, cfg.m, AXIS_ROWS), ref)
+        del ref
+    ref = oracle_stage_b(Wd, norm32, AXIS_COLS, 1.0, cfg.n_keep, cfg.m, AXIS_COLS)
+    got = gpu_stage_b(Wd, norm, AXIS_COLS, 1.0, cfg.n_keep, cfg.m, AXIS_COLS)
+    assert_stage_b_equal(got, ref)
+    mk = unpack_mask(got["words"], cfg.I)
+    assert np.all(mk.reshape(cfg.d, cfg.I // cfg.m, cfg.m).sum(-1) == cfg.n_keep)
