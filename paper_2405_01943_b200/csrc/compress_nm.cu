@@ -251,11 +251,15 @@ static cudaError_t launch_compress(const CompressParams &p, bool group_cols, int
 }
 
 int device_sm_count();   // dass_abi.cu
+cudaError_t compress_cols_bf16_launch(const void *W, const uint32_t *mask_bits, int64_t rows, int64_t cols, int64_t ld,
+                                      int n_keep, int m, void *values, uint32_t *meta, cudaStream_t st);   // compress_nm_bf16.cu
 
 cudaError_t compress_nm_launch(const void *W, const uint32_t *mask_bits, int64_t rows, int64_t cols, int64_t ld,
                                bool bf16, int n_keep, int m, bool group_cols,
                                void *values, uint32_t *meta, cudaStream_t st)
 {
+    if (bf16 && group_cols)   // permute-table kernel of compress_nm_bf16.cu
+        return compress_cols_bf16_launch(W, mask_bits, rows, cols, ld, n_keep, m, values, meta, st);
     CompressParams p;
     p.W = W; p.mask = mask_bits; p.values = values; p.meta = meta;
     p.rows = rows; p.cols = cols; p.ld = ld;
