@@ -128,7 +128,8 @@ __global__ void norm_finalize_kernel(const double *__restrict__ sumsq, int64_t I
     if (i < I) norm[i] = __double2float_rn(sqrt(sumsq[i]));
 }
 
-__global__ void status_clear_kernel(int *status) { *status = 0; }
+// word 0: device status; word 1: the tensor-core kernel's alignment counter
+__global__ void status_clear_kernel(int *status) { status[0] = 0; status[1] = 0; }
 
 int64_t calib_simt_parts(int64_t T)
 {
