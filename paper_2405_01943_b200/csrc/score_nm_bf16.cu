@@ -5,9 +5,8 @@
 // integer and bit-sliced logic instead of per-element double arithmetic:
 //
 //   * p = fl32(|w| * scale).  Rounding is monotone, so p_b > p_a proves score_b > score_a for the
-//     exact products; non-negative floats order like their bit patterns, so the comparison is the
-//     sign of an integer subtraction, shifted into a bit-sliced word with one funnel shift (bit j of a
-//     word = column j, or row j, of the lane's tile).
+//     exact products; the comparison is the sign of the float difference p_a - p_b (never wrong), shifted
+//     into a bit-sliced word with one funnel shift (bit j of a word = column j, or row j, of the lane's tile).
 //   * ranks are counted with full adders on those words (one LOP3 each) and compared with n_keep, which
 //     yields the keep bits of 8 groups at once;
 //   * only when two rounded products of a group are EQUAL is the order not proven; the lane then
@@ -40,6 +39,9 @@ constexpr int F_THREADS = 256;
 #define F_MIN_BLOCKS 4
 #endif
 constexpr int F_COLS = 256;          // columns per warp strip
+// prefetch depth of the shared-memory slab ring (slabs of R rows x 512 bytes per warp)
+__host__ __device__ constexpr int ring_stages(int rows_per_unit) { return rows_per_unit >= 8 ? 2 : 3; }
+__host__ __device__ constexpr int ring_bytes(int rows_per_unit) { return (F_THREADS / 32) * ring_stages(rows_per_unit) * rows_per_unit * 512; }
 #ifndef F_SLAB_ROWS
 #define F_SLAB_ROWS 4
 #endif
@@ -49,6 +51,52 @@ constexpr int F_SLAB = F_SLAB_ROWS;  // rows per unit when groups run along the 
 // budget of the streaming loops, and they run once per strip or per 32 rows only.
 __device__ __noinline__ float scale_of(float n, int mode, float alpha) { return scale_from_norm(n, mode, alpha); }
 
+// 16-byte asynchronous copy global -> shared (src_bytes = 0 writes zeros and reads nothing)
+__device__ __forceinline__ void cp_async16(void *smem_dst, const void *gsrc, int src_bytes)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;"
+                 ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gsrc), "r"(src_bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+// Prefetch ring of a warp: STAGES slabs of R rows x 32 lanes x 16 bytes in shared memory.  A lane only ever
+// reads back the 16 bytes it copied itself, so the per-thread wait_group is the only synchronisation needed.
+template <int R, int STAGES>
+struct SlabRing {
+    uint4 *buf;   // this warp's [STAGES][R][32]
+    __device__ __forceinline__ uint4 *slot(int stage, int row, int lane) const { return buf + (stage * R + row) * 32 + lane; }
+    // starts the copy of the unit at `cur` (rows r0..r0+R-1 of the lane's 8 columns) into `stage` and
+    // commits the group; `live` is false past the warp's last unit (an empty group keeps the count uniform)
+    __device__ __forceinline__ void issue(const ScoreFastParams &p, int strip, int g, bool live, int stage, int lane) const
+    {
+        if (live) {
+            const int64_t r0 = (int64_t)g * R;
+            const int64_t c0 = (int64_t)strip * F_COLS + lane * 8;
+            const bool col_ok = c0 < p.cols;
+            const uint16_t *src = p.W + r0 * p.ld + c0;
+#pragma unroll
+            for (int i = 0; i < R; ++i) {
+                const bool ok = col_ok && (r0 + i < p.rows);
+                cp_async16(slot(stage, i, lane), ok ? (const void *)src : (const void *)p.W, ok ? 16 : 0);
+                src += p.ld;
+            }
+        }
+        cp_async_commit();
+    }
+};
+
+// Position of a unit: which 256-column strip and which slab inside it.  Units of a warp are consecutive,
+// so the position is advanced instead of being divided out of the unit index each time.
+struct UnitCursor {
+    int strip, g;
+    __device__ __forceinline__ void advance(int units_per_strip)
+    {
+        if (++g == units_per_strip) { g = 0; ++strip; }
+    }
+};
+
 __device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel)
 {
     uint32_t d;
@@ -56,11 +104,52 @@ __device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel)
     return d;
 }
 
-// bits of fl32(|element| * scale); element = low (hi == false) or high half of a word of two bf16
-__device__ __forceinline__ uint32_t prod_bits(uint32_t word, bool hi, float scale)
+// fl32(|element| * scale); element = low (hi == false) or high half of a word of two bf16.  The low half is
+// moved up with a multiply so that it runs on the FMA pipe (the integer/logic pipe is the busy one here).
+__device__ __forceinline__ float prod_of(uint32_t word, bool hi, float scale)
 {
-    const uint32_t fb = hi ? (word & 0xffff0000u) : (word << 16);
-    return __float_as_uint(fabsf(__uint_as_float(fb)) * scale);
+    const uint32_t fb = hi ? (word & 0xffff0000u) : (word * 65536u);
+    return fabsf(__uint_as_float(fb)) * scale;
+}
+
+// Pair index of (a, b), a < b, in the order (0,1),(0,2),...,(0,M-1),(1,2),...
+template <int M>
+__host__ __device__ constexpr int pair_index(int a, int b) { return a * M - a * (a + 1) / 2 + (b - a - 1); }
+
+// Pairwise comparisons of one group of M rounded products: shifts "p_b > p_a" (the sign of p_a - p_b, which
+// floating-point subtraction never gets wrong) into the bit-sliced words C and returns true if two products may
+// be equal.  Equality is found with a running product of the differences (FMA pipe): it is 0 -- or NaN after an
+// overflow -- exactly when some difference is 0, and it can only err towards "maybe" (underflow), which sends
+// the lane to the exact path.
+template <int M>
+__device__ __forceinline__ bool compare_group(const float (&pf)[M], uint32_t (&C)[M * (M - 1) / 2])
+{
+    bool maybe_tie = false;
+    if constexpr (M == 4) {
+        float t = 1.2676506e30f;   // 2^100: head-room against underflow of six small differences
+#pragma unroll
+        for (int a = 0; a < M; ++a)
+#pragma unroll
+            for (int b = a + 1; b < M; ++b) {
+                const float dlt = __fsub_rn(pf[a], pf[b]);
+                C[pair_index<M>(a, b)] = __funnelshift_l(__float_as_uint(dlt), C[pair_index<M>(a, b)], 1);
+                t = __fmul_rn(t, dlt);
+            }
+        maybe_tie = !(fabsf(t) > 0.0f);
+    } else {
+#pragma unroll
+        for (int a = 0; a < M - 1; ++a) {
+            float t = 1.8446744e19f;   // 2^64 per chain of at most 7 differences
+#pragma unroll
+            for (int b = a + 1; b < M; ++b) {
+                const float dlt = __fsub_rn(pf[a], pf[b]);
+                C[pair_index<M>(a, b)] = __funnelshift_l(__float_as_uint(dlt), C[pair_index<M>(a, b)], 1);
+                t = __fmul_rn(t, dlt);
+            }
+            maybe_tie |= !(fabsf(t) > 0.0f);
+        }
+    }
+    return maybe_tie;
 }
 
 // full adder on bit-sliced words
@@ -81,9 +170,6 @@ __device__ __forceinline__ uint32_t rank_below(uint32_t b2, uint32_t b1, uint32_
     }
 }
 
-// Pair index of (a, b), a < b, in the order (0,1),(0,2),...,(0,M-1),(1,2),...
-template <int M>
-__host__ __device__ constexpr int pair_index(int a, int b) { return a * M - a * (a + 1) / 2 + (b - a - 1); }
 
 // Keep words from the bit-sliced comparison words C[pair] (bit set: the later element b beats a).
 // Element a is preceded by every earlier k that b-beats... i.e. rank_a = sum_{k<a} !C[k,a] + sum_{k>a} C[a,k].
@@ -194,21 +280,38 @@ template <int M, bool NORM_COLS>
 __global__ void __launch_bounds__(F_THREADS, F_MIN_BLOCKS) score_rows_bf16_kernel(const ScoreFastParams p)
 {
     constexpr int NP = M * (M - 1) / 2;
+    constexpr int STAGES = ring_stages(M);
+    extern __shared__ uint4 ring_mem[];
     const int lane = threadIdx.x & 31;
     const int64_t warp = (int64_t)blockIdx.x * (F_THREADS / 32) + (threadIdx.x >> 5);
     const int64_t nwarps = (int64_t)gridDim.x * (F_THREADS / 32);
     const int64_t u_begin = p.units * warp / nwarps;
     const int64_t u_end = p.units * (warp + 1) / nwarps;
+    SlabRing<M, STAGES> ring;
+    ring.buf = ring_mem + (threadIdx.x >> 5) * (STAGES * M * 32);
+    const int ups = (int)p.units_per_strip;
+    UnitCursor cur, pre;
+    cur.strip = (int)(u_begin / p.units_per_strip);
+    cur.g = (int)(u_begin - (int64_t)cur.strip * p.units_per_strip);
+    pre = cur;
+    int64_t u_pre = u_begin;
+#pragma unroll
+    for (int s = 0; s < STAGES - 1; ++s) {
+        ring.issue(p, pre.strip, pre.g, u_pre < u_end, s, lane);
+        pre.advance(ups);
+        ++u_pre;
+    }
 
     int64_t cached_strip = -1, cached_base = -1;
     float sc[8];          // per-column scales of the strip (NORM_COLS)
     float lane_scale = 0.0f;   // scale of row cached_base + lane (!NORM_COLS)
     int nvalid = 0;
     int64_t c0 = 0;
+    int stage = 0;
 
-    for (int64_t u = u_begin; u < u_end; ++u) {
-        const int64_t strip = u / p.units_per_strip;
-        const int64_t r0 = (u - strip * p.units_per_strip) * M;
+    for (int64_t u = u_begin; u < u_end; ++u, cur.advance(ups)) {
+        const int64_t strip = cur.strip;
+        const int64_t r0 = (int64_t)cur.g * M;
         if (strip != cached_strip) {
             cached_strip = strip;
             cached_base = -1;
@@ -230,12 +333,16 @@ __global__ void __launch_bounds__(F_THREADS, F_MIN_BLOCKS) score_rows_bf16_kerne
             }
         }
 
+        // this unit's slab has landed once at most STAGES-2 younger groups are pending; then refill the
+        // slot that was consumed one iteration ago with the unit STAGES-1 ahead
+        cp_async_wait<STAGES - 2>();
         uint4 v[M];
 #pragma unroll
-        for (int q = 0; q < M; ++q) {
-            if (nvalid > 0) v[q] = __ldcs(reinterpret_cast<const uint4 *>(p.W + (r0 + q) * p.ld + c0));
-            else v[q] = make_uint4(0u, 0u, 0u, 0u);
-        }
+        for (int q = 0; q < M; ++q) v[q] = *ring.slot(stage, q, lane);
+        ring.issue(p, pre.strip, pre.g, u_pre < u_end, stage == 0 ? STAGES - 1 : stage - 1, lane);
+        pre.advance(ups);
+        ++u_pre;
+        stage = stage + 1 == STAGES ? 0 : stage + 1;
         float rs[M];
 #pragma unroll
         for (int q = 0; q < M; ++q) {
@@ -249,17 +356,10 @@ __global__ void __launch_bounds__(F_THREADS, F_MIN_BLOCKS) score_rows_bf16_kerne
         bool tie = false;
 #pragma unroll
         for (int j = 7; j >= 0; --j) {       // column 7 first: after 8 inserts column j sits at bit j
-            uint32_t pb[M];
+            float pf[M];
 #pragma unroll
-            for (int q = 0; q < M; ++q) pb[q] = prod_bits(word_of(v[q], j >> 1), (j & 1) != 0, NORM_COLS ? sc[j] : rs[q]);
-#pragma unroll
-            for (int a = 0; a < M; ++a)
-#pragma unroll
-                for (int b = a + 1; b < M; ++b) {
-                    const uint32_t dlt = pb[a] - pb[b];                     // negative iff p_b > p_a
-                    C[pair_index<M>(a, b)] = __funnelshift_l(dlt, C[pair_index<M>(a, b)], 1);
-                    tie |= (dlt == 0u);
-                }
+            for (int q = 0; q < M; ++q) pf[q] = prod_of(word_of(v[q], j >> 1), (j & 1) != 0, NORM_COLS ? sc[j] : rs[q]);
+            tie |= compare_group<M>(pf, C);
         }
         uint32_t K[M];
         keep_from_pairs<M>(C, p.n_keep, K);
@@ -294,21 +394,38 @@ __global__ void __launch_bounds__(F_THREADS, F_MIN_BLOCKS) score_cols_bf16_kerne
 {
     constexpr int NP = M * (M - 1) / 2;
     constexpr int G = 8 / M;             // groups inside a lane's 8 columns
+    constexpr int STAGES = ring_stages(F_SLAB);
+    extern __shared__ uint4 ring_mem[];
     const int lane = threadIdx.x & 31;
     const int64_t warp = (int64_t)blockIdx.x * (F_THREADS / 32) + (threadIdx.x >> 5);
     const int64_t nwarps = (int64_t)gridDim.x * (F_THREADS / 32);
     const int64_t u_begin = p.units * warp / nwarps;
     const int64_t u_end = p.units * (warp + 1) / nwarps;
+    SlabRing<F_SLAB, STAGES> ring;
+    ring.buf = ring_mem + (threadIdx.x >> 5) * (STAGES * F_SLAB * 32);
+    const int ups = (int)p.units_per_strip;
+    UnitCursor cur, pre;
+    cur.strip = (int)(u_begin / p.units_per_strip);
+    cur.g = (int)(u_begin - (int64_t)cur.strip * p.units_per_strip);
+    pre = cur;
+    int64_t u_pre = u_begin;
+#pragma unroll
+    for (int s = 0; s < STAGES - 1; ++s) {
+        ring.issue(p, pre.strip, pre.g, u_pre < u_end, s, lane);
+        pre.advance(ups);
+        ++u_pre;
+    }
 
     int64_t cached_strip = -1, cached_base = -1;
     float sc[8];
     float lane_scale = 0.0f;
     int nvalid = 0;
     int64_t c0 = 0;
+    int stage = 0;
 
-    for (int64_t u = u_begin; u < u_end; ++u) {
-        const int64_t strip = u / p.units_per_strip;
-        const int64_t r0 = (u - strip * p.units_per_strip) * F_SLAB;
+    for (int64_t u = u_begin; u < u_end; ++u, cur.advance(ups)) {
+        const int64_t strip = cur.strip;
+        const int64_t r0 = (int64_t)cur.g * F_SLAB;
         if (strip != cached_strip) {
             cached_strip = strip;
             cached_base = -1;
@@ -330,12 +447,14 @@ __global__ void __launch_bounds__(F_THREADS, F_MIN_BLOCKS) score_cols_bf16_kerne
             }
         }
 
+        cp_async_wait<STAGES - 2>();
         uint4 v[F_SLAB];
 #pragma unroll
-        for (int i = 0; i < F_SLAB; ++i) {
-            if (nvalid > 0 && r0 + i < p.rows) v[i] = __ldcs(reinterpret_cast<const uint4 *>(p.W + (r0 + i) * p.ld + c0));
-            else v[i] = make_uint4(0u, 0u, 0u, 0u);
-        }
+        for (int i = 0; i < F_SLAB; ++i) v[i] = *ring.slot(stage, i, lane);
+        ring.issue(p, pre.strip, pre.g, u_pre < u_end, stage == 0 ? STAGES - 1 : stage - 1, lane);
+        pre.advance(ups);
+        ++u_pre;
+        stage = stage + 1 == STAGES ? 0 : stage + 1;
 
         uint32_t C[G][NP];
 #pragma unroll
@@ -351,20 +470,13 @@ __global__ void __launch_bounds__(F_THREADS, F_MIN_BLOCKS) score_cols_bf16_kerne
             rsv[i] = rs;
 #pragma unroll
             for (int g = 0; g < G; ++g) {
-                uint32_t pb[M];
+                float pf[M];
 #pragma unroll
                 for (int q = 0; q < M; ++q) {
                     const int j = g * M + q;
-                    pb[q] = prod_bits(word_of(v[i], j >> 1), (j & 1) != 0, NORM_COLS ? sc[j] : rs);
+                    pf[q] = prod_of(word_of(v[i], j >> 1), (j & 1) != 0, NORM_COLS ? sc[j] : rs);
                 }
-#pragma unroll
-                for (int a = 0; a < M; ++a)
-#pragma unroll
-                    for (int b = a + 1; b < M; ++b) {
-                        const uint32_t dlt = pb[a] - pb[b];
-                        C[g][pair_index<M>(a, b)] = __funnelshift_l(dlt, C[g][pair_index<M>(a, b)], 1);
-                        tie |= (dlt == 0u);
-                    }
+                tie |= compare_group<M>(pf, C[g]);
             }
         }
         // Q[h]: byte a = keep bits (bit i = row i) of column 4h + a
@@ -417,17 +529,28 @@ __global__ void __launch_bounds__(F_THREADS, F_MIN_BLOCKS) score_cols_bf16_kerne
 
 int device_sm_count();   // dass_abi.cu
 
+template <typename K>
+static cudaError_t launch_with_ring(K kernel, int smem, const ScoreFastParams &p, int grid, cudaStream_t st)
+{
+    if (smem > 48 * 1024) {
+        const cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        if (e != cudaSuccess) return e;
+    }
+    kernel<<<grid, F_THREADS, smem, st>>>(p);
+    return cudaGetLastError();
+}
+
 template <int M>
 static cudaError_t launch_fast(const ScoreFastParams &p, bool norm_cols, bool group_cols, int grid, cudaStream_t st)
 {
     if (group_cols) {
-        if (norm_cols) score_cols_bf16_kernel<M, true><<<grid, F_THREADS, 0, st>>>(p);
-        else score_cols_bf16_kernel<M, false><<<grid, F_THREADS, 0, st>>>(p);
-    } else {
-        if (norm_cols) score_rows_bf16_kernel<M, true><<<grid, F_THREADS, 0, st>>>(p);
-        else score_rows_bf16_kernel<M, false><<<grid, F_THREADS, 0, st>>>(p);
+        constexpr int smem = ring_bytes(F_SLAB);
+        return norm_cols ? launch_with_ring(score_cols_bf16_kernel<M, true>, smem, p, grid, st)
+                         : launch_with_ring(score_cols_bf16_kernel<M, false>, smem, p, grid, st);
     }
-    return cudaGetLastError();
+    constexpr int smem = ring_bytes(M);
+    return norm_cols ? launch_with_ring(score_rows_bf16_kernel<M, true>, smem, p, grid, st)
+                     : launch_with_ring(score_rows_bf16_kernel<M, false>, smem, p, grid, st);
 }
 
 cudaError_t score_nm_bf16_launch(const void *W, int64_t rows, int64_t cols, int64_t ld,
