@@ -159,6 +159,25 @@ dass_status dass_compress_nm(const void *W, const uint32_t *mask_bits,
                              int n_keep, int m, dass_axis group_axis,
                              void *values, uint32_t *meta, void *cuda_stream);
 
+/* Unstructured DaSS selection (Section 3, "Pruning Granularity"): inside every comparison line the
+ * floor(sparsity * L) weights with the lowest Eq. 4 / Eq. 5 score are pruned, L being the line length.
+ *     compare_axis = ROWS: a line is a whole column (all rows at one input: "input-balanced", the paper's
+ *                          choice for gate / up, with norm_axis = ROWS and alpha = 0.5)
+ *     compare_axis = COLS: a line is a whole row ("output-balanced", the paper's choice for down and what
+ *                          Wanda does, with norm_axis = COLS and alpha = 1)
+ * Score, scale rounding and order are those of dass_score_nm: exact products, higher score first, lower
+ * index first.  sparsity in [0, 1).  mask_bits / W_pruned as for dass_score_nm (at least one; mask_bits is
+ * written in full, padding bits 0).  workspace: dass_select_workspace_bytes(...) bytes, 16-byte aligned (holds
+ * the rounded norm^alpha vector).  A line (in the matrix dtype) must fit twice into shared memory: up to
+ * about 50 000 bf16 or 25 000 f32 elements, else DASS_ERR_UNSUPPORTED.
+ * Errors: NULL / DTYPE / SHAPE (sizes, sparsity outside [0,1)) / ALIGN / UNSUPPORTED / WORKSPACE / CUDA. */
+dass_status dass_select_workspace_bytes(int64_t rows, int64_t cols, dass_axis norm_axis, size_t *bytes /* HOST */);
+dass_status dass_select_unstructured(const void *W, int64_t rows, int64_t cols, int64_t ld, dass_dtype dt,
+                                     const float *norm, dass_axis norm_axis, float alpha,
+                                     double sparsity, dass_axis compare_axis,
+                                     uint32_t *mask_bits, void *W_pruned,
+                                     void *workspace, size_t workspace_bytes, void *cuda_stream);
+
 /* ------------------------------------------------------------------ misc */
 const char *dass_status_string(dass_status s);   /* static string, never NULL */
 int dass_version(void);                          /* major * 10000 + minor * 100 + patch */

@@ -26,7 +26,8 @@ ACT_BY_NAME = {"silu": ACT_SILU, "gelu_tanh": ACT_GELU_TANH, "relu": ACT_RELU}
 EXPORTS = (
     "dass_calib_workspace_bytes", "dass_calib_accumulate", "dass_calib_accumulate_static", "dass_calib_status",
     "dass_norm_finalize",
-    "dass_score_nm", "dass_compress_nm", "dass_status_string", "dass_version",
+    "dass_score_nm", "dass_compress_nm", "dass_select_workspace_bytes", "dass_select_unstructured",
+    "dass_status_string", "dass_version",
 )
 
 
@@ -67,6 +68,11 @@ def load() -> ctypes.CDLL:
     lib.dass_compress_nm.restype = ctypes.c_int
     lib.dass_compress_nm.argtypes = [vp, vp, i64, i64, i64, ctypes.c_int, ctypes.c_int, ctypes.c_int,
                                      ctypes.c_int, vp, vp, vp]
+    lib.dass_select_workspace_bytes.restype = ctypes.c_int
+    lib.dass_select_workspace_bytes.argtypes = [i64, i64, ctypes.c_int, ctypes.POINTER(sz)]
+    lib.dass_select_unstructured.restype = ctypes.c_int
+    lib.dass_select_unstructured.argtypes = [vp, i64, i64, i64, ctypes.c_int, vp, ctypes.c_int, ctypes.c_float,
+                                             ctypes.c_double, ctypes.c_int, vp, vp, vp, sz, vp]
     lib.dass_status_string.restype = ctypes.c_char_p
     lib.dass_status_string.argtypes = [ctypes.c_int]
     lib.dass_version.restype = ctypes.c_int
@@ -254,3 +260,31 @@ def compress_nm(W: torch.Tensor, mask_bits: torch.Tensor, n_keep: int, m: int, g
                                    _stream(stream))
     _check(code, "dass_compress_nm")
     return values, meta
+
+
+def select_unstructured(W: torch.Tensor, norm: torch.Tensor, norm_axis: int, alpha: float, sparsity: float,
+                        compare_axis: int, mask_bits: Optional[torch.Tensor] = None,
+                        W_pruned: Optional[torch.Tensor] = None, want_mask: bool = True, want_pruned: bool = True,
+                        workspace: Optional[torch.Tensor] = None, stream: Optional[torch.cuda.Stream] = None):
+    """Unstructured selection at `sparsity` inside every column (compare_axis = ROWS) or row (COLS).
+    Returns (mask_bits or None, W_pruned or None)."""
+    rows, cols, ld = _matrix(W, "W")
+    if norm.dtype != torch.float32 or not norm.is_cuda or not norm.is_contiguous():
+        raise ValueError("norm must be a contiguous CUDA float32 tensor")
+    if norm.numel() != (rows if norm_axis == AXIS_ROWS else cols):
+        raise ValueError("norm has the wrong length for norm_axis")
+    if mask_bits is None and want_mask:
+        mask_bits = torch.empty((rows, mask_words_per_row(cols)), dtype=torch.int32, device=W.device)
+    if W_pruned is None and want_pruned:
+        W_pruned = torch.empty_strided((rows, cols), (ld, 1), dtype=W.dtype, device=W.device)
+    need = ctypes.c_size_t(0)
+    _check(load().dass_select_workspace_bytes(rows, cols, int(norm_axis), ctypes.byref(need)), "dass_select_workspace_bytes")
+    if workspace is None:
+        workspace = torch.empty(need.value + 16, dtype=torch.uint8, device=W.device)
+        off = (-workspace.data_ptr()) % 16
+        workspace = workspace[off:off + need.value]
+    code = load().dass_select_unstructured(W.data_ptr(), rows, cols, ld, _dtype_code(W), norm.data_ptr(), int(norm_axis),
+                                           float(alpha), float(sparsity), int(compare_axis), _ptr(mask_bits),
+                                           _ptr(W_pruned), workspace.data_ptr(), workspace.numel(), _stream(stream))
+    _check(code, "dass_select_unstructured")
+    return mask_bits, W_pruned
