@@ -109,4 +109,4 @@ def test_argument_errors():
     assert f(F, 8, 64, 64, 0, F, 1, 1.0, -0.1, 1, F, F, F, 1 << 20, None) == 2
     assert f(F, 8, 64, 68, 0, F, 1, 1.0, 0.5, 1, F, F, F, 1 << 20, None) == 3
     assert f(F, 8, 64, 64, 0, F, 1, 1.0, 0.5, 1, F, F, None, 0, None) == 6
-    assert f(F, 8, 200000, 200000, 0, F, 1, 1.0, 0.5, 1, F, F, F, 1 << 20, None) == 5   # a line does not fit in shared memory
+    assert f(F, 8, 200000, 200000, 0, F, 1, 1.0, 0.5, 1, F, F, F, 1 << 26, None) == 5   # a line does not fit in shared memory
