@@ -288,7 +288,7 @@ def run_ours(args):
                        "parallelism": "independent layers per GPU, no collective" if world > 1 else "single GPU"},
             "stage_ms": {"calib": calib_ms, "score_x3": score_ms, "compress_x3": comp_ms},
             "score_gbs": score_gbs, "compress_gbs": comp_gbs,
-            "roofline": {"bound": "tensor", "kernel": "calib_tc_kernel", "achieved": achieved_tf,
+            "roofline": {"bound": "tensor", "kernel": "calib_tc2_kernel", "achieved": achieved_tf,
                          "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
                          "frac": achieved_tf / peaks["bf16_tflops_sustained"],
                          "frac_of_burst_peak": achieved_tf / peaks["bf16_tflops"], "peak_source": peak_src,

@@ -260,7 +260,7 @@ static EncodeTiledFn encode_tiled_fn()
 
 // Row-major bf16 matrix [rows x cols] with pitch ld: dimension 0 = the contiguous k axis.  Boxes are
 // 64 x box_rows elements with the 128-byte swizzle; out-of-range elements read as zero.
-static bool make_map(CUtensorMap *map, const void *ptr, int64_t rows, int64_t cols, int64_t ld, int box_rows)
+bool tc_make_map(CUtensorMap *map, const void *ptr, int64_t rows, int64_t cols, int64_t ld, int box_rows)
 {
     EncodeTiledFn fn = encode_tiled_fn();
     if (!fn) return false;
@@ -297,13 +297,23 @@ static cudaError_t launch_tc(const CUtensorMap &mx, const CUtensorMap &mg, const
     return cudaGetLastError();
 }
 
+#ifndef DASS_CALIB_PAIR
+#define DASS_CALIB_PAIR 1
+#endif
+dass_status calib_tc2_launch(const void *X, int64_t T, int64_t ldx, const void *Wg, const void *Wu,
+                             int64_t I, int64_t d, int64_t ldw, int act, double *partial, int *status,
+                             cudaStream_t st);   // calib_tc2.cu
+
 dass_status calib_tc_launch(const void *X, int64_t T, int64_t ldx, const void *Wg, const void *Wu,
                             int64_t I, int64_t d, int64_t ldw, int act, double *partial, int *status,
                             cudaStream_t st)
 {
+#if DASS_CALIB_PAIR
+    if (I > TC_BM) return calib_tc2_launch(X, T, ldx, Wg, Wu, I, d, ldw, act, partial, status, st);   // CTA-pair kernel
+#endif
     if (d > 0x7fffffffll - TC_BK || T > 0x7fffffffll - TC_BN || I > 0x7fffffffll - TC_BM) return DASS_ERR_UNSUPPORTED;
     CUtensorMap mx, mg, mu;
-    if (!make_map(&mx, X, T, d, ldx, TC_BN) || !make_map(&mg, Wg, I, d, ldw, TC_BM) || !make_map(&mu, Wu, I, d, ldw, TC_BM))
+    if (!tc_make_map(&mx, X, T, d, ldx, TC_BN) || !tc_make_map(&mg, Wg, I, d, ldw, TC_BM) || !tc_make_map(&mu, Wu, I, d, ldw, TC_BM))
         return DASS_ERR_CUDA;
     TcParams p;
     p.partial = partial; p.status = status; p.align_counter = status + 1;

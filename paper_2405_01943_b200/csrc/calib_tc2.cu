@@ -1,0 +1,338 @@
+// Stage (a) for bf16 inputs, CTA-pair version: the same fused GLU GEMM as calib_tc.cu, but two CTAs (the two
+// SMs of a TPC, a cluster of 2) drive one tcgen05.mma.cta_group::2 of shape 256 x 256:
+//
+//   * each CTA owns 128 neurons (its own Wg and Wu tiles, TMEM lanes 0..127 of its own SM) and loads only HALF of
+//     the 256-token X tile; the hardware feeds both halves of B to both tensor cores.  Per k-slice a CTA therefore
+//     moves 48 KB through shared memory instead of 64 KB and its MMAs read 64 KB instead of 96 KB -- the
+//     single-CTA kernel is limited by exactly that shared-memory traffic (writes 64 + reads 96 bytes per clock
+//     against 128 available).
+//   * the leader CTA (cluster rank 0) issues all MMAs; both CTAs' TMA loads complete on the leader's "full"
+//     barrier; tcgen05.commit multicasts the "slot free" and "accumulators ready" arrivals to both CTAs; the
+//     peer's epilogue warps release the accumulators with remote mbarrier arrives.
+//   * no TMA multicast is used anywhere.
+// Everything else (item order, tile-boundary alignment barrier, L2 eviction hints, lane = neuron epilogue,
+// per-band partial sums, bounded waits) is as in calib_tc.cu.
+#include "tc_common.cuh"
+
+namespace dass {
+
+constexpr int T2_BM = 128;          // neurons per CTA (256 per pair)
+constexpr int T2_BN = 256;          // tokens per tile (each CTA loads 128 of them)
+constexpr int T2_BK = 64;
+constexpr int T2_UMMA_K = 16;
+constexpr int T2_STAGES = 4;
+constexpr int T2_BAND_TILES = 16;
+constexpr int T2_SUPER_BANDS = 16;
+constexpr unsigned long long T2_ALIGN_NS = 20000ull;
+constexpr int T2_THREADS = 192;
+constexpr uint32_t T2_TILE_BYTES = 128 * T2_BK * 2;                 // 16 KB: a 128-row, 64-column bf16 tile
+constexpr uint32_t T2_STAGE_BYTES = 3 * T2_TILE_BYTES;              // Wg + Wu + X half = 48 KB per CTA
+constexpr uint32_t T2_TMEM_COLS = 512;
+constexpr uint32_t T2_SMEM_BYTES = T2_STAGES * T2_STAGE_BYTES + 1024 + 256;
+
+// ------------------------------------------------------------------ cluster / pair PTX wrappers
+__device__ __forceinline__ uint32_t cluster_ctarank()
+{
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all()
+{
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// shared::cluster address of the same shared-memory location in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t smem_addr, uint32_t rank)
+{
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr)
+{
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// TMA load whose completion bytes are credited to a barrier that may live in the peer CTA of the pair
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap *map, uint32_t bar_cluster_addr,
+                                                 int x, int y, uint64_t policy)
+{
+    asm volatile("cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint"
+                 " [%0], [%1, {%3, %4}], [%2], %5;"
+                 ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar_cluster_addr), "r"(x), "r"(y), "l"(policy)
+                 : "memory");
+}
+__device__ __forceinline__ void tmem_alloc_pair(uint32_t dst_smem, uint32_t ncols)
+{
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish_pair()
+{
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t ncols)
+{
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void umma_bf16_pair(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile("{\n\t.reg .pred p;\n\t"
+                 "setp.ne.b32 p, %4, 0;\n\t"
+                 "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+                 ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// arrives (once the MMAs issued so far have completed) on the barrier at this shared-memory offset in every CTA of `mask`
+__device__ __forceinline__ void umma_commit_pair(uint32_t bar, uint16_t mask)
+{
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                 ::"r"(bar), "h"(mask) : "memory");
+}
+
+struct T2Params {
+    double *partial;     // [bands][I]
+    int *status;
+    int *align_counter;
+    int64_t T, I, d;
+    int64_t neuron_pairs, token_tiles, bands, items, k_blocks;   // items = neuron_pairs * bands (one per CTA pair)
+};
+
+struct T2Item { int64_t np, band; };
+
+__device__ __forceinline__ T2Item t2_decode(const T2Params &p, int64_t idx)
+{
+    const int64_t per_super = p.neuron_pairs * T2_SUPER_BANDS;
+    const int64_t sb = idx / per_super;
+    const int64_t rem = idx - sb * per_super;
+    const int64_t left = p.bands - sb * T2_SUPER_BANDS;
+    const int64_t nb = left < T2_SUPER_BANDS ? left : T2_SUPER_BANDS;
+    T2Item c;
+    c.np = rem / nb;
+    c.band = sb * T2_SUPER_BANDS + (rem - c.np * nb);
+    return c;
+}
+
+template <int ACT>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(T2_THREADS, 1)
+calib_tc2_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_wg,
+                 const __grid_constant__ CUtensorMap map_wu, const T2Params p)
+{
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;
+    uint8_t *aligned = smem_raw + (base - raw);
+    uint64_t *bars = reinterpret_cast<uint64_t *>(aligned + T2_STAGES * T2_STAGE_BYTES);
+    const uint32_t bar_full = smem_u32(bars);                     // [T2_STAGES], used in the leader CTA only
+    const uint32_t bar_empty = bar_full + 8 * T2_STAGES;          // [T2_STAGES], one set per CTA
+    const uint32_t bar_acc_full = bar_empty + 8 * T2_STAGES;      // per CTA
+    const uint32_t bar_acc_empty = bar_acc_full + 8;              // leader CTA only: 8 epilogue warps arrive
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * T2_STAGES + 2);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_ctarank();                      // 0 = leader
+    const int64_t cluster_id = blockIdx.x >> 1;
+    const int64_t nclusters = gridDim.x >> 1;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < T2_STAGES; ++s) {
+            mbar_init(bar_full + 8 * s, 1);
+            mbar_init(bar_empty + 8 * s, 1);
+        }
+        mbar_init(bar_acc_full, 1);
+        mbar_init(bar_acc_empty, 8);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) {
+        tmem_alloc_pair(smem_u32(tmem_slot), T2_TMEM_COLS);
+        tmem_relinquish_pair();
+    }
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();            // both CTAs' barriers are initialised and both TMEM allocations exist
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ TMA producer (one per CTA)
+        if (lane == 0) {
+            uint32_t stage = 0, phase = 0;
+            bool ok = true;
+            const uint64_t pol_w = l2_policy_evict_last();
+            const uint64_t pol_x = l2_policy_evict_first();
+            const uint32_t leader_full = map_to_cta(bar_full, 0);
+            int64_t round = 0;
+            for (int64_t idx = cluster_id; idx < p.items && ok; idx += nclusters, ++round) {
+                const T2Item c = t2_decode(p, idx);
+                const int64_t tt0 = c.band * T2_BAND_TILES;
+                const int64_t tt1 = tt0 + T2_BAND_TILES < p.token_tiles ? tt0 + T2_BAND_TILES : p.token_tiles;
+                const int64_t left = p.items - round * nclusters;
+                const int round_ctas = 2 * (int)(left < nclusters ? left : nclusters);
+                const int w_row = (int)(c.np * 2 * T2_BM + rank * T2_BM);
+                for (int64_t tt = tt0; tt < tt1 && ok; ++tt) {
+                    {   // tile-boundary alignment of all CTAs of the round (bounded wait), see calib_tc.cu
+                        const int t_in_item = (int)(tt - tt0);
+                        const int target = (int)(round * gridDim.x) * T2_BAND_TILES + round_ctas * (t_in_item + 1);
+                        atomicAdd(p.align_counter, 1);
+                        const unsigned long long t0 = global_ns();
+                        while (*reinterpret_cast<volatile int *>(p.align_counter) < target && global_ns() - t0 < T2_ALIGN_NS) { }
+                    }
+                    const int x_row = (int)(tt * T2_BN + rank * (T2_BN / 2));
+                    for (int64_t kb = 0; kb < p.k_blocks; ++kb) {
+                        if (!mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
+                        const uint32_t sbase = base + stage * T2_STAGE_BYTES;
+                        const uint32_t fb = leader_full + 8 * stage;
+                        if (rank == 0) mbar_arrive_expect_tx(bar_full + 8 * stage, 2 * T2_STAGE_BYTES);   // both CTAs' bytes
+                        tma_load_2d_pair(sbase, &map_wg, fb, (int)(kb * T2_BK), w_row, pol_w);
+                        tma_load_2d_pair(sbase + T2_TILE_BYTES, &map_wu, fb, (int)(kb * T2_BK), w_row, pol_w);
+                        tma_load_2d_pair(sbase + 2 * T2_TILE_BYTES, &map_x, fb, (int)(kb * T2_BK), x_row, pol_x);
+                        if (++stage == T2_STAGES) { stage = 0; phase ^= 1u; }
+                    }
+                }
+                if (tt1 - tt0 < T2_BAND_TILES) atomicAdd(p.align_counter, (int)(T2_BAND_TILES - (tt1 - tt0)));
+            }
+            if (!ok) { *abort_flag = 1; atomicExch(p.status, (int)DASS_ERR_TIMEOUT); }
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        // ------------------------------------------------------------ MMA issuer (leader CTA only)
+        if (lane == 0 && rank == 0) {
+            constexpr uint32_t idesc = idesc_bf16_f32(2 * T2_BM, T2_BN);
+            uint32_t stage = 0, phase = 0, tile = 0;
+            bool ok = true;
+            for (int64_t idx = cluster_id; idx < p.items && ok; idx += nclusters) {
+                const T2Item c = t2_decode(p, idx);
+                const int64_t tt0 = c.band * T2_BAND_TILES;
+                const int64_t tt1 = tt0 + T2_BAND_TILES < p.token_tiles ? tt0 + T2_BAND_TILES : p.token_tiles;
+                for (int64_t tt = tt0; tt < tt1 && ok; ++tt, ++tile) {
+                    if (!mbar_wait(bar_acc_empty, (tile & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+                    tc_fence_after();
+                    for (int64_t kb = 0; kb < p.k_blocks; ++kb) {
+                        if (!mbar_wait(bar_full + 8 * stage, phase, abort_flag)) { ok = false; break; }
+                        tc_fence_after();
+                        const uint32_t sbase = base + stage * T2_STAGE_BYTES;
+                        const uint64_t dg = smem_desc_sw128(sbase);
+                        const uint64_t du = smem_desc_sw128(sbase + T2_TILE_BYTES);
+                        const uint64_t dx = smem_desc_sw128(sbase + 2 * T2_TILE_BYTES);
+#pragma unroll
+                        for (int k = 0; k < T2_BK / T2_UMMA_K; ++k) {
+                            const uint32_t acc = (kb > 0 || k > 0) ? 1u : 0u;
+                            const uint64_t koff = (uint64_t)(k * T2_UMMA_K * 2 / 16);
+                            umma_bf16_pair(tmem_base, dg + koff, dx + koff, idesc, acc);
+                            umma_bf16_pair(tmem_base + T2_BN, du + koff, dx + koff, idesc, acc);
+                        }
+                        umma_commit_pair(bar_empty + 8 * stage, (uint16_t)3);   // slot free in both CTAs
+                        if (++stage == T2_STAGES) { stage = 0; phase ^= 1u; }
+                    }
+                    if (ok) umma_commit_pair(bar_acc_full, (uint16_t)3);        // accumulators ready in both CTAs
+                }
+            }
+            if (!ok) { *abort_flag = 1; atomicExch(p.status, (int)DASS_ERR_TIMEOUT); }
+        }
+        __syncwarp();
+    } else {
+        // ------------------------------------------------------------ epilogue (4 warps, this CTA's 128 neurons)
+        const int quad = warp & 3;
+        const uint32_t lane_addr = tmem_base + ((uint32_t)(quad * 32) << 16);
+        const uint32_t leader_acc_empty = map_to_cta(bar_acc_empty, 0);
+        uint32_t tile = 0;
+        bool ok = true;
+        for (int64_t idx = cluster_id; idx < p.items && ok; idx += nclusters) {
+            const T2Item c = t2_decode(p, idx);
+            const int64_t tt0 = c.band * T2_BAND_TILES;
+            const int64_t tt1 = tt0 + T2_BAND_TILES < p.token_tiles ? tt0 + T2_BAND_TILES : p.token_tiles;
+            double acc = 0.0;
+            for (int64_t tt = tt0; tt < tt1 && ok; ++tt, ++tile) {
+                if (!mbar_wait(bar_acc_full, tile & 1u, abort_flag)) { ok = false; break; }
+                tc_fence_after();
+                float s = 0.0f;
+#pragma unroll 1
+                for (int col = 0; col < T2_BN; col += 32) {
+                    uint32_t g[32], u[32];
+                    tmem_ld_32(lane_addr + col, g);
+                    tmem_ld_32(lane_addr + T2_BN + col, u);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) {
+                        const float h = glu_h<ACT>(__uint_as_float(g[j]), __uint_as_float(u[j]));
+                        s = fmaf(h, h, s);
+                    }
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) {                         // release the accumulators to the leader's MMA warp
+                    if (rank == 0) mbar_arrive(bar_acc_empty);
+                    else mbar_arrive_cluster(leader_acc_empty);
+                }
+                acc += (double)s;
+            }
+            const int64_t neuron = c.np * 2 * T2_BM + rank * T2_BM + quad * 32 + lane;
+            if (ok && neuron < p.I) p.partial[c.band * p.I + neuron] = acc;
+        }
+        if (!ok && lane == 0) { *abort_flag = 1; atomicExch(p.status, (int)DASS_ERR_TIMEOUT); }
+    }
+    // ---------------------------------------------------------------- teardown
+    tc_fence_before();
+    __syncthreads();
+    if (*abort_flag) {
+        for (int i = 0; i < 20; ++i) __nanosleep(1000000);   // failure path: let issued copies / MMAs land
+        __syncthreads();
+    }
+    cluster_sync_all();            // the peer no longer signals into this CTA's shared memory or uses the pair's TMEM
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc_pair(tmem_base, T2_TMEM_COLS);
+    }
+}
+
+// ------------------------------------------------------------------ host side
+bool tc_make_map(CUtensorMap *map, const void *ptr, int64_t rows, int64_t cols, int64_t ld, int box_rows);   // calib_tc.cu
+int64_t calib_tc_parts(int64_t T, int64_t I);                                                                 // calib_tc.cu
+int device_sm_count();                                                                                        // dass_abi.cu
+
+template <int ACT>
+static cudaError_t launch_tc2(const CUtensorMap &mx, const CUtensorMap &mg, const CUtensorMap &mu, const T2Params &p,
+                              int grid, cudaStream_t st)
+{
+    static bool configured = false;
+    if (!configured) {
+        const cudaError_t e = cudaFuncSetAttribute(calib_tc2_kernel<ACT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                   (int)T2_SMEM_BYTES);
+        if (e != cudaSuccess) return e;
+        configured = true;
+    }
+    calib_tc2_kernel<ACT><<<grid, T2_THREADS, T2_SMEM_BYTES, st>>>(mx, mg, mu, p);
+    return cudaGetLastError();
+}
+
+// CTA-pair launch; same contract as calib_tc_launch (partials per band, status word, alignment counter behind it).
+dass_status calib_tc2_launch(const void *X, int64_t T, int64_t ldx, const void *Wg, const void *Wu,
+                             int64_t I, int64_t d, int64_t ldw, int act, double *partial, int *status,
+                             cudaStream_t st)
+{
+    if (d > 0x7fffffffll - T2_BK || T > 0x7fffffffll - T2_BN || I > 0x7fffffffll - 2 * T2_BM) return DASS_ERR_UNSUPPORTED;
+    CUtensorMap mx, mg, mu;
+    if (!tc_make_map(&mx, X, T, d, ldx, T2_BN / 2) || !tc_make_map(&mg, Wg, I, d, ldw, T2_BM) ||
+        !tc_make_map(&mu, Wu, I, d, ldw, T2_BM))
+        return DASS_ERR_CUDA;
+    T2Params p;
+    p.partial = partial; p.status = status; p.align_counter = status + 1;
+    p.T = T; p.I = I; p.d = d;
+    p.neuron_pairs = (I + 2 * T2_BM - 1) / (2 * T2_BM);
+    p.token_tiles = (T + T2_BN - 1) / T2_BN;
+    p.bands = calib_tc_parts(T, I);
+    p.items = p.neuron_pairs * p.bands;
+    p.k_blocks = (d + T2_BK - 1) / T2_BK;
+    const int64_t max_pairs = device_sm_count() / 2;
+    const int grid = 2 * (int)(p.items < max_pairs ? p.items : max_pairs);
+    cudaError_t e;
+    switch (act) {
+    case DASS_ACT_SILU: e = launch_tc2<DASS_ACT_SILU>(mx, mg, mu, p, grid, st); break;
+    case DASS_ACT_GELU_TANH: e = launch_tc2<DASS_ACT_GELU_TANH>(mx, mg, mu, p, grid, st); break;
+    default: e = launch_tc2<DASS_ACT_RELU>(mx, mg, mu, p, grid, st); break;
+    }
+    return e == cudaSuccess ? DASS_OK : DASS_ERR_CUDA;
+}
+
+}  // namespace dass
