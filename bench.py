@@ -59,9 +59,9 @@ def stage_b_bytes(cfg, compress=True):
 
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per launch from one ncu capture of this very
 # command on the default workload; see profiles/.  None where the kernel changed after the capture.
-NCU_DRAM_BYTES = {"llama2_70b": {"calib": 113.21e9 + 23.0e6,                                  # one launch, T = 262144
-                                 "score": (469.9 + 445.7 + 469.9 + 445.0 + 470.0 + 447.1) * 1e6,   # gate + up + down
-                                 "compress": (499.1 + 203.9 + 499.1 + 204.0 + 500.2 + 216.0) * 1e6}}
+NCU_DRAM_BYTES = {"llama2_70b": {"calib": 126.73e9 + 24.7e6,                                  # one launch, T = 262144
+                                 "score": (470.3 + 445.1 + 470.3 + 445.5 + 471.0 + 455.8) * 1e6,   # gate + up + down
+                                 "compress": (499.1 + 203.7 + 499.1 + 204.0 + 537.6 + 238.3) * 1e6}}
 
 
 def roofline_b(kernel, algorithmic_bytes, in_step_ms, isolated_ms, peaks, peak_src, traffic):
