@@ -85,6 +85,14 @@ dass_status dass_calib_accumulate(const void *X, int64_t T, int64_t ldx,
  * the kernel gave up (the results of that call are then invalid; the context stays usable). */
 dass_status dass_calib_status(const void *workspace, void *cuda_stream);
 
+/* Failure-path self-test (no counterpart in the paper).  Every wait inside the tensor-core kernels is bounded; when one
+ * runs out the kernel records DASS_ERR_TIMEOUT in its status word, drains and returns, and the CUDA context stays
+ * usable.  This call exercises exactly that mechanism without disturbing the GPU: a one-warp kernel waits, with the same
+ * bounded-wait routine, on a barrier that nothing will ever complete, for at most limit_us microseconds (1 .. 1 000 000),
+ * and then writes the outcome to status_word (a 4-byte aligned device int), which dass_calib_status reads.
+ * Errors: NULL / SHAPE (limit out of range) / ALIGN / CUDA. */
+dass_status dass_selftest_wait_timeout(void *status_word, int64_t limit_us, void *cuda_stream);
+
 /* The paper has no counterpart for this entry point: it exists for callers that cannot allocate.
  * Some users of this library may not call cudaMalloc where they calibrate -- code inside a framework's
  * memory-planned region or allocator callback, plugins that own nothing but the tensors they are

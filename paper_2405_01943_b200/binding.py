@@ -27,7 +27,7 @@ EXPORTS = (
     "dass_calib_workspace_bytes", "dass_calib_accumulate", "dass_calib_accumulate_static", "dass_calib_status",
     "dass_norm_finalize",
     "dass_score_nm", "dass_compress_nm", "dass_select_workspace_bytes", "dass_select_unstructured",
-    "dass_status_string", "dass_version",
+    "dass_selftest_wait_timeout", "dass_status_string", "dass_version",
 )
 
 
@@ -73,6 +73,8 @@ def load() -> ctypes.CDLL:
     lib.dass_select_unstructured.restype = ctypes.c_int
     lib.dass_select_unstructured.argtypes = [vp, i64, i64, i64, ctypes.c_int, vp, ctypes.c_int, ctypes.c_float,
                                              ctypes.c_double, ctypes.c_int, vp, vp, vp, sz, vp]
+    lib.dass_selftest_wait_timeout.restype = ctypes.c_int
+    lib.dass_selftest_wait_timeout.argtypes = [vp, i64, vp]
     lib.dass_status_string.restype = ctypes.c_char_p
     lib.dass_status_string.argtypes = [ctypes.c_int]
     lib.dass_version.restype = ctypes.c_int
@@ -288,3 +290,11 @@ def select_unstructured(W: torch.Tensor, norm: torch.Tensor, norm_axis: int, alp
                                            _ptr(W_pruned), workspace.data_ptr(), workspace.numel(), _stream(stream))
     _check(code, "dass_select_unstructured")
     return mask_bits, W_pruned
+
+
+def selftest_wait_timeout(status_word: torch.Tensor, limit_us: int, stream: Optional[torch.cuda.Stream] = None) -> None:
+    """Launches the bounded-wait self-test; read the outcome with calib_status(status_word)."""
+    if not status_word.is_cuda or status_word.dtype != torch.int32 or status_word.numel() < 1:
+        raise ValueError("status_word must be a CUDA int32 tensor")
+    _check(load().dass_selftest_wait_timeout(status_word.data_ptr(), int(limit_us), _stream(stream)),
+           "dass_selftest_wait_timeout")

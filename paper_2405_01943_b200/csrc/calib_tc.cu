@@ -297,6 +297,27 @@ static cudaError_t launch_tc(const CUtensorMap &mx, const CUtensorMap &mg, const
     return cudaGetLastError();
 }
 
+// Self-test of the failure path: one thread waits, with the kernels' bounded wait, on an mbarrier that nothing will
+// ever arrive at, and reports what the calibration kernels report when a wait runs out.
+__global__ void bounded_wait_selftest_kernel(int *status, unsigned long long limit_ns)
+{
+    __shared__ uint64_t bar;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) {
+        abort_flag = 0;
+        mbar_init(smem_u32(&bar), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        const bool done = mbar_wait(smem_u32(&bar), 0u, &abort_flag, limit_ns);
+        *status = done ? 0 : (int)DASS_ERR_TIMEOUT;
+    }
+}
+
+cudaError_t bounded_wait_selftest_launch(int *status, unsigned long long limit_ns, cudaStream_t st)
+{
+    bounded_wait_selftest_kernel<<<1, 32, 0, st>>>(status, limit_ns);
+    return cudaGetLastError();
+}
+
 #ifndef DASS_CALIB_PAIR
 #define DASS_CALIB_PAIR 1
 #endif

@@ -24,6 +24,8 @@ dass_status calib_tc_launch(const void *X, int64_t T, int64_t ldx, const void *W
                             int64_t I, int64_t d, int64_t ldw, int act, double *partial, int *status,
                             cudaStream_t st);
 
+cudaError_t bounded_wait_selftest_launch(int *status, unsigned long long limit_ns, cudaStream_t st);
+
 int device_sm_count()
 {
     static int cached_dev = -1, cached_sms = 0;
@@ -135,6 +137,17 @@ dass_status dass_calib_status(const void *workspace, void *cuda_stream)
     if (cudaMemcpyAsync(&host, workspace, sizeof(int), cudaMemcpyDeviceToHost, st) != cudaSuccess) return DASS_ERR_CUDA;
     if (cudaStreamSynchronize(st) != cudaSuccess) return DASS_ERR_CUDA;
     return host == 0 ? DASS_OK : DASS_ERR_TIMEOUT;
+}
+
+dass_status dass_selftest_wait_timeout(void *status_word, int64_t limit_us, void *cuda_stream)
+{
+    if (!status_word) return DASS_ERR_NULL;
+    if (limit_us < 1 || limit_us > 1000000) return DASS_ERR_SHAPE;
+    if (reinterpret_cast<uintptr_t>(status_word) & 3u) return DASS_ERR_ALIGN;
+    if (bounded_wait_selftest_launch(static_cast<int *>(status_word), (unsigned long long)limit_us * 1000ull,
+                                     static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
+        return DASS_ERR_CUDA;
+    return DASS_OK;
 }
 
 dass_status dass_norm_finalize(const double *sumsq, int64_t I, float *norm, void *cuda_stream)

@@ -41,8 +41,9 @@ __device__ __forceinline__ unsigned long long global_ns()
     asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
     return t;
 }
-// Bounded wait: true when the phase completed, false after TC_WAIT_NS (or when another role aborted).
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag)
+// Bounded wait: true when the phase completed, false after limit_ns (or when another role aborted).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag,
+                                          unsigned long long limit_ns = TC_WAIT_NS)
 {
     if (mbar_try_wait(bar, parity)) return true;
     const unsigned long long t0 = global_ns();
@@ -50,7 +51,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
         if (mbar_try_wait(bar, parity)) return true;
         if ((spin & 255u) == 0) {
             if (*abort_flag) return false;
-            if (global_ns() - t0 > TC_WAIT_NS) return false;
+            if (global_ns() - t0 > limit_ns) return false;
         }
     }
     return false;
