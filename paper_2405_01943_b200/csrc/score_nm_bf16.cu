@@ -277,7 +277,7 @@ __device__ __noinline__ KeepWords<F_SLAB> exact_keep_cols(TileWords<F_SLAB> t, S
 
 // ---------------------------------------------------------------- groups along the rows (gate / up)
 template <int M, bool NORM_COLS>
-__global__ void __launch_bounds__(F_THREADS, F_MIN_BLOCKS) score_rows_bf16_kernel(const ScoreFastParams p)
+__global__ void __launch_bounds__(F_THREADS, M == 8 ? 2 : F_MIN_BLOCKS) score_rows_bf16_kernel(const ScoreFastParams p)
 {
     constexpr int NP = M * (M - 1) / 2;
     constexpr int STAGES = ring_stages(M);
@@ -390,7 +390,7 @@ __global__ void __launch_bounds__(F_THREADS, F_MIN_BLOCKS) score_rows_bf16_kerne
 
 // ---------------------------------------------------------------- groups along the columns (down)
 template <int M, bool NORM_COLS>
-__global__ void __launch_bounds__(F_THREADS, F_MIN_BLOCKS) score_cols_bf16_kernel(const ScoreFastParams p)
+__global__ void __launch_bounds__(F_THREADS, M == 8 ? 3 : F_MIN_BLOCKS) score_cols_bf16_kernel(const ScoreFastParams p)
 {
     constexpr int NP = M * (M - 1) / 2;
     constexpr int G = 8 / M;             // groups inside a lane's 8 columns
