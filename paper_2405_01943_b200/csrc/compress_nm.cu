@@ -5,7 +5,8 @@
 // fields are produced in registers and packed into 32-bit words with warp shuffles (groups along the
 // columns: four lanes share a word) or directly per lane (groups along the rows: a lane's 8 columns
 // fill whole words).  Bandwidth-bound: reads W and one mask bit per weight, writes n_keep/m of W plus
-// the fields.
+// the fields.  These generic kernels serve fp32 weights and bf16 row groups; bf16 column groups take the
+// permute-table kernel of compress_nm_bf16.cu.
 #include "dass_device.cuh"
 
 namespace dass {

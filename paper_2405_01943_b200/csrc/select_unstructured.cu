@@ -2,13 +2,15 @@
 // line -- a column of Wg / Wu (all neurons at one input: input-balanced) or a row of Wd (output-balanced) --
 // the floor(s * L) weights with the lowest Eq. 4 / Eq. 5 score are pruned.  No sort: an exact radix select.
 //
-// A CTA caches its lines (two of them) in shared memory and finds, per line, the k-th largest 64-bit key in
-// eight 8-bit passes; the key is the bit pattern of the exact double product |w| * scale, which orders like the
-// real score.  A last pass keeps every key above the threshold and, among keys equal to it, the ones with the
-// lowest indices (found with an ordered prefix count), which is the oracle's "higher score first, lower index
-// first" order.  Lines that are matrix rows are read with 16-byte loads; lines that are matrix columns are read
-// two adjacent columns at a time (4 or 8 bytes per row, neighbouring CTAs share the sectors through L2) and
-// their mask bits are OR-ed into the packed mask with atomics (the mask is zeroed first).
+// A CTA caches its line(s) in shared memory and finds the threshold in two stages.  Stage A works on the rounded
+// products p = fl32(|w| * scale), four 8-bit passes; rounding is monotone, so p decides every pair of weights
+// whose rounded products differ.  Only if more products equal the threshold than may stay does stage B repeat the
+// selection among those with the exact double products as keys (eight passes); exact ties are then broken towards
+// the lower index with an ordered prefix count -- the oracle's "higher score first, lower index first".
+// Lines that are matrix rows (one per CTA, 16-byte loads) are emitted by the same kernel.  Lines that are matrix
+// columns are read two adjacent columns per CTA (neighbouring CTAs share the 32-byte sectors through L2); the
+// kernel publishes (tau32, exact, tau64, cut) per column and select_emit_cols_kernel applies them in a streaming
+// pass with coalesced rows.
 #include <cmath>
 #include <type_traits>
 
@@ -17,7 +19,6 @@
 namespace dass {
 
 constexpr int U_THREADS = 256;
-constexpr int U_MAX_LINES = 2;        // lines per CTA: 1 when lines are rows, 2 adjacent columns otherwise
 constexpr int U_WARPS = U_THREADS / 32;
 
 // What the selection found for one line; enough to decide every element of the line locally:
