@@ -113,6 +113,17 @@ __global__ void __launch_bounds__(CF_THREADS, 4) compress_cols_bf16_kernel(const
 #pragma unroll
     for (int s = 0; s < CF_STAGES - 1; ++s) issue(s);
 
+    // mask words of a unit (one per row; the lane's byte is cut out later), fetched one unit ahead
+    auto load_mask_words = [&](int st_, int g_, uint32_t (&mw)[CF_SLAB]) {
+        const int64_t r0 = (int64_t)g_ * CF_SLAB;
+        const int64_t c0 = (int64_t)st_ * CF_COLS + lane * 8;
+#pragma unroll
+        for (int i = 0; i < CF_SLAB; ++i)
+            mw[i] = (c0 < p.cols && r0 + i < p.rows) ? __ldg(p.mask + (r0 + i) * p.wpr + (c0 >> 5)) : 0u;
+    };
+    uint32_t mw_next[CF_SLAB];
+    if (u_begin < u_end) load_mask_words(strip, g, mw_next);
+
     int stage = 0;
     for (int64_t u = u_begin; u < u_end; ++u) {
         const int64_t r0 = (int64_t)g * CF_SLAB;
@@ -124,9 +135,8 @@ __global__ void __launch_bounds__(CF_THREADS, 4) compress_cols_bf16_kernel(const
 
         uint32_t mb[CF_SLAB];
 #pragma unroll
-        for (int i = 0; i < CF_SLAB; ++i)
-            mb[i] = (nvalid > 0 && r0 + i < p.rows)
-                        ? (__ldg(p.mask + (r0 + i) * p.wpr + (c0 >> 5)) >> (8 * (lane & 3))) & 0xffu : 0u;
+        for (int i = 0; i < CF_SLAB; ++i) mb[i] = (mw_next[i] >> (8 * (lane & 3))) & 0xffu;
+        if (u + 1 < u_end) load_mask_words(strip, g, mw_next);              // (strip, g) already point at unit u + 1
         asm volatile("cp.async.wait_group %0;" ::"n"(CF_STAGES - 2) : "memory");
         uint4 v[CF_SLAB];
 #pragma unroll
