@@ -52,6 +52,8 @@ def _load():
         lib.dass_oracle_act.argtypes = [ctypes.c_int, ctypes.c_double]
         lib.dass_oracle_calib_sumsq.restype = None
         lib.dass_oracle_calib_sumsq.argtypes = [f32p, i64, i64, f32p, f32p, i64, i64, i64, ctypes.c_int, f64p]
+        lib.dass_oracle_feature_sumsq.restype = None
+        lib.dass_oracle_feature_sumsq.argtypes = [f32p, i64, i64, i64, f64p]
         lib.dass_oracle_glu_row.restype = None
         lib.dass_oracle_glu_row.argtypes = [f32p, f32p, f32p, i64, i64, i64, ctypes.c_int, f64p]
         lib.dass_oracle_norm.restype = None
@@ -109,6 +111,17 @@ def calib_sumsq(X, Wg, Wu, act_kind: int, sumsq=None) -> np.ndarray:
     assert sumsq.dtype == np.float64 and sumsq.shape == (I,) and sumsq.flags.c_contiguous
     _load().dass_oracle_calib_sumsq(_p(X, ctypes.c_float), T, d, _p(Wg, ctypes.c_float), _p(Wu, ctypes.c_float),
                                     I, d, d, int(act_kind), _p(sumsq, ctypes.c_double))
+    return sumsq
+
+
+def feature_sumsq(X, sumsq=None) -> np.ndarray:
+    """sumsq[j] (+)= sum_t X[t,j]^2: the squared input-feature norms of Eq. 1."""
+    X = _f32(X)
+    T, d = X.shape
+    if sumsq is None:
+        sumsq = np.zeros(d, dtype=np.float64)
+    assert sumsq.dtype == np.float64 and sumsq.shape == (d,) and sumsq.flags.c_contiguous
+    _load().dass_oracle_feature_sumsq(_p(X, ctypes.c_float), T, d, d, _p(sumsq, ctypes.c_double))
     return sumsq
 
 

@@ -22,6 +22,7 @@
  *
  * Pins (what each function is checked against, see tests/test_oracle_*.py):
  *   activations      closed forms, odd-part identities, torch fp64 functional
+ *   feature_sumsq    numpy sum of squares, linearity, known vectors
  *   calib_sumsq      numpy matmul special case, one-hot closed forms,
  *                    batching / linearity / power-of-two scaling invariants
  *   scale, score_nm  exact-rational brute force over all N:M subsets,
@@ -85,6 +86,21 @@ void dass_oracle_calib_sumsq(const float *X, int64_t T, int64_t ldx,
             s += h * h;
         }
         sumsq[i] += s;
+    }
+}
+
+/* Eq. 1's input-feature norms (Wanda, used by the paper for the attention projections):
+ * sumsq[j] += sum_t X[t,j]^2, the squared l2 norm of feature j over all tokens. */
+void dass_oracle_feature_sumsq(const float *X, int64_t T, int64_t d, int64_t ldx, double *sumsq)
+{
+#pragma omp parallel for schedule(static)
+    for (int64_t j = 0; j < d; ++j) {
+        double s = 0.0;
+        for (int64_t t = 0; t < T; ++t) {
+            double x = (double)X[t * ldx + j];
+            s += x * x;
+        }
+        sumsq[j] += s;
     }
 }
 

@@ -134,6 +134,33 @@ def test_norm_is_correctly_rounded_sqrt():
     assert n[1] == 2.0 and n[0] == 0.0
 
 
+def test_feature_sumsq_matches_numpy_and_known_vector():
+    rng = np.random.default_rng(31)
+    X = rng.standard_normal((29, 13)).astype(np.float32)
+    ref = (X.astype(np.float64) ** 2).sum(0)
+    np.testing.assert_allclose(oracle.feature_sumsq(X), ref, rtol=1e-14)
+    acc = oracle.feature_sumsq(X[:10])
+    oracle.feature_sumsq(X[10:], acc)
+    np.testing.assert_allclose(acc, ref, rtol=1e-14)
+    K = np.array([[3.0, 0.0], [4.0, 2.0]], dtype=np.float32)          # columns (3,4) and (0,2): 25 and 4
+    assert oracle.feature_sumsq(K).tolist() == [25.0, 4.0]
+
+
+def test_wanda_eq1_through_score_nm():
+    """Eq. 1 on an attention-style projection: |W_ij| * ||X_j||_2 compared per output row."""
+    rng = np.random.default_rng(32)
+    X = rng.standard_normal((40, 16)).astype(np.float32)
+    W = (rng.standard_normal((12, 16)) * 0.02).astype(np.float32)
+    norm = oracle.norm_from_sumsq(oracle.feature_sumsq(X))
+    mask, _ = oracle.score_nm(W, norm, AXIS_COLS, 1.0, 2, 4, AXIS_COLS)
+    score = np.abs(W.astype(np.float64)) * np.linalg.norm(X.astype(np.float64), axis=0).astype(np.float32).astype(np.float64)[None, :]
+    ref = np.zeros_like(mask)
+    for r in range(12):
+        for c0 in range(0, 16, 4):
+            ref[r, c0 + np.argsort(-score[r, c0:c0 + 4], kind="stable")[:2]] = 1
+    assert np.array_equal(mask, ref)
+
+
 # --------------------------------------------------------------------------- scale recipe
 
 def test_scale_special_exponents():
