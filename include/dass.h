@@ -167,6 +167,17 @@ dass_status dass_compress_nm(const void *W, const uint32_t *mask_bits,
                              int n_keep, int m, dass_axis group_axis,
                              void *values, uint32_t *meta, void *cuda_stream);
 
+/* Eq. 1's input-feature norms (Wanda; the paper prunes the attention projections with it, Section 4.1 "Sparsity"):
+ *     sumsq[j] += sum_{t < T} X[t,j]^2      for j in [0, d)
+ * X [T x d, ldx] in `dt`; sumsq [d] doubles, in/out (accumulates over calls, fixed reduction order inside a call).
+ * dass_norm_finalize turns it into ||X_j||_2; dass_score_nm / dass_select_unstructured with norm_axis = COLS and row
+ * lines (group_axis / compare_axis = COLS), alpha = 1, then are Wanda for any weight matrix [out x d].
+ * workspace: dass_feature_workspace_bytes(T, d) bytes, 16-byte aligned.
+ * Errors: NULL / DTYPE / SHAPE / ALIGN / WORKSPACE / CUDA. */
+dass_status dass_feature_workspace_bytes(int64_t T, int64_t d, size_t *bytes /* HOST */);
+dass_status dass_feature_sumsq(const void *X, int64_t T, int64_t d, int64_t ldx, dass_dtype dt,
+                               double *sumsq, void *workspace, size_t workspace_bytes, void *cuda_stream);
+
 /* Unstructured DaSS selection (Section 3, "Pruning Granularity"): inside every comparison line the
  * floor(sparsity * L) weights with the lowest Eq. 4 / Eq. 5 score are pruned, L being the line length.
  *     compare_axis = ROWS: a line is a whole column (all rows at one input: "input-balanced", the paper's

@@ -27,7 +27,8 @@ EXPORTS = (
     "dass_calib_workspace_bytes", "dass_calib_accumulate", "dass_calib_accumulate_static", "dass_calib_status",
     "dass_norm_finalize",
     "dass_score_nm", "dass_compress_nm", "dass_select_workspace_bytes", "dass_select_unstructured",
-    "dass_selftest_wait_timeout", "dass_status_string", "dass_version",
+    "dass_selftest_wait_timeout", "dass_feature_workspace_bytes", "dass_feature_sumsq",
+    "dass_status_string", "dass_version",
 )
 
 
@@ -75,6 +76,10 @@ def load() -> ctypes.CDLL:
                                              ctypes.c_double, ctypes.c_int, vp, vp, vp, sz, vp]
     lib.dass_selftest_wait_timeout.restype = ctypes.c_int
     lib.dass_selftest_wait_timeout.argtypes = [vp, i64, vp]
+    lib.dass_feature_workspace_bytes.restype = ctypes.c_int
+    lib.dass_feature_workspace_bytes.argtypes = [i64, i64, ctypes.POINTER(sz)]
+    lib.dass_feature_sumsq.restype = ctypes.c_int
+    lib.dass_feature_sumsq.argtypes = [vp, i64, i64, i64, ctypes.c_int, vp, vp, sz, vp]
     lib.dass_status_string.restype = ctypes.c_char_p
     lib.dass_status_string.argtypes = [ctypes.c_int]
     lib.dass_version.restype = ctypes.c_int
@@ -298,3 +303,23 @@ def selftest_wait_timeout(status_word: torch.Tensor, limit_us: int, stream: Opti
         raise ValueError("status_word must be a CUDA int32 tensor")
     _check(load().dass_selftest_wait_timeout(status_word.data_ptr(), int(limit_us), _stream(stream)),
            "dass_selftest_wait_timeout")
+
+
+def feature_sumsq(X: torch.Tensor, sumsq: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None,
+                  stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
+    """sumsq[j] += sum_t X[t,j]^2 (Eq. 1's squared input-feature norms). Returns sumsq (float64 [d])."""
+    T, d, ldx = _matrix(X, "X")
+    if sumsq is None:
+        sumsq = torch.zeros(d, dtype=torch.float64, device=X.device)
+    if sumsq.dtype != torch.float64 or not sumsq.is_cuda or sumsq.numel() != d or not sumsq.is_contiguous():
+        raise ValueError("sumsq must be a contiguous CUDA float64 tensor of d elements")
+    need = ctypes.c_size_t(0)
+    _check(load().dass_feature_workspace_bytes(T, d, ctypes.byref(need)), "dass_feature_workspace_bytes")
+    if workspace is None:
+        workspace = torch.empty(need.value + 16, dtype=torch.uint8, device=X.device)
+        off = (-workspace.data_ptr()) % 16
+        workspace = workspace[off:off + need.value]
+    code = load().dass_feature_sumsq(X.data_ptr(), T, d, ldx, _dtype_code(X), sumsq.data_ptr(), workspace.data_ptr(),
+                                     workspace.numel(), _stream(stream))
+    _check(code, "dass_feature_sumsq")
+    return sumsq
