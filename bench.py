@@ -208,14 +208,14 @@ def run_ours(args):
     if not torch.cuda.is_available():
         raise SystemExit("bench.py: no CUDA device; the DaSS path has no CPU fallback (use --impl reference for the oracle)")
     from paper_2405_01943_b200 import binding, build
-    if build.is_stale() and os.environ.get("DASS_NO_BUILD") != "1":
-        if local_rank == 0:
-            build.build()
     torch.cuda.set_device(local_rank)
     device = torch.device("cuda", local_rank)
     if world > 1:
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=device)
+    if os.environ.get("DASS_NO_BUILD") != "1" and local_rank == 0 and build.is_stale():
+        build.build()                    # one rank per node builds; the others wait at the barrier below
+    if world > 1:
         dist.barrier()
     binding.load()
 
