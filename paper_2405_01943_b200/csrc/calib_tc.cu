@@ -318,9 +318,7 @@ cudaError_t bounded_wait_selftest_launch(int *status, unsigned long long limit_n
     return cudaGetLastError();
 }
 
-#ifndef DASS_CALIB_PAIR
-#define DASS_CALIB_PAIR 1
-#endif
+constexpr bool TC_USE_PAIR_KERNEL = true;   // layers with more than one neuron tile take the CTA-pair kernel (calib_tc2.cu)
 dass_status calib_tc2_launch(const void *X, int64_t T, int64_t ldx, const void *Wg, const void *Wu,
                              int64_t I, int64_t d, int64_t ldw, int act, double *partial, int *status,
                              cudaStream_t st);   // calib_tc2.cu
@@ -329,9 +327,7 @@ dass_status calib_tc_launch(const void *X, int64_t T, int64_t ldx, const void *W
                             int64_t I, int64_t d, int64_t ldw, int act, double *partial, int *status,
                             cudaStream_t st)
 {
-#if DASS_CALIB_PAIR
-    if (I > TC_BM) return calib_tc2_launch(X, T, ldx, Wg, Wu, I, d, ldw, act, partial, status, st);   // CTA-pair kernel
-#endif
+    if (TC_USE_PAIR_KERNEL && I > TC_BM) return calib_tc2_launch(X, T, ldx, Wg, Wu, I, d, ldw, act, partial, status, st);
     if (d > 0x7fffffffll - TC_BK || T > 0x7fffffffll - TC_BN || I > 0x7fffffffll - TC_BM) return DASS_ERR_UNSUPPORTED;
     CUtensorMap mx, mg, mu;
     if (!tc_make_map(&mx, X, T, d, ldx, TC_BN) || !tc_make_map(&mg, Wg, I, d, ldw, TC_BM) || !tc_make_map(&mu, Wu, I, d, ldw, TC_BM))

@@ -35,17 +35,12 @@ struct ScoreFastParams {
 };
 
 constexpr int F_THREADS = 256;
-#ifndef F_MIN_BLOCKS
-#define F_MIN_BLOCKS 4
-#endif
+constexpr int F_MIN_BLOCKS = 4;      // CTAs per SM the 2:4 kernels are compiled for (64 registers: measured best)
 constexpr int F_COLS = 256;          // columns per warp strip
 // prefetch depth of the shared-memory slab ring (slabs of R rows x 512 bytes per warp)
 __host__ __device__ constexpr int ring_stages(int rows_per_unit) { return rows_per_unit >= 8 ? 2 : 3; }
 __host__ __device__ constexpr int ring_bytes(int rows_per_unit) { return (F_THREADS / 32) * ring_stages(rows_per_unit) * rows_per_unit * 512; }
-#ifndef F_SLAB_ROWS
-#define F_SLAB_ROWS 4
-#endif
-constexpr int F_SLAB = F_SLAB_ROWS;  // rows per unit when groups run along the columns (4 or 8)
+constexpr int F_SLAB = 4;            // rows per unit when groups run along the columns
 
 // Out of line on purpose: the double-precision sqrt / pow sequences would otherwise inflate the register
 // budget of the streaming loops, and they run once per strip or per 32 rows only.
