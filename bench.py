@@ -262,7 +262,7 @@ def run_ours(args):
     score_gbs, comp_gbs = sb / (score_ms * 1e-3) / 1e9, cb / (comp_ms * 1e-3) / 1e9
 
     # stage (b) alone: the same launches back to back, away from the power-capped GEMM, so that the
-    # bandwidth-bound kernels are judged at the clocks they get by themselves
+    # bandwidth-bound kernels are measured at the clocks they get by themselves
     iso = isolated_stage_b(path, pool, alpha, iters=args.iso_iters) if args.iso_iters > 0 else None
 
     # end to end: pinned host inputs -> device -> path -> results back to the host, every step

@@ -46,7 +46,7 @@ typedef enum {
     DASS_ERR_SHAPE = 2,        /* non-positive size, extent not divisible by m, bad n_keep */
     DASS_ERR_ALIGN = 3,        /* pointer or leading dimension not aligned as required */
     DASS_ERR_DTYPE = 4,        /* unknown dass_dtype / dass_act / dass_axis value */
-    DASS_ERR_UNSUPPORTED = 5,  /* a valid request this build has no kernel for */
+    DASS_ERR_UNSUPPORTED = 5,  /* a valid request the library has no kernel for */
     DASS_ERR_WORKSPACE = 6,    /* workspace NULL or smaller than the query says */
     DASS_ERR_CUDA = 7,         /* a CUDA runtime / driver call failed */
     DASS_ERR_TIMEOUT = 8       /* a bounded device-side wait ran out (reported by dass_calib_status) */

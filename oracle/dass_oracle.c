@@ -32,7 +32,7 @@
  *   compress_nm      round trip to the pruned matrix, metadata well-formedness
  *   pack_mask        bit-by-bit re-derivation in the tests
  * The absolute layout of mask words / metadata and the tie-break are readings
- * of this build (the paper is silent): those are "parity unpinned" in the
+ * of this library (the paper is silent): those are "parity unpinned" in the
  * sense that only this project's documents fix them.
  */
 #include <math.h>
