@@ -476,7 +476,7 @@ def main():
     ap.add_argument("--config", default="llama2_70b", choices=sorted(synth.CONFIGS))
     ap.add_argument("--tokens", type=int, default=0, help="override the number of calibration tokens (debugging)")
     ap.add_argument("--pool", type=int, default=3, help="distinct synthetic layers cycled through the steps")
-    ap.add_argument("--e2e-steps", type=int, default=4)
+    ap.add_argument("--e2e-steps", type=int, default=6)
     ap.add_argument("--iso-iters", type=int, default=20, help="iterations of the stage-(b)-only timing loop (0 = skip)")
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
