@@ -18,8 +18,6 @@
 
 namespace dass {
 
-constexpr int U_THREADS = 256;
-constexpr int U_WARPS = U_THREADS / 32;
 
 // What the selection found for one line; enough to decide every element of the line locally:
 // keep iff p > tau32, or p == tau32 and (not exact, or k64 > tau64, or k64 == tau64 and index <= cut).
@@ -82,14 +80,14 @@ struct LineState {
 
 // One warp per line: finds the bucket (8-bit digit) that holds the krem-th largest candidate.
 // Returns through lane-uniform values: the digit, the number of candidates in higher buckets, the bucket count.
-__device__ __forceinline__ void find_bucket(const uint32_t *hist_line /* [U_WARPS][256] */, uint32_t krem, int lane,
+__device__ __forceinline__ void find_bucket(const uint32_t *hist_line /* [nwarps][256] */, int nwarps, uint32_t krem, int lane,
                                             uint32_t &digit, uint32_t &greater, uint32_t &bucket)
 {
     uint32_t cnt[8], lane_sum = 0u;
 #pragma unroll
     for (int b = 0; b < 8; ++b) {
         uint32_t c = 0u;
-        for (int w = 0; w < U_WARPS; ++w) c += hist_line[w * 256 + lane * 8 + b];
+        for (int w = 0; w < nwarps; ++w) c += hist_line[w * 256 + lane * 8 + b];
         cnt[b] = c;
         lane_sum += c;
     }
@@ -124,8 +122,10 @@ __device__ __forceinline__ void find_bucket(const uint32_t *hist_line /* [U_WARP
 // them stay and the line is done.  Otherwise stage B repeats the selection among those equal products with the exact
 // double products as keys (eight passes), and the emit pass breaks remaining exact ties towards the lower index.
 template <bool BF16, bool LINE_IS_ROW>
-__global__ void __launch_bounds__(U_THREADS) select_unstructured_kernel(const SelectParams p)
+__global__ void __launch_bounds__(LINE_IS_ROW ? 256 : 512) select_unstructured_kernel(const SelectParams p)
 {
+    constexpr int U_THREADS = LINE_IS_ROW ? 256 : 512;   // row lines: 3 CTAs per SM; column lines: one CTA (2 lines) per SM
+    constexpr int U_WARPS = U_THREADS / 32;
     using elem_t = typename std::conditional<BF16, uint16_t, uint32_t>::type;
     constexpr int U_LINES = LINE_IS_ROW ? 1 : 2;
     extern __shared__ __align__(16) unsigned char u_smem[];
@@ -231,7 +231,7 @@ __global__ void __launch_bounds__(U_THREADS) select_unstructured_kernel(const Se
         __syncthreads();
         if (warp < nl) {
             uint32_t digit, greater, bucket;
-            find_bucket(hist + warp * U_WARPS * 256, st[warp].krem, lane, digit, greater, bucket);
+            find_bucket(hist + warp * U_WARPS * 256, U_WARPS, st[warp].krem, lane, digit, greater, bucket);
             if (lane == 0) {
                 st[warp].tau32 |= digit << shift;
                 st[warp].krem -= greater;
@@ -278,7 +278,7 @@ __global__ void __launch_bounds__(U_THREADS) select_unstructured_kernel(const Se
             __syncthreads();
             if (warp < nl && st[warp].exact) {
                 uint32_t digit, greater, bucket;
-                find_bucket(hist + warp * U_WARPS * 256, st[warp].krem, lane, digit, greater, bucket);
+                find_bucket(hist + warp * U_WARPS * 256, U_WARPS, st[warp].krem, lane, digit, greater, bucket);
                 if (lane == 0) {
                     st[warp].tau64 |= (unsigned long long)digit << shift;
                     st[warp].krem -= greater;
@@ -487,7 +487,8 @@ size_t select_smem_bytes(int64_t L, bool bf16, bool line_is_row)
 {
     const int64_t lpad = (L + 7) / 8 * 8;
     const size_t lines = line_is_row ? 1 : 2;
-    return lines * lpad * (bf16 ? 2 : 4) + lines * U_WARPS * 256 * sizeof(uint32_t);
+    const size_t warps = line_is_row ? 8 : 16;
+    return lines * lpad * (bf16 ? 2 : 4) + lines * warps * 256 * sizeof(uint32_t);
 }
 
 template <bool BF16, bool ROW>
@@ -497,7 +498,7 @@ static cudaError_t launch_select(const SelectParams &p, size_t smem, cudaStream_
     if (e != cudaSuccess) return e;
     constexpr int lines = ROW ? 1 : 2;
     const int64_t grid = (p.nlines + lines - 1) / lines;
-    select_unstructured_kernel<BF16, ROW><<<(unsigned)grid, U_THREADS, smem, st>>>(p);
+    select_unstructured_kernel<BF16, ROW><<<(unsigned)grid, ROW ? 256 : 512, smem, st>>>(p);
     return cudaGetLastError();
 }
 
