@@ -111,3 +111,21 @@ def test_stage_b_full_matrices_bit_exact(layer):
     assert_stage_b_equal(got, ref)
     mk = unpack_mask(got["words"], cfg.I)
     assert np.all(mk.reshape(cfg.d, cfg.I // cfg.m, cfg.m).sum(-1) == cfg.n_keep)
+
+
+@pytest.mark.parametrize("layer_id", [39, 79])
+def test_70b_stream_other_layers_sampled_neurons(layer_id):
+    """The 80-layer stream draws every layer from its own seed: check two more of them (middle and last)
+    on sampled neurons over all tokens, as for layer 0 above."""
+    cfg = synth.CONFIGS["llama2_70b"]
+    X = synth.make_x(cfg, DEV)
+    Wg, Wu, _ = synth.make_weights(cfg, DEV, layer=layer_id)
+    got = _gpu_sumsq(cfg, X, Wg, Wu).cpu().numpy()
+    idx = np.unique(np.concatenate([np.argsort(-got)[:4], np.linspace(0, cfg.I - 1, 12).astype(np.int64)]))
+    sel = torch.from_numpy(idx).to(DEV)
+    wg, wu = to_np32(Wg[sel]), to_np32(Wu[sel])
+    ref = np.zeros(len(idx), dtype=np.float64)
+    for t0 in range(0, cfg.T, 32768):
+        oracle.calib_sumsq(to_np32(X[t0:t0 + 32768]), wg, wu, ORACLE_ACT[cfg.act], ref)
+    rel = np.abs(np.sqrt(got[idx]) - np.sqrt(ref)) / np.sqrt(ref)
+    assert rel.max() <= 2e-3, f"layer {layer_id}: sampled-neuron norm error {rel.max():.3e}"
