@@ -52,6 +52,9 @@ CONFIGS = {
     "llama2_7b": LayerConfig("llama2_7b", d=4096, I=11008, T=128 * 2048, dtype="bf16", act="silu",
                              n_keep=2, m=4, sigma=0.02, row_frac=0.005, row_scale=4.0,
                              outlier_frac=0.01, seed=1, layers=32),
+    "llama2_13b": LayerConfig("llama2_13b", d=5120, I=13824, T=128 * 2048, dtype="bf16", act="silu",
+                              n_keep=2, m=4, sigma=0.02, row_frac=0.005, row_scale=4.0,
+                              outlier_frac=0.01, seed=6, layers=40),
     "relullama_7b": LayerConfig("relullama_7b", d=4096, I=11008, T=128 * 2048, dtype="bf16", act="relu",
                                 n_keep=2, m=4, sigma=0.02, row_frac=0.005, row_scale=4.0,
                                 outlier_frac=0.01, seed=5, layers=32),

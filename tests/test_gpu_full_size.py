@@ -1,4 +1,4 @@
-"""Parity at the full sizes of the four large layer shapes (LLaMA2-7B, Mistral-7B, Gemma-7B, LLaMA2-70B),
+"""Parity at the full sizes of the large layer shapes (LLaMA2-7B / 13B / 70B, Mistral-7B, Gemma-7B),
 in the launch configuration the benchmark times (whole 262144-token calibration batch in one call).
 
 The oracle cannot redo 10^13..10^14 flops, so stage (a) is checked on outputs it can compute one by one:
@@ -18,7 +18,7 @@ from paper_2405_01943_b200.binding import AXIS_COLS, AXIS_ROWS
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda"
-NAMES = ["llama2_7b", "mistral_7b", "gemma_7b", "llama2_70b"]
+NAMES = ["llama2_7b", "llama2_13b", "mistral_7b", "gemma_7b", "llama2_70b"]
 ORACLE_ACT = {"silu": oracle.ACT_SILU, "gelu_tanh": oracle.ACT_GELU_TANH}
 T_PREFIX = 300
 N_SAMPLED = 64
