@@ -56,6 +56,11 @@ def _load():
         lib.dass_oracle_feature_sumsq.argtypes = [f32p, i64, i64, i64, f64p]
         lib.dass_oracle_glu_row.restype = None
         lib.dass_oracle_glu_row.argtypes = [f32p, f32p, f32p, i64, i64, i64, ctypes.c_int, f64p]
+        lib.dass_oracle_round_bf16.restype = ctypes.c_double
+        lib.dass_oracle_round_bf16.argtypes = [ctypes.c_double]
+        lib.dass_oracle_mlp_forward.restype = None
+        lib.dass_oracle_mlp_forward.argtypes = [f32p, i64, i64, f32p, f32p, i64, i64, i64, f32p, i64,
+                                                ctypes.c_int, ctypes.c_int, f64p, f64p]
         lib.dass_oracle_norm.restype = None
         lib.dass_oracle_norm.argtypes = [f64p, i64, f32p]
         lib.dass_oracle_scale.restype = ctypes.c_float
@@ -133,6 +138,28 @@ def glu_row(x, Wg, Wu, act_kind: int) -> np.ndarray:
     _load().dass_oracle_glu_row(_p(x, ctypes.c_float), _p(Wg, ctypes.c_float), _p(Wu, ctypes.c_float),
                                 I, d, d, int(act_kind), _p(h, ctypes.c_double))
     return h
+
+
+def round_bf16(v: float) -> float:
+    """v rounded to the nearest bf16 value, ties to even."""
+    return float(_load().dass_oracle_round_bf16(float(v)))
+
+
+def mlp_forward(X, Wg, Wu, Wd, act_kind: int, h_round: bool, want_h: bool = False):
+    """Eq. 2 then Eq. 3 for every token: z = (act(x Wg^T) * (x Wu^T)) Wd^T.
+
+    ``h_round`` rounds the intermediate activation to bf16 before Eq. 3.  Returns Z [T x d] (fp64), or
+    (Z, H) with H [T x I] as Eq. 3 used it."""
+    X, Wg, Wu, Wd = _f32(X), _f32(Wg), _f32(Wu), _f32(Wd)
+    T, d = X.shape
+    I, d2 = Wg.shape
+    assert d2 == d and Wu.shape == Wg.shape and Wd.shape == (d, I)
+    Z = np.zeros((T, d), dtype=np.float64)
+    H = np.zeros((T, I), dtype=np.float64) if want_h else None
+    _load().dass_oracle_mlp_forward(_p(X, ctypes.c_float), T, d, _p(Wg, ctypes.c_float), _p(Wu, ctypes.c_float),
+                                    I, d, d, _p(Wd, ctypes.c_float), I, int(act_kind), int(bool(h_round)),
+                                    _p(Z, ctypes.c_double), _p(H, ctypes.c_double) if want_h else None)
+    return (Z, H) if want_h else Z
 
 
 def norm_from_sumsq(sumsq) -> np.ndarray:

@@ -30,6 +30,9 @@
  *                    magnitude-only reduction for alpha = 0 / equal norms
  *   select_unstructured   monotonicity invariants of the dependency metric
  *   compress_nm      round trip to the pruned matrix, metadata well-formedness
+ *   round_bf16       torch's float32 -> bfloat16 conversion, hand-picked ties
+ *   mlp_forward      hand-worked fixture, numpy float64 matmul composition,
+ *                    identity / one-hot down projections, linearity in Wd
  *   pack_mask        bit-by-bit re-derivation in the tests
  * The absolute layout of mask words / metadata and the tie-break are readings
  * of this library (the paper is silent): those are "parity unpinned" in the
@@ -116,6 +119,57 @@ void dass_oracle_glu_row(const float *x, const float *Wg, const float *Wu,
             u += (double)x[k] * (double)Wu[i * ldw + k];
         }
         h[i] = dass_oracle_act(act, g) * u;
+    }
+}
+
+/* Round a double to the nearest bf16 value (8 significant bits, float's exponent
+ * range), ties to even; the result is returned as a double.  Written out from
+ * the format's definition: find the binade, scale so that one unit in the last
+ * place is 1, round to the nearest integer with ties to even, scale back. */
+double dass_oracle_round_bf16(double v)
+{
+    if (v == 0.0 || isnan(v) || isinf(v)) return v;
+    int e;
+    (void)frexp(v, &e);            /* |v| = f * 2^e with f in [0.5, 1)  ->  binade exponent e - 1 */
+    int ex = e - 1;
+    if (ex < -126) ex = -126;      /* subnormal range: fixed spacing 2^-133 */
+    const double ulp = ldexp(1.0, ex - 7);
+    const double r = nearbyint(v / ulp) * ulp;      /* default rounding mode: to nearest, ties to even */
+    if (fabs(r) >= ldexp(1.0, 128)) return v > 0 ? INFINITY : -INFINITY;
+    return r;
+}
+
+/* ---- the pruned layer's forward pass, Eq. 2 then Eq. 3 ---------------------
+ * y_t = act(x_t Wg^T) * (x_t Wu^T),  z_t = y_t Wd^T, for every token t, with whatever
+ * (pruned) weights are passed in.  h_round = 1 rounds every y to bf16 before Eq. 3,
+ * which is what a model whose activations are stored in bf16 does between the two
+ * projections; h_round = 0 keeps y in double.  Z is [T x d] (ld = d); H, when not
+ * NULL, receives y as used by Eq. 3, [T x I] (ld = I). */
+void dass_oracle_mlp_forward(const float *X, int64_t T, int64_t ldx,
+                             const float *Wg, const float *Wu, int64_t I, int64_t d, int64_t ldw,
+                             const float *Wd, int64_t ldd, int act, int h_round,
+                             double *Z, double *H)
+{
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int64_t t = 0; t < T; ++t) {
+        double *y = (double *)malloc((size_t)I * sizeof(double));
+        for (int64_t i = 0; i < I; ++i) {
+            double g = 0.0, u = 0.0;
+            for (int64_t k = 0; k < d; ++k) {
+                double x = (double)X[t * ldx + k];
+                g += x * (double)Wg[i * ldw + k];
+                u += x * (double)Wu[i * ldw + k];
+            }
+            double h = dass_oracle_act(act, g) * u;
+            y[i] = h_round ? dass_oracle_round_bf16(h) : h;
+            if (H) H[t * I + i] = y[i];
+        }
+        for (int64_t n = 0; n < d; ++n) {
+            double z = 0.0;
+            for (int64_t i = 0; i < I; ++i) z += y[i] * (double)Wd[n * ldd + i];
+            Z[t * d + n] = z;
+        }
+        free(y);
     }
 }
 
