@@ -197,6 +197,31 @@ dass_status dass_select_unstructured(const void *W, int64_t rows, int64_t cols, 
                                      uint32_t *mask_bits, void *W_pruned,
                                      void *workspace, size_t workspace_bytes, void *cuda_stream);
 
+/* Forward pass of one GLU MLP layer with the weights given, Eq. 2 then Eq. 3 (Section 2.2):
+ *     H[t,i] = act(X[t,:] . Wg[i,:]) * (X[t,:] . Wu[i,:])        rounded to `dt`
+ *     Z[t,n] = sum_i H[t,i] * Wd[n,i]                             rounded to `dt`
+ * Called with the pruned weights (zeros stored in place, as dass_score_nm's W_pruned writes them) it gives the
+ * pruned layer's output, which is what the next layer's calibration reads when a model is pruned layer by
+ * layer.  X [T x d, ldx], Wg / Wu [I x d, ldw], Wd [d x I, ldd], Z [T x d, ldz], all in `dt`, row-major, device.
+ * bf16: tensor-core path, fp32 accumulation, H held in bf16 between the two contractions (as a bf16 model holds
+ * it).  f32: plain fp32 FMA path, H held in fp32.
+ * workspace: 256-byte aligned device scratch holding the status word and H for a chunk of tokens.  Any size
+ * from *min_bytes up is accepted; with *full_bytes all T tokens go through in one pass, with less the tokens are
+ * processed in chunks (whole multiples of 4096 or 256 tokens).  Its first word receives the device status that
+ * dass_calib_status reads (DASS_ERR_TIMEOUT if a bounded device-side wait gave up).  It must not be shared by
+ * calls that may overlap on the device.  After the call the workspace still holds the last chunk's H, row-major
+ * from byte 256 on, with a pitch of I rounded up to 8 (bf16) or 4 (f32) elements -- after a one-pass call, all of H.
+ * Errors: NULL / DTYPE / SHAPE (sizes < 1, pitches below the row length) / ALIGN (X, Wg, Wu, Wd 16-byte aligned,
+ * their pitches multiples of 16 bytes) / UNSUPPORTED (a dimension beyond the kernels' 32-bit coordinates) /
+ * WORKSPACE / CUDA. */
+dass_status dass_mlp_forward_workspace_bytes(int64_t T, int64_t d, int64_t I, dass_dtype dt,
+                                             size_t *min_bytes /* HOST, nullable */, size_t *full_bytes /* HOST, nullable */);
+dass_status dass_mlp_forward(const void *X, int64_t T, int64_t ldx,
+                             const void *Wg, const void *Wu, int64_t I, int64_t d, int64_t ldw,
+                             const void *Wd, int64_t ldd, dass_dtype dt, dass_act act,
+                             void *Z, int64_t ldz,
+                             void *workspace, size_t workspace_bytes, void *cuda_stream);
+
 /* ------------------------------------------------------------------ misc */
 const char *dass_status_string(dass_status s);   /* static string, never NULL */
 int dass_version(void);                          /* major * 10000 + minor * 100 + patch */

@@ -28,6 +28,7 @@ EXPORTS = (
     "dass_norm_finalize",
     "dass_score_nm", "dass_compress_nm", "dass_select_workspace_bytes", "dass_select_unstructured",
     "dass_selftest_wait_timeout", "dass_feature_workspace_bytes", "dass_feature_sumsq",
+    "dass_mlp_forward_workspace_bytes", "dass_mlp_forward",
     "dass_status_string", "dass_version",
 )
 
@@ -80,6 +81,11 @@ def load() -> ctypes.CDLL:
     lib.dass_feature_workspace_bytes.argtypes = [i64, i64, ctypes.POINTER(sz)]
     lib.dass_feature_sumsq.restype = ctypes.c_int
     lib.dass_feature_sumsq.argtypes = [vp, i64, i64, i64, ctypes.c_int, vp, vp, sz, vp]
+    lib.dass_mlp_forward_workspace_bytes.restype = ctypes.c_int
+    lib.dass_mlp_forward_workspace_bytes.argtypes = [i64, i64, i64, ctypes.c_int, ctypes.POINTER(sz), ctypes.POINTER(sz)]
+    lib.dass_mlp_forward.restype = ctypes.c_int
+    lib.dass_mlp_forward.argtypes = [vp, i64, i64, vp, vp, i64, i64, i64, vp, i64, ctypes.c_int, ctypes.c_int,
+                                     vp, i64, vp, sz, vp]
     lib.dass_status_string.restype = ctypes.c_char_p
     lib.dass_status_string.argtypes = [ctypes.c_int]
     lib.dass_version.restype = ctypes.c_int
@@ -323,3 +329,52 @@ def feature_sumsq(X: torch.Tensor, sumsq: Optional[torch.Tensor] = None, workspa
                                      workspace.numel(), _stream(stream))
     _check(code, "dass_feature_sumsq")
     return sumsq
+
+
+# ----------------------------------------------------------------------------- forward pass (Eq. 2, Eq. 3)
+
+def mlp_forward_workspace_bytes(T: int, d: int, I: int, dtype: torch.dtype) -> Tuple[int, int]:
+    """(smallest accepted, one-pass) workspace sizes of mlp_forward."""
+    lo, full = ctypes.c_size_t(0), ctypes.c_size_t(0)
+    code = load().dass_mlp_forward_workspace_bytes(int(T), int(d), int(I), BF16 if dtype == torch.bfloat16 else F32,
+                                                   ctypes.byref(lo), ctypes.byref(full))
+    _check(code, "dass_mlp_forward_workspace_bytes")
+    return int(lo.value), int(full.value)
+
+
+def mlp_forward_workspace(nbytes: int, device="cuda") -> torch.Tensor:
+    """A 256-byte aligned uint8 CUDA tensor of nbytes."""
+    buf = torch.empty(nbytes + 256, dtype=torch.uint8, device=device)
+    off = (-buf.data_ptr()) % 256
+    return buf[off:off + nbytes]
+
+
+def mlp_forward(X: torch.Tensor, Wg: torch.Tensor, Wu: torch.Tensor, Wd: torch.Tensor, act: int,
+                Z: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None,
+                stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
+    """Z = (act(X Wg^T) * (X Wu^T)) Wd^T in X's dtype, with the weights as given (pruned = zeros in place).
+
+    Without ``workspace`` a one-pass workspace is allocated; a smaller one makes the call process the
+    tokens in chunks.  The workspace's status word is read by calib_status(workspace)."""
+    T, d, ldx = _matrix(X, "X")
+    I, d2, ldw = _matrix(Wg, "Wg")
+    I3, d3, ldw3 = _matrix(Wu, "Wu")
+    d4, I4, ldd = _matrix(Wd, "Wd")
+    if (d2, I3, d3, ldw3) != (d, I, d, ldw) or (d4, I4) != (d, I):
+        raise ValueError("X [T x d], Wg / Wu [I x d] (same pitch) and Wd [d x I] must agree in d and I")
+    if not (Wg.dtype == Wu.dtype == Wd.dtype == X.dtype):
+        raise ValueError("X, Wg, Wu, Wd must have one dtype")
+    if Z is None:
+        Z = torch.empty((T, d), dtype=X.dtype, device=X.device)
+    Tz, dz, ldz = _matrix(Z, "Z")
+    if (Tz, dz) != (T, d) or Z.dtype != X.dtype:
+        raise ValueError("Z must be [T x d] in X's dtype")
+    if workspace is None:
+        workspace = mlp_forward_workspace(mlp_forward_workspace_bytes(T, d, I, X.dtype)[1], X.device)
+    if not workspace.is_cuda or workspace.dtype != torch.uint8:
+        raise ValueError("workspace must be a CUDA uint8 tensor (see mlp_forward_workspace)")
+    code = load().dass_mlp_forward(X.data_ptr(), T, ldx, Wg.data_ptr(), Wu.data_ptr(), I, d, ldw,
+                                   Wd.data_ptr(), ldd, _dtype_code(X), int(act), Z.data_ptr(), ldz,
+                                   workspace.data_ptr(), workspace.numel(), _stream(stream))
+    _check(code, "dass_mlp_forward")
+    return Z
