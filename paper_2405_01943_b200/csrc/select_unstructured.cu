@@ -2,13 +2,13 @@
 // line -- a column of Wg / Wu (all neurons at one input: input-balanced) or a row of Wd (output-balanced) --
 // the floor(s * L) weights with the lowest Eq. 4 / Eq. 5 score are pruned.  No sort: an exact radix select.
 //
-// A CTA caches its line(s) in shared memory and finds the threshold in two stages.  Stage A works on the rounded
-// products p = fl32(|w| * scale), four 8-bit passes; rounding is monotone, so p decides every pair of weights
-// whose rounded products differ.  Only if more products equal the threshold than may stay does stage B repeat the
-// selection among those with the exact double products as keys (eight passes); exact ties are then broken towards
-// the lower index with an ordered prefix count -- the oracle's "higher score first, lower index first".
-// Lines that are matrix rows (one per CTA, 16-byte loads) are emitted by the same kernel.  Lines that are matrix
-// columns are read two adjacent columns per CTA (neighbouring CTAs share the 32-byte sectors through L2); the
+// The order of the oracle, "higher score first, lower index first", is the order of a three-part key: the
+// rounded product fl32(|w| * scale), then the exact double product, then the index counted from the top.  Its
+// k-th largest value per line is found 11 bits at a time with shared-memory histograms, and a line stops as soon
+// as the bucket at the cut holds exactly the survivors still wanted (after two or three passes on real data;
+// exact products and indices are consulted only where rounded products tie across the cut).
+// Lines that are matrix rows: one CTA per row, the row cached in shared memory, outputs written by the same CTA.
+// Lines that are matrix columns: one CTA per strip of 8 adjacent columns, re-read from L2 on every pass; the
 // kernel publishes (tau32, exact, tau64, cut) per column and select_emit_cols_kernel applies them in a streaming
 // pass with coalesced rows.
 #include <cmath>
@@ -30,16 +30,16 @@ struct LineResult {
 
 struct SelectParams {
     const void *W;
-    void *Wp;            // nullable
-    uint32_t *mask;      // nullable
-    const float *scale;  // precomputed fl32(norm^alpha)
-    struct LineResult *results;   // per-line thresholds (column lines only: a second, streaming kernel emits)
+    void *Wp;            // nullable (row lines only: the kernel emits)
+    uint32_t *mask;      // nullable (row lines only)
+    const float *scale;  // precomputed fl32(norm^alpha), padded with zeros to a multiple of 8
+    struct LineResult *results;   // per-column thresholds (column lines only: a second, streaming kernel emits)
     int64_t rows, cols, ld;
-    int64_t wpr;
+    int64_t wpr;         // mask words per matrix row
     int64_t L;           // line length
-    int64_t nlines;
     int64_t lpad;        // L rounded up to 8
     uint32_t k;          // survivors per line
+    int idx_bits;        // bits of L - 1 (at least 1): width of the index part of the key
     int scale_along_line;   // 1: scale[e] varies along the line; 0: scale[line]
 };
 
@@ -53,122 +53,222 @@ __global__ void scale_vector_kernel(const float *__restrict__ norm, int64_t n, i
     else if (i < npad) out[i] = 0.0f;
 }
 
-template <bool BF16>
-__device__ __forceinline__ float abs_of(uint32_t raw)
-{
-    return BF16 ? __uint_as_float((raw & 0x7fffu) << 16) : __uint_as_float(raw & 0x7fffffffu);
-}
+// ---------------------------------------------------------------- radix select on a three-part key
+// The order "higher score first, lower index first" is the order of the key (p, r, ~index), compared part by
+// part: p = bits of fl32(|w| * scale) (rounding is monotone, so p decides every pair whose rounded products
+// differ), r = bits of the exact double product minus a per-line base (decides pairs whose rounded products are
+// equal), and the index counted down from the top (lower index first).  The k-th largest key of a line is found
+// digit by digit, 11 bits per pass, with one shared-memory histogram of 2048 bins per line.  A line is decided as
+// soon as the bucket that holds the k-th key holds exactly as many candidates as are still to be kept: all of
+// them stay, and "key >= chosen prefix" is the rule; most lines end inside p, after two or three passes.
+constexpr int HB = 11;                          // bits per digit
+constexpr int HBINS = 1 << HB;
+constexpr int HWORDS = HBINS + HBINS / 64;      // a pad word per 64 bins: lanes that scan 64 bins each hit 32 banks
+__device__ __forceinline__ uint32_t hslot(uint32_t bin) { return bin + (bin >> 6); }
 
-// Adds 1 to bin `digit` of a shared-memory histogram for every lane with `active` set.  Lanes of the warp that hit
-// the same bin are combined into one atomic (the top digits of a line are nearly all equal).
-__device__ __forceinline__ void hist_add(uint32_t *h, uint32_t digit, bool active)
-{
-    const unsigned act = __ballot_sync(FULL_MASK, active);
-    if (active) {
-        const unsigned peers = __match_any_sync(act, digit);
-        if ((threadIdx.x & 31) == __ffs(peers) - 1) atomicAdd(h + digit, (uint32_t)__popc(peers));
-    }
-}
+enum : int { STAGE_ROUNDED = 0, STAGE_EXACT = 1, STAGE_INDEX = 2 };
 
-struct LineState {
-    unsigned long long tau64;   // threshold of the exact stage
-    uint32_t tau32;             // threshold among the rounded products (bit pattern)
-    uint32_t krem;              // survivors still to be taken at the current stage
-    uint32_t neq;               // candidates in the last chosen bucket
-    uint32_t exact;             // 1: rounded products tie across the cut, the exact stage decides
+struct Line {                    // selection state of one comparison line (shared memory)
+    unsigned long long tau64;    // digits chosen so far of r = (bits of the exact product) - base
+    unsigned long long base;
+    uint32_t tau32;              // digits chosen so far of p
+    uint32_t tauidx;             // digits chosen so far of (idx_top - index)
+    uint32_t krem;               // survivors still to be taken among the current candidates
+    uint32_t pending;            // 1 until the line is decided
+    uint32_t done_stage;         // part of the key in which it was decided
+    uint32_t pad_;
 };
 
-// One warp per line: finds the bucket (8-bit digit) that holds the krem-th largest candidate.
-// Returns through lane-uniform values: the digit, the number of candidates in higher buckets, the bucket count.
-__device__ __forceinline__ void find_bucket(const uint32_t *hist_line /* [nwarps][256] */, int nwarps, uint32_t krem, int lane,
-                                            uint32_t &digit, uint32_t &greater, uint32_t &bucket)
+// The digit being counted: bits [shift, shift + bits) of the current part of the key.  A part ends when its
+// digits reach bit `stop` (the bits below are known to be zero) or bit 0.
+struct Sched { int stage, shift, bits, stop; };
+
+__device__ __forceinline__ void sched_begin(Sched &s, int stage, int key_bits, int stop)
 {
-    uint32_t cnt[8], lane_sum = 0u;
-#pragma unroll
-    for (int b = 0; b < 8; ++b) {
-        uint32_t c = 0u;
-        for (int w = 0; w < nwarps; ++w) c += hist_line[w * 256 + lane * 8 + b];
-        cnt[b] = c;
-        lane_sum += c;
+    s.stage = stage;
+    s.bits = key_bits < HB ? key_bits : HB;
+    s.shift = key_bits - s.bits;
+    s.stop = stop;
+}
+
+// Moves to the next digit; false when the whole key has been used (cannot happen while a line is pending: the
+// index part makes all keys distinct).  `long_exact`: some line's threshold product is a float denormal, where the
+// distance between neighbouring floats is not 2^29 doubles: r is then the whole 63-bit pattern (base 0).
+template <bool BF16>
+__device__ __forceinline__ bool sched_next(Sched &s, bool long_exact, int idx_bits)
+{
+    if (s.shift > 0 && s.shift > s.stop) {
+        const int b = s.shift < HB ? s.shift : HB;
+        s.shift -= b;
+        s.bits = b;
+        return true;
     }
-    uint32_t v = lane_sum;                          // becomes the sum over lanes >= this one
+    if (s.stage == STAGE_ROUNDED) {
+        // equal rounded products: the exact products lie within half a float ulp = 2^28 doubles of the threshold,
+        // so r < 2^30; a bf16 x float product has at most 32 significant bits: the low 21 bits of r are zero
+        if (long_exact) sched_begin(s, STAGE_EXACT, 63, 0);
+        else sched_begin(s, STAGE_EXACT, 30, BF16 ? 21 : 0);
+        return true;
+    }
+    if (s.stage == STAGE_EXACT) { sched_begin(s, STAGE_INDEX, idx_bits, 0); return true; }
+    return false;
+}
+
+__device__ __forceinline__ unsigned long long exact_key(float a, float s)
+{
+    return (unsigned long long)__double_as_longlong((double)a * (double)s);   // exact: at most 48 significant bits
+}
+
+// Counts one element of a line in the current pass.  t32 = the line's tau32, or 0xffffffff when the line is decided.
+__device__ __forceinline__ void count_element(uint32_t *h, const Line &ln, uint32_t t32, float a, float s, uint32_t idx,
+                                              const Sched &sc, uint32_t idx_top)
+{
+    const uint32_t pk = __float_as_uint(__fmul_rn(a, s));
+    const uint32_t dmask = (1u << sc.bits) - 1u;
+    if (sc.stage == STAGE_ROUNDED) {
+        const uint32_t known = ~0u << (sc.shift + sc.bits);       // shift + bits <= 31: bit 31 is always "known"
+        if (((pk ^ t32) & known) == 0u) atomicAdd(h + hslot((pk >> sc.shift) & dmask), 1u);
+    } else if (pk == t32) {
+        const unsigned long long r = exact_key(a, s) - ln.base;
+        if (sc.stage == STAGE_EXACT) {
+            const unsigned long long known = ~0ull << (sc.shift + sc.bits);   // shift + bits <= 63
+            if (((r ^ ln.tau64) & known) == 0ull) atomicAdd(h + hslot((uint32_t)(r >> sc.shift) & dmask), 1u);
+        } else if (r == ln.tau64) {
+            const uint32_t ik = idx_top - idx;
+            const uint32_t known = ~0u << (sc.shift + sc.bits);   // shift + bits <= 31
+            if (((ik ^ ln.tauidx) & known) == 0u) atomicAdd(h + hslot((ik >> sc.shift) & dmask), 1u);
+        }
+    }
+}
+
+// One warp, one pending line: finds the bin that holds the krem-th largest candidate, appends its digit to the
+// line's threshold and decides the line when the bin holds exactly the candidates still to be taken.
+__device__ __forceinline__ void bucket_step(const uint32_t *h, Line &ln, const Sched &sc, int lane, uint32_t *s_long)
+{
+    const uint32_t *mine_bins = h + lane * 65;        // hslot(lane * 64 + i) = lane * 65 + i
+    uint32_t lane_sum = 0u;
+#pragma unroll 8
+    for (int i = 0; i < 64; ++i) lane_sum += mine_bins[i];
+    uint32_t v = lane_sum;                            // becomes the sum over lanes >= this one
 #pragma unroll
     for (int off = 1; off < 32; off <<= 1) {
         const uint32_t t = __shfl_down_sync(FULL_MASK, v, off);
         if (lane + off < 32) v += t;
     }
-    uint32_t above = v - lane_sum;                  // candidates in higher buckets than this lane's
+    const uint32_t krem = ln.krem;
+    uint32_t above = v - lane_sum;                    // candidates in bins above this lane's
     const bool mine = above < krem && krem <= above + lane_sum;
     uint32_t d = 0u, g = 0u, bc = 0u;
     if (mine) {
-#pragma unroll
-        for (int b = 7; b >= 0; --b) {
-            if (krem <= above + cnt[b]) { d = (uint32_t)(lane * 8 + b); g = above; bc = cnt[b]; break; }
-            above += cnt[b];
+        for (int i = 63; i >= 0; --i) {
+            const uint32_t c = mine_bins[i];
+            if (krem <= above + c) { d = (uint32_t)(lane * 64 + i); g = above; bc = c; break; }
+            above += c;
         }
     }
     const uint32_t who = __ballot_sync(FULL_MASK, mine);
     const int src = who ? __ffs(who) - 1 : 0;
-    digit = __shfl_sync(FULL_MASK, d, src);
-    greater = __shfl_sync(FULL_MASK, g, src);
-    bucket = __shfl_sync(FULL_MASK, bc, src);
-}
-
-// LINE_IS_ROW: the CTA's line is matrix row b.  Otherwise its two lines are the matrix columns 2b, 2b+1 (one 4- or
-// 8-byte load per row fetches both).  Every thread works on all lines of its CTA.
-//
-// Stage A selects on p = fl32(|w| * scale) (rounding is monotone, so p decides every pair whose rounded products
-// differ): four 8-bit passes give the threshold tau32.  If exactly the needed number of products equal tau32, all of
-// them stay and the line is done.  Otherwise stage B repeats the selection among those equal products with the exact
-// double products as keys (eight passes), and the emit pass breaks remaining exact ties towards the lower index.
-template <bool BF16, bool LINE_IS_ROW>
-__global__ void __launch_bounds__(LINE_IS_ROW ? 256 : 512) select_unstructured_kernel(const SelectParams p)
-{
-    constexpr int U_THREADS = LINE_IS_ROW ? 256 : 512;   // row lines: 3 CTAs per SM; column lines: one CTA (2 lines) per SM
-    constexpr int U_WARPS = U_THREADS / 32;
-    using elem_t = typename std::conditional<BF16, uint16_t, uint32_t>::type;
-    constexpr int U_LINES = LINE_IS_ROW ? 1 : 2;
-    extern __shared__ __align__(16) unsigned char u_smem[];
-    elem_t *line_mem = reinterpret_cast<elem_t *>(u_smem);                       // [U_LINES][lpad]
-    uint32_t *hist = reinterpret_cast<uint32_t *>(u_smem + (size_t)U_LINES * p.lpad * sizeof(elem_t));   // [U_LINES][U_WARPS][256]
-    __shared__ LineState st[U_LINES];
-    __shared__ uint32_t s_warp_tot[U_WARPS];
-    __shared__ uint32_t s_any_exact;
-
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int64_t line0 = (int64_t)blockIdx.x * U_LINES;
-    const int nl = (int)((p.nlines - line0) < U_LINES ? (p.nlines - line0) : U_LINES);
-    const int64_t nchunks = p.lpad >> 3;
-    constexpr int TPL = U_THREADS;                                              // threads per line
-    constexpr int my_first = 0;
-    constexpr int my_count = U_LINES;
-    const int tau = tid;
-    const int64_t nbatches = (nchunks + TPL - 1) / TPL;
-
-    // ---------------------------------------------------------------- phase 0: lines -> shared memory
-    if constexpr (LINE_IS_ROW) {
-        // 16-byte loads: rows are 16-byte aligned and padded to whole vectors by the ld rule; elements past L
-        // that a vector drags in are never used (every consumer checks the index against L)
-        const uint4 *src = reinterpret_cast<const uint4 *>(static_cast<const elem_t *>(p.W) + line0 * p.ld);
-        uint4 *dst = reinterpret_cast<uint4 *>(line_mem);
-        constexpr int EPV = 16 / sizeof(elem_t);
-        const int64_t nvec = (p.L + EPV - 1) / EPV;
-        for (int64_t v = tid; v < (int64_t)(p.lpad / EPV); v += U_THREADS) dst[v] = v < nvec ? __ldcs(src + v) : make_uint4(0u, 0u, 0u, 0u);
-    } else {
-        const elem_t *src = static_cast<const elem_t *>(p.W) + line0;            // column line0 of row r at src[r * ld]
-        for (int64_t r = tid; r < p.lpad; r += U_THREADS) {
-#pragma unroll
-            for (int ln = 0; ln < U_LINES; ++ln)
-                line_mem[ln * p.lpad + r] = (r < p.L && ln < nl) ? src[r * p.ld + ln] : (elem_t)0;
+    const uint32_t digit = __shfl_sync(FULL_MASK, d, src);
+    const uint32_t greater = __shfl_sync(FULL_MASK, g, src);
+    const uint32_t bucket = __shfl_sync(FULL_MASK, bc, src);
+    if (lane == 0) {
+        const uint32_t left = krem - greater;
+        ln.krem = left;
+        if (sc.stage == STAGE_ROUNDED) ln.tau32 |= digit << sc.shift;
+        else if (sc.stage == STAGE_EXACT) ln.tau64 |= (unsigned long long)digit << sc.shift;
+        else ln.tauidx |= digit << sc.shift;
+        if (bucket == left) {
+            ln.pending = 0u;
+            ln.done_stage = (uint32_t)sc.stage;
+        } else if (sc.stage == STAGE_ROUNDED && sc.shift == 0) {
+            // the rounded products tie across the cut: the exact part of the key goes on
+            const uint32_t t = ln.tau32;
+            if (t >= 0x00800000u) {
+                ln.base = (unsigned long long)__double_as_longlong((double)__uint_as_float(t)) - (1ull << 28);
+            } else {
+                ln.base = 0ull;
+                atomicOr(s_long, 1u);
+            }
         }
     }
-    if (tid < U_LINES) { st[tid].tau64 = 0ull; st[tid].tau32 = 0u; st[tid].krem = p.k; st[tid].neq = 0u; st[tid].exact = 0u; }
-    if (tid == 0) s_any_exact = 0u;
-    __syncthreads();
+}
 
-    // the 8 rounded products of chunk q of line ln (0 for positions past the line's end)
-    auto products = [&](int ln, int64_t q, float line_scale, float (&pf)[8]) {
-        float sc[8];
+// What the emit step needs of a decided line.
+__device__ __forceinline__ LineResult line_result(const Line &ln, uint32_t idx_top)
+{
+    LineResult r;
+    r.tau32 = ln.tau32;
+    r.exact = ln.done_stage != STAGE_ROUNDED ? 1u : 0u;
+    r.tau64 = ln.base + ln.tau64;
+    r.cut = ln.done_stage == STAGE_INDEX ? (long long)(idx_top - ln.tauidx) : 0x7fffffffffffffffll;
+    return r;
+}
+
+__device__ __forceinline__ void line_init(Line &ln, uint32_t k)
+{
+    ln.tau64 = 0ull; ln.base = 0ull; ln.tau32 = 0u; ln.tauidx = 0u; ln.krem = k; ln.pending = 1u;
+    ln.done_stage = STAGE_ROUNDED; ln.pad_ = 0u;
+}
+
+template <bool BF16>
+__device__ __forceinline__ void chunk_from(Chunk<BF16> &c, const uint4 *src)    // shared or global, 16-byte aligned
+{
+    const uint4 a = src[0];
+    c.w[0] = a.x; c.w[1] = a.y; c.w[2] = a.z; c.w[3] = a.w;
+    if constexpr (!BF16) {
+        const uint4 b = src[1];
+        c.w[4] = b.x; c.w[5] = b.y; c.w[6] = b.z; c.w[7] = b.w;
+    }
+}
+
+// keep bit of one element under a decided line's rule
+__device__ __forceinline__ bool keeps(const LineResult &res, float a, float s, long long idx)
+{
+    const uint32_t key = __float_as_uint(__fmul_rn(a, s));
+    if (key != res.tau32) return key > res.tau32;
+    if (!res.exact) return true;
+    const unsigned long long k64 = exact_key(a, s);
+    return k64 > res.tau64 || (k64 == res.tau64 && idx <= res.cut);
+}
+
+// ---------------------------------------------------------------- lines that are matrix rows
+// One CTA per row: the row is read once with 16-byte loads into shared memory, selected there and written out
+// (mask bytes and the pruned copy) by the same CTA.
+constexpr int ROW_THREADS = 256;
+
+template <bool BF16>
+__global__ void __launch_bounds__(ROW_THREADS) select_rows_kernel(const SelectParams p)
+{
+    using elem_t = typename std::conditional<BF16, uint16_t, uint32_t>::type;
+    constexpr int EPV = 16 / sizeof(elem_t);                     // elements per 16-byte vector
+    extern __shared__ __align__(16) unsigned char u_smem[];
+    elem_t *line_mem = reinterpret_cast<elem_t *>(u_smem);       // [lpad]
+    uint32_t *hist = reinterpret_cast<uint32_t *>(u_smem + (size_t)p.lpad * sizeof(elem_t));   // [HWORDS]
+    __shared__ Line st;
+    __shared__ uint32_t s_long;
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int64_t row = blockIdx.x;
+    const int64_t nchunks = p.lpad >> 3;
+    const uint32_t idx_top = (uint32_t)((1ull << p.idx_bits) - 1ull);
+
+    {   // rows are 16-byte aligned and padded to whole vectors by the ld rule; what a vector drags in past L is
+        // never used (every consumer checks the index against L)
+        const uint4 *src = reinterpret_cast<const uint4 *>(static_cast<const elem_t *>(p.W) + row * p.ld);
+        uint4 *dst = reinterpret_cast<uint4 *>(line_mem);
+        const int64_t nvec = (p.L + EPV - 1) / EPV;
+        for (int64_t v = tid; v < (int64_t)(p.lpad / EPV); v += ROW_THREADS)
+            dst[v] = v < nvec ? __ldcs(src + v) : make_uint4(0u, 0u, 0u, 0u);
+    }
+    if (tid == 0) { line_init(st, p.k); s_long = 0u; }
+    const float line_scale = p.scale_along_line ? 0.0f : p.scale[row];
+
+    // the 8 magnitudes and scales of chunk q
+    auto fetch = [&](int64_t q, float (&a)[8], float (&sc)[8]) {
+        Chunk<BF16> ch;
+        chunk_from<BF16>(ch, reinterpret_cast<const uint4 *>(line_mem + q * 8));
+#pragma unroll
+        for (int j = 0; j < 8; ++j) a[j] = chunk_abs<BF16>(ch, j);
         if (p.scale_along_line) {
             const float4 s0 = __ldg(reinterpret_cast<const float4 *>(p.scale + q * 8));
             const float4 s1 = __ldg(reinterpret_cast<const float4 *>(p.scale + q * 8) + 1);   // the vector is padded to 8
@@ -177,233 +277,120 @@ __global__ void __launch_bounds__(LINE_IS_ROW ? 256 : 512) select_unstructured_k
 #pragma unroll
             for (int j = 0; j < 8; ++j) sc[j] = line_scale;
         }
-#pragma unroll
-        for (int j = 0; j < 8; ++j) pf[j] = __fmul_rn(abs_of<BF16>(line_mem[ln * p.lpad + q * 8 + j]), sc[j]);
     };
 
-    // ---------------------------------------------------------------- stage A: radix select on the rounded products
-    for (int shift = 24; shift >= 0; shift -= 8) {
-        for (int i = tid; i < U_LINES * U_WARPS * 256; i += U_THREADS) hist[i] = 0u;
+    Sched sc;
+    sched_begin(sc, STAGE_ROUNDED, 31, 0);
+    for (;;) {
+        for (int i = tid; i < HWORDS; i += ROW_THREADS) hist[i] = 0u;
         __syncthreads();
-        const uint32_t known = shift == 24 ? 0u : (~0u << (shift + 8));
-        for (int m = 0; m < my_count; ++m) {
-            const int ln = my_first + m;
-            const bool live = ln < nl;
-            const uint32_t prefix = live ? st[ln].tau32 : 0u;
-            const float line_scale = (!live || p.scale_along_line) ? 0.0f : p.scale[line0 + ln];
-            uint32_t *h = hist + ((live ? ln : 0) * U_WARPS + warp) * 256;
-            for (int64_t bt = 0; bt < nbatches; ++bt) {          // same trip count for every lane (warp-wide votes inside)
-                const int64_t q = bt * TPL + tau;
-                const bool have = live && q < nchunks;
-                float pf[8];
-                if (have) products(ln, q, line_scale, pf);
-                if (shift == 24) {
-                    // first pass: every element is a candidate and the top byte (sign and high exponent bits) is the
-                    // same for most of a line, so whole chunks are counted at once and merged across the warp
-                    uint32_t d0 = 0u;
-                    bool same = have && (q * 8 + 7 < p.L);
-                    if (have) {
-                        d0 = __float_as_uint(pf[0]) >> 24;
+        const uint32_t t32 = st.tau32;
+        for (int64_t q = tid; q < nchunks; q += ROW_THREADS) {
+            float a[8], s[8];
+            fetch(q, a, s);
 #pragma unroll
-                        for (int j = 1; j < 8; ++j) same = same && ((__float_as_uint(pf[j]) >> 24) == d0);
-                    }
-                    if (__all_sync(FULL_MASK, same || !have)) {
-                        const unsigned act = __ballot_sync(FULL_MASK, have);
-                        if (have) {
-                            const unsigned peers = __match_any_sync(act, d0);
-                            if (lane == __ffs(peers) - 1) atomicAdd(h + d0, 8u * (uint32_t)__popc(peers));
-                        }
-                    } else {
-#pragma unroll
-                        for (int j = 0; j < 8; ++j)
-                            hist_add(h, have ? (__float_as_uint(pf[j]) >> 24) : 0u, have && (q * 8 + j < p.L));
-                    }
-                } else if (have) {
-                    // later passes: few candidates, spread over many bins: plain atomics
-#pragma unroll
-                    for (int j = 0; j < 8; ++j) {
-                        const uint32_t key = __float_as_uint(pf[j]);
-                        if ((q * 8 + j < p.L) && (((key ^ prefix) & known) == 0u)) atomicAdd(h + ((key >> shift) & 0xffu), 1u);
-                    }
-                }
-            }
+            for (int j = 0; j < 8; ++j)
+                if (q * 8 + j < p.L) count_element(hist, st, t32, a[j], s[j], (uint32_t)(q * 8 + j), sc, idx_top);
         }
         __syncthreads();
-        if (warp < nl) {
-            uint32_t digit, greater, bucket;
-            find_bucket(hist + warp * U_WARPS * 256, U_WARPS, st[warp].krem, lane, digit, greater, bucket);
-            if (lane == 0) {
-                st[warp].tau32 |= digit << shift;
-                st[warp].krem -= greater;
-                if (shift == 0) {
-                    st[warp].neq = bucket;
-                    if (bucket != st[warp].krem) { st[warp].exact = 1u; s_any_exact = 1u; }
-                }
-            }
-        }
+        if (warp == 0) bucket_step(hist, st, sc, lane, &s_long);
         __syncthreads();
+        if (!st.pending) break;
+        const bool was_rounded = sc.stage == STAGE_ROUNDED;
+        if (!sched_next<BF16>(sc, s_long != 0u, p.idx_bits)) break;
+        if (was_rounded && s_long && tid == 0) st.base = 0ull;     // read again only after the next barrier
     }
 
-    // ---------------------------------------------------------------- stage B: exact keys among the tied products
-    if (s_any_exact) {
-        for (int shift = 56; shift >= 0; shift -= 8) {
-            for (int i = tid; i < U_LINES * U_WARPS * 256; i += U_THREADS) hist[i] = 0u;
-            __syncthreads();
-            const unsigned long long known = shift == 56 ? 0ull : (~0ull << (shift + 8));
-            for (int m = 0; m < my_count; ++m) {
-                const int ln = my_first + m;
-                const bool live = ln < nl && st[ln < nl ? ln : 0].exact;
-                const uint32_t t32 = live ? st[ln].tau32 : 0u;
-                const unsigned long long prefix = live ? st[ln].tau64 : 0ull;
-                const float line_scale = (!live || p.scale_along_line) ? 0.0f : p.scale[line0 + ln];
-                uint32_t *h = hist + ((live ? ln : 0) * U_WARPS + warp) * 256;
-                for (int64_t bt = 0; bt < nbatches; ++bt) {
-                    const int64_t q = bt * TPL + tau;
-                    const bool have = live && q < nchunks;
-                    float pf[8];
-                    if (have) products(ln, q, line_scale, pf);
+    // ---------------------------------------------------------------- emit in place
+    const LineResult res = line_result(st, idx_top);
+    for (int64_t q = tid; q < nchunks; q += ROW_THREADS) {
+        float a[8], s[8];
+        fetch(q, a, s);
+        uint32_t keep = 0u;
 #pragma unroll
-                    for (int j = 0; j < 8; ++j) {
-                        bool cand = have && (q * 8 + j < p.L) && __float_as_uint(pf[j]) == t32;
-                        unsigned long long key = 0ull;
-                        if (cand) {
-                            const float sc = p.scale_along_line ? __ldg(p.scale + q * 8 + j) : line_scale;
-                            key = (unsigned long long)__double_as_longlong((double)abs_of<BF16>(line_mem[ln * p.lpad + q * 8 + j]) * (double)sc);
-                            cand = ((key ^ prefix) & known) == 0ull;
-                        }
-                        if (cand) atomicAdd(h + (uint32_t)((key >> shift) & 0xffull), 1u);
-                    }
-                }
-            }
-            __syncthreads();
-            if (warp < nl && st[warp].exact) {
-                uint32_t digit, greater, bucket;
-                find_bucket(hist + warp * U_WARPS * 256, U_WARPS, st[warp].krem, lane, digit, greater, bucket);
-                if (lane == 0) {
-                    st[warp].tau64 |= (unsigned long long)digit << shift;
-                    st[warp].krem -= greater;
-                }
-            }
-            __syncthreads();
+        for (int j = 0; j < 8; ++j)
+            if (q * 8 + j < p.L && keeps(res, a[j], s[j], q * 8 + j)) keep |= 1u << j;
+        const int64_t e0 = q * 8;
+        const int64_t left = p.L - e0;
+        const int nvalid = left >= 8 ? 8 : (int)left;
+        if (p.mask) reinterpret_cast<uint8_t *>(p.mask + row * p.wpr)[q] = (uint8_t)keep;   // byte q = columns 8q..8q+7
+        if (p.Wp) {
+            Chunk<BF16> ch;
+            chunk_from<BF16>(ch, reinterpret_cast<const uint4 *>(line_mem + e0));
+            chunk_apply_mask<BF16>(ch, keep);
+            chunk_store<BF16>(ch, p.Wp, row * p.ld + e0, nvalid);
         }
     }
+}
 
-    if constexpr (!LINE_IS_ROW) {
-        // column lines: publish the thresholds; select_emit_cols_kernel writes the outputs with coalesced rows.
-        // The loop below then only locates the cut among exact ties (skipped when no line of the CTA has any).
-        if (tid < nl) {
-            LineResult r;
-            r.tau64 = st[tid].tau64; r.cut = -1; r.tau32 = st[tid].tau32; r.exact = st[tid].exact;
-            p.results[line0 + tid] = r;
+// ---------------------------------------------------------------- lines that are matrix columns
+// One CTA per strip of 8 adjacent columns (16 bytes of every row for bf16, 32 for f32).  The strip is not cached:
+// every pass reads it again with one vector load per row and thread, and one CTA per SM keeps the strips in
+// flight (148 x 0.46 MB on the 70B-shaped matrix) inside L2, so only the first pass reads DRAM.  The kernel
+// publishes (tau32, exact, tau64, cut) per column; select_emit_cols_kernel applies them with coalesced rows.
+constexpr int COL_THREADS = 1024;
+constexpr int COL_LINES = 8;
+
+template <bool BF16>
+__global__ void __launch_bounds__(COL_THREADS, 1) select_cols_kernel(const SelectParams p)
+{
+    using elem_t = typename std::conditional<BF16, uint16_t, uint32_t>::type;
+    extern __shared__ __align__(16) unsigned char u_smem[];
+    uint32_t *hist = reinterpret_cast<uint32_t *>(u_smem);       // [COL_LINES][HWORDS]
+    __shared__ Line st[COL_LINES];
+    __shared__ uint32_t s_long;
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int64_t c0 = (int64_t)blockIdx.x * COL_LINES;
+    const int nl = (int)((p.cols - c0) < COL_LINES ? (p.cols - c0) : COL_LINES);
+    const uint32_t idx_top = (uint32_t)((1ull << p.idx_bits) - 1ull);
+    const elem_t *strip = static_cast<const elem_t *>(p.W) + c0;
+
+    if (tid < COL_LINES) line_init(st[tid], p.k);
+    if (tid == 0) s_long = 0u;
+    float col_scale[COL_LINES];
+#pragma unroll
+    for (int j = 0; j < COL_LINES; ++j) col_scale[j] = (!p.scale_along_line && j < nl) ? p.scale[c0 + j] : 0.0f;
+
+    Sched sc;
+    sched_begin(sc, STAGE_ROUNDED, 31, 0);
+    for (;;) {
+        for (int i = tid; i < COL_LINES * HWORDS; i += COL_THREADS) hist[i] = 0u;
+        __syncthreads();
+        uint32_t t32[COL_LINES];
+#pragma unroll
+        for (int j = 0; j < COL_LINES; ++j) t32[j] = (j < nl && st[j].pending) ? st[j].tau32 : 0xffffffffu;
+        for (int64_t r = tid; r < p.L; r += COL_THREADS) {
+            // the row pitch is a multiple of 16 bytes and c0 of 8 elements: aligned vectors inside the row's pitch
+            // (an f32 row is padded to 4 elements only: its second vector is read when it holds a real column)
+            Chunk<BF16> ch;
+            const uint4 *src = reinterpret_cast<const uint4 *>(strip + r * p.ld);
+            const uint4 v0 = __ldg(src);
+            ch.w[0] = v0.x; ch.w[1] = v0.y; ch.w[2] = v0.z; ch.w[3] = v0.w;
+            if constexpr (!BF16) {
+                uint4 v1 = make_uint4(0u, 0u, 0u, 0u);
+                if (nl > 4) v1 = __ldg(src + 1);
+                ch.w[4] = v1.x; ch.w[5] = v1.y; ch.w[6] = v1.z; ch.w[7] = v1.w;
+            }
+            const float row_scale = p.scale_along_line ? __ldg(p.scale + r) : 0.0f;
+#pragma unroll
+            for (int j = 0; j < COL_LINES; ++j) {
+                const float s = p.scale_along_line ? row_scale : col_scale[j];
+                count_element(hist + j * HWORDS, st[j], t32[j], chunk_abs<BF16>(ch, j), s, (uint32_t)r, sc, idx_top);
+            }
         }
         __syncthreads();
-        if (!s_any_exact) return;
+        if (warp < nl && st[warp].pending) bucket_step(hist + warp * HWORDS, st[warp], sc, lane, &s_long);
+        __syncthreads();
+        uint32_t pending = 0u;
+#pragma unroll
+        for (int j = 0; j < COL_LINES; ++j) pending |= (j < nl) ? st[j].pending : 0u;
+        if (!pending) break;
+        const bool was_rounded = sc.stage == STAGE_ROUNDED;
+        if (!sched_next<BF16>(sc, s_long != 0u, p.idx_bits)) break;
+        if (was_rounded && s_long && tid < COL_LINES) st[tid].base = 0ull;   // read again only after the next barrier
     }
-    // ---------------------------------------------------------------- emit in index order
-    for (int m = 0; m < my_count; ++m) {
-        const int ln = my_first + m;
-        const bool live = ln < nl;
-        const LineState ls = st[live ? ln : 0];
-        const float line_scale = (!live || p.scale_along_line) ? 0.0f : p.scale[line0 + ln];
-        uint32_t base = 0u;                                  // exact ties seen before this batch
-        for (int64_t bt = 0; bt < nbatches; ++bt) {
-            const int64_t q = bt * TPL + tau;
-            const bool have = live && q < nchunks;
-            uint32_t keep = 0u, eq = 0u;
-            if (have) {
-                float pf[8];
-                products(ln, q, line_scale, pf);
-#pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    if (q * 8 + j < p.L) {
-                        const uint32_t key = __float_as_uint(pf[j]);
-                        if (key > ls.tau32) {
-                            keep |= 1u << j;
-                        } else if (key == ls.tau32) {
-                            if (!ls.exact) {
-                                keep |= 1u << j;             // all products equal to the threshold stay
-                            } else {
-                                const float sc = p.scale_along_line ? __ldg(p.scale + q * 8 + j) : line_scale;
-                                const unsigned long long k64 = (unsigned long long)__double_as_longlong(
-                                    (double)abs_of<BF16>(line_mem[ln * p.lpad + q * 8 + j]) * (double)sc);
-                                if (k64 > ls.tau64) keep |= 1u << j;
-                                else if (k64 == ls.tau64) eq |= 1u << j;
-                            }
-                        }
-                    }
-                }
-            }
-            if (s_any_exact) {
-                // exclusive prefix of the exact-tie counts over the line's threads, in thread (= index) order
-                const uint32_t mycnt = __popc(eq);
-                uint32_t incl = mycnt;
-#pragma unroll
-                for (int off = 1; off < 32; off <<= 1) {
-                    const uint32_t t = __shfl_up_sync(FULL_MASK, incl, off);
-                    if (lane >= off) incl += t;
-                }
-                if (lane == 31) s_warp_tot[warp] = incl;
-                __syncthreads();
-                const int w_first = 0;
-                uint32_t before = base, batch_total = 0u;
-                for (int w = 0; w < TPL / 32; ++w) {
-                    const uint32_t t = s_warp_tot[w_first + w];
-                    if (w_first + w < warp) before += t;
-                    batch_total += t;
-                }
-                __syncthreads();
-                uint32_t rank = before + incl - mycnt;       // exact ties with a lower index than this thread's first
-#pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    if ((eq >> j) & 1u) {
-                        if (rank < ls.krem) keep |= 1u << j;
-                        if constexpr (!LINE_IS_ROW) {
-                            if (ls.exact && rank + 1 == ls.krem) p.results[line0 + ln].cut = q * 8 + j;   // last exact tie that stays
-                        }
-                        ++rank;
-                    }
-                }
-                base += batch_total;
-            }
-
-            if (have) {
-                const int64_t e0 = q * 8;
-                const int64_t left = p.L - e0;
-                const int nvalid = left >= 8 ? 8 : (int)left;
-                if constexpr (LINE_IS_ROW) {
-                    const int64_t r = line0 + ln;
-                    if (p.mask) {
-                        uint8_t *mrow = reinterpret_cast<uint8_t *>(p.mask + r * p.wpr);
-                        mrow[q] = (uint8_t)keep;             // byte q = columns 8q..8q+7 (little endian words)
-                    }
-                    if (p.Wp) {
-                        elem_t *dst = static_cast<elem_t *>(p.Wp) + r * p.ld + e0;
-                        const elem_t *srcl = line_mem + ln * p.lpad + e0;
-                        if (nvalid == 8) {      // whole chunk: 16-byte stores (rows are 16-byte aligned by the ld rule)
-                            constexpr int EPV = 16 / sizeof(elem_t);     // elements per vector
-#pragma unroll
-                            for (int vsel = 0; vsel < 8 / EPV; ++vsel) {
-                                uint4 x = reinterpret_cast<const uint4 *>(srcl)[vsel];
-                                uint32_t *xw = reinterpret_cast<uint32_t *>(&x);
-#pragma unroll
-                                for (int wi = 0; wi < 4; ++wi) {
-                                    if constexpr (BF16) {
-                                        const uint32_t mm = (keep >> (2 * wi)) & 3u;
-                                        xw[wi] &= ((mm & 1u) ? 0x0000ffffu : 0u) | ((mm & 2u) ? 0xffff0000u : 0u);
-                                    } else {
-                                        xw[wi] = ((keep >> (vsel * 4 + wi)) & 1u) ? xw[wi] : 0u;
-                                    }
-                                }
-                                reinterpret_cast<uint4 *>(dst)[vsel] = x;
-                            }
-                        } else {
-                            for (int j = 0; j < nvalid; ++j) dst[j] = ((keep >> j) & 1u) ? srcl[j] : (elem_t)0;
-                        }
-                    }
-                }
-            }
-        }
-    }
+    if (tid < nl) p.results[c0 + tid] = line_result(st[tid], idx_top);
 }
 
 // ---------------------------------------------------------------- column lines: streaming emit
@@ -483,22 +470,30 @@ __global__ void __launch_bounds__(256) select_emit_cols_kernel(const EmitParams 
 
 int device_sm_count();   // dass_abi.cu
 
-size_t select_smem_bytes(int64_t L, bool bf16, bool line_is_row)
+// Dynamic shared memory of the row-line kernel: the cached line and one histogram.
+size_t select_row_smem_bytes(int64_t L, bool bf16)
 {
     const int64_t lpad = (L + 7) / 8 * 8;
-    const size_t lines = line_is_row ? 1 : 2;
-    const size_t warps = line_is_row ? 8 : 16;
-    return lines * lpad * (bf16 ? 2 : 4) + lines * warps * 256 * sizeof(uint32_t);
+    return (size_t)lpad * (bf16 ? 2 : 4) + (size_t)HWORDS * sizeof(uint32_t);
 }
 
-template <bool BF16, bool ROW>
-static cudaError_t launch_select(const SelectParams &p, size_t smem, cudaStream_t st)
+template <bool BF16>
+static cudaError_t launch_rows(const SelectParams &p, cudaStream_t st)
 {
-    cudaError_t e = cudaFuncSetAttribute(select_unstructured_kernel<BF16, ROW>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    const size_t smem = select_row_smem_bytes(p.L, BF16);
+    cudaError_t e = cudaFuncSetAttribute(select_rows_kernel<BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    constexpr int lines = ROW ? 1 : 2;
-    const int64_t grid = (p.nlines + lines - 1) / lines;
-    select_unstructured_kernel<BF16, ROW><<<(unsigned)grid, ROW ? 256 : 512, smem, st>>>(p);
+    select_rows_kernel<BF16><<<(unsigned)p.rows, ROW_THREADS, smem, st>>>(p);
+    return cudaGetLastError();
+}
+
+template <bool BF16>
+static cudaError_t launch_cols(const SelectParams &p, cudaStream_t st)
+{
+    const size_t smem = (size_t)COL_LINES * HWORDS * sizeof(uint32_t);
+    cudaError_t e = cudaFuncSetAttribute(select_cols_kernel<BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    select_cols_kernel<BF16><<<(unsigned)((p.cols + COL_LINES - 1) / COL_LINES), COL_THREADS, smem, st>>>(p);
     return cudaGetLastError();
 }
 
@@ -521,19 +516,19 @@ cudaError_t select_unstructured_launch(const void *W, int64_t rows, int64_t cols
     p.rows = rows; p.cols = cols; p.ld = ld;
     p.wpr = (cols + 31) / 32;
     p.L = line_is_row ? cols : rows;
-    p.nlines = line_is_row ? rows : cols;
     p.lpad = (p.L + 7) / 8 * 8;
     p.k = k;
+    p.idx_bits = 1;
+    while (((int64_t)1 << p.idx_bits) < p.L) ++p.idx_bits;
     p.scale_along_line = (line_is_row == norm_cols) ? 1 : 0;   // the norm index runs along the line
-    const size_t smem = select_smem_bytes(p.L, bf16, line_is_row);
     if (line_is_row) {
         if (mask_bits) {   // the kernel writes whole bytes of real columns; the padding of each mask row must read 0
             e = cudaMemsetAsync(mask_bits, 0, (size_t)rows * p.wpr * sizeof(uint32_t), st);
             if (e != cudaSuccess) return e;
         }
-        return bf16 ? launch_select<true, true>(p, smem, st) : launch_select<false, true>(p, smem, st);
+        return bf16 ? launch_rows<true>(p, st) : launch_rows<false>(p, st);
     }
-    e = bf16 ? launch_select<true, false>(p, smem, st) : launch_select<false, false>(p, smem, st);
+    e = bf16 ? launch_cols<true>(p, st) : launch_cols<false>(p, st);
     if (e != cudaSuccess) return e;
     EmitParams q;
     q.W = W; q.Wp = W_pruned; q.mask = mask_bits; q.scale = scale_ws; q.results = results;
@@ -588,7 +583,7 @@ extern "C" dass_status dass_select_unstructured(const void *W, int64_t rows, int
     const bool line_is_row = compare_axis == DASS_AXIS_COLS;         // the index that varies inside a line
     const int64_t L = line_is_row ? cols : rows;
     if (L >= (int64_t)1 << 31) return DASS_ERR_UNSUPPORTED;
-    if (select_smem_bytes(L, bf16, false) > (size_t)220 * 1024) return DASS_ERR_UNSUPPORTED;   // two lines must fit in shared memory
+    if (line_is_row && select_row_smem_bytes(L, bf16) > (size_t)220 * 1024) return DASS_ERR_UNSUPPORTED;   // a row line is cached in shared memory
     const int64_t n_prune = (int64_t)std::floor(sparsity * (double)L);
     const uint32_t k = (uint32_t)(L - n_prune);
     if (select_unstructured_launch(W, rows, cols, ld, bf16, norm, norm_axis == DASS_AXIS_COLS, alpha, k, line_is_row,
