@@ -265,6 +265,8 @@ def run_ours(args):
     # bandwidth-bound kernels are measured at the clocks they get by themselves
     iso = isolated_stage_b(path, pool, alpha, iters=args.iso_iters) if args.iso_iters > 0 else None
 
+    unstructured = unstructured_leg(path, pool, alpha, args.unstructured_iters, peaks) if args.unstructured_iters > 0 else None
+
     # end to end: pinned host inputs -> device -> path -> results back to the host, every step
     e2e = None
     if args.e2e_steps > 0:
@@ -297,6 +299,7 @@ def run_ours(args):
                                          peaks, peak_src, traffic.get("score")),
             "roofline_compress": roofline_b("compress_* kernels x3", cb, comp_ms, iso and iso["compress"],
                                             peaks, peak_src, traffic.get("compress")),
+            "unstructured": unstructured,
             "e2e": e2e, "gpu_launches": KERNEL_LAUNCHES_PER_STEP * args.steps, "clocks": clocks,
             "cpu_baseline": cpu,
         }
@@ -342,6 +345,40 @@ def isolated_stage_b(path, pool, alpha, iters):
         torch.cuda.synchronize()
         out[key] = e0.elapsed_time(e1) / iters
     return out
+
+
+def unstructured_leg(path, pool, alpha, iters, peaks, sparsity=0.5):
+    """The paper's unstructured setting on the same three matrices, timed alone: per input column of gate / up
+    (input-balanced) and per output row of down (output-balanced) the floor(s * L) lowest scores are pruned."""
+    b, cfg = path.b, path.cfg
+
+    def run(ws):
+        Wg, Wu, Wd = ws
+        for name, W, na, a, ca in (("gate", Wg, b.AXIS_ROWS, alpha, b.AXIS_ROWS), ("up", Wu, b.AXIS_ROWS, alpha, b.AXIS_ROWS),
+                                   ("down", Wd, b.AXIS_COLS, 1.0, b.AXIS_COLS)):
+            o = path.out[name]
+            b.select_unstructured(W, path.norm, na, a, sparsity, ca, mask_bits=o["mask"], W_pruned=o["pruned"],
+                                  workspace=path.select_ws[name])
+
+    path.select_ws = {}
+    for name, (rows, cols, na) in {"gate": (cfg.I, cfg.d, b.AXIS_ROWS), "up": (cfg.I, cfg.d, b.AXIS_ROWS),
+                                   "down": (cfg.d, cfg.I, b.AXIS_COLS)}.items():
+        path.select_ws[name] = b.select_workspace(rows, cols, na, path.dev)
+    for i in range(3):
+        run(pool[i % len(pool)])
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(iters):
+        run(pool[i % len(pool)])
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / iters
+    nbytes, _ = stage_b_bytes(cfg, compress=False)
+    gbs = nbytes / (ms * 1e-3) / 1e9
+    return {"sparsity": sparsity, "ms_x3": ms, "achieved": gbs, "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"],
+            "kernels": "select_cols_kernel + select_emit_cols_kernel (gate, up), select_rows_kernel (down)",
+            "algorithmic_bytes_per_step": nbytes, "timed": "alone, back to back, after the step loop"}
 
 
 def run_e2e(cfg, path, X, weights, alpha, steps, world, device):
@@ -478,6 +515,8 @@ def main():
     ap.add_argument("--pool", type=int, default=3, help="distinct synthetic layers cycled through the steps")
     ap.add_argument("--e2e-steps", type=int, default=6)
     ap.add_argument("--iso-iters", type=int, default=20, help="iterations of the stage-(b)-only timing loop (0 = skip)")
+    ap.add_argument("--unstructured-iters", type=int, default=10,
+                    help="iterations of the unstructured-selection timing loop on the same matrices (0 = skip)")
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--ref-tokens", type=int, default=64, help="tokens per step of the reference (oracle) arm")

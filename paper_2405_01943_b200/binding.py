@@ -275,6 +275,16 @@ def compress_nm(W: torch.Tensor, mask_bits: torch.Tensor, n_keep: int, m: int, g
     return values, meta
 
 
+def select_workspace(rows: int, cols: int, norm_axis: int, device="cuda") -> torch.Tensor:
+    """A 16-byte aligned uint8 CUDA tensor of the size dass_select_unstructured needs."""
+    need = ctypes.c_size_t(0)
+    _check(load().dass_select_workspace_bytes(int(rows), int(cols), int(norm_axis), ctypes.byref(need)),
+           "dass_select_workspace_bytes")
+    buf = torch.empty(need.value + 16, dtype=torch.uint8, device=device)
+    off = (-buf.data_ptr()) % 16
+    return buf[off:off + need.value]
+
+
 def select_unstructured(W: torch.Tensor, norm: torch.Tensor, norm_axis: int, alpha: float, sparsity: float,
                         compare_axis: int, mask_bits: Optional[torch.Tensor] = None,
                         W_pruned: Optional[torch.Tensor] = None, want_mask: bool = True, want_pruned: bool = True,
@@ -290,12 +300,8 @@ def select_unstructured(W: torch.Tensor, norm: torch.Tensor, norm_axis: int, alp
         mask_bits = torch.empty((rows, mask_words_per_row(cols)), dtype=torch.int32, device=W.device)
     if W_pruned is None and want_pruned:
         W_pruned = torch.empty_strided((rows, cols), (ld, 1), dtype=W.dtype, device=W.device)
-    need = ctypes.c_size_t(0)
-    _check(load().dass_select_workspace_bytes(rows, cols, int(norm_axis), ctypes.byref(need)), "dass_select_workspace_bytes")
     if workspace is None:
-        workspace = torch.empty(need.value + 16, dtype=torch.uint8, device=W.device)
-        off = (-workspace.data_ptr()) % 16
-        workspace = workspace[off:off + need.value]
+        workspace = select_workspace(rows, cols, norm_axis, W.device)
     code = load().dass_select_unstructured(W.data_ptr(), rows, cols, ld, _dtype_code(W), norm.data_ptr(), int(norm_axis),
                                            float(alpha), float(sparsity), int(compare_axis), _ptr(mask_bits),
                                            _ptr(W_pruned), workspace.data_ptr(), workspace.numel(), _stream(stream))

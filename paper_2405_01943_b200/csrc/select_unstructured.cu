@@ -58,13 +58,11 @@ __global__ void scale_vector_kernel(const float *__restrict__ norm, int64_t n, i
 // part: p = bits of fl32(|w| * scale) (rounding is monotone, so p decides every pair whose rounded products
 // differ), r = bits of the exact double product minus a per-line base (decides pairs whose rounded products are
 // equal), and the index counted down from the top (lower index first).  The k-th largest key of a line is found
-// digit by digit, 11 bits per pass, with one shared-memory histogram of 2048 bins per line.  A line is decided as
+// digit by digit, 11 bits per pass, with a shared-memory histogram of 2048 bins per line.  A line is decided as
 // soon as the bucket that holds the k-th key holds exactly as many candidates as are still to be kept: all of
 // them stay, and "key >= chosen prefix" is the rule; most lines end inside p, after two or three passes.
 constexpr int HB = 11;                          // bits per digit
 constexpr int HBINS = 1 << HB;
-constexpr int HWORDS = HBINS + HBINS / 64;      // a pad word per 64 bins: lanes that scan 64 bins each hit 32 banks
-__device__ __forceinline__ uint32_t hslot(uint32_t bin) { return bin + (bin >> 6); }
 
 enum : int { STAGE_ROUNDED = 0, STAGE_EXACT = 1, STAGE_INDEX = 2 };
 
@@ -119,36 +117,76 @@ __device__ __forceinline__ unsigned long long exact_key(float a, float s)
     return (unsigned long long)__double_as_longlong((double)a * (double)s);   // exact: at most 48 significant bits
 }
 
-// Counts one element of a line in the current pass.  t32 = the line's tau32, or 0xffffffff when the line is decided.
-__device__ __forceinline__ void count_element(uint32_t *h, const Line &ln, uint32_t t32, float a, float s, uint32_t idx,
+__device__ __forceinline__ uint32_t bit_field(uint32_t v, int pos, int len)
+{
+    uint32_t d;
+    asm("bfe.u32 %0, %1, %2, %3;" : "=r"(d) : "r"(v), "r"(pos), "r"(len));
+    return d;
+}
+
+// Element j of a chunk widened to float with its sign (exact for both types).
+template <bool BF16>
+__device__ __forceinline__ float chunk_float(const Chunk<BF16> &c, int j)
+{
+    if constexpr (BF16) return __uint_as_float((j & 1) ? (c.w[j >> 1] & 0xffff0000u) : (c.w[j >> 1] << 16));
+    else return __uint_as_float(c.w[j]);
+}
+
+// How a pass treats an element: COUNT_ALL (first digit of p: every element is a candidate), COUNT_ROUNDED (later
+// digits of p: candidates agree with the digits chosen so far), COUNT_TIED (exact and index parts: candidates
+// have the threshold's rounded product).
+enum : int { COUNT_ALL = 0, COUNT_ROUNDED = 1, COUNT_TIED = 2 };
+
+// Counts one element (signed weight wf, scale s >= 0) of a line in the current pass.  The sign of the product is
+// the weight's and sits in bit 31, which no digit and no comparison below looks at.  t32 = the line's tau32, or
+// 0xffffffff when the line is decided (then only a non-finite product could match; its count is never read).
+template <int MODE>
+__device__ __forceinline__ void count_element(uint32_t *h, const Line &ln, uint32_t t32, float wf, float s, uint32_t idx,
                                               const Sched &sc, uint32_t idx_top)
 {
-    const uint32_t pk = __float_as_uint(__fmul_rn(a, s));
-    const uint32_t dmask = (1u << sc.bits) - 1u;
-    if (sc.stage == STAGE_ROUNDED) {
-        const uint32_t known = ~0u << (sc.shift + sc.bits);       // shift + bits <= 31: bit 31 is always "known"
-        if (((pk ^ t32) & known) == 0u) atomicAdd(h + hslot((pk >> sc.shift) & dmask), 1u);
-    } else if (pk == t32) {
-        const unsigned long long r = exact_key(a, s) - ln.base;
+    const uint32_t pk = __float_as_uint(__fmul_rn(wf, s));
+    if (MODE == COUNT_ALL) {
+        atomicAdd(h + bit_field(pk, sc.shift, sc.bits), 1u);
+    } else if (MODE == COUNT_ROUNDED) {
+        const uint32_t known = (~0u << (sc.shift + sc.bits)) & 0x7fffffffu;      // shift + bits <= 31
+        if (((pk ^ t32) & known) == 0u) atomicAdd(h + bit_field(pk, sc.shift, sc.bits), 1u);
+    } else if (((pk ^ t32) << 1) == 0u) {
+        const unsigned long long r = exact_key(fabsf(wf), s) - ln.base;
         if (sc.stage == STAGE_EXACT) {
-            const unsigned long long known = ~0ull << (sc.shift + sc.bits);   // shift + bits <= 63
-            if (((r ^ ln.tau64) & known) == 0ull) atomicAdd(h + hslot((uint32_t)(r >> sc.shift) & dmask), 1u);
+            const unsigned long long known = ~0ull << (sc.shift + sc.bits);       // shift + bits <= 63
+            if (((r ^ ln.tau64) & known) == 0ull) atomicAdd(h + bit_field((uint32_t)(r >> sc.shift), 0, sc.bits), 1u);
         } else if (r == ln.tau64) {
             const uint32_t ik = idx_top - idx;
-            const uint32_t known = ~0u << (sc.shift + sc.bits);   // shift + bits <= 31
-            if (((ik ^ ln.tauidx) & known) == 0u) atomicAdd(h + hslot((ik >> sc.shift) & dmask), 1u);
+            const uint32_t known = ~0u << (sc.shift + sc.bits);                   // shift + bits <= 31
+            if (((ik ^ ln.tauidx) & known) == 0u) atomicAdd(h + bit_field(ik, sc.shift, sc.bits), 1u);
         }
     }
 }
 
+__device__ __forceinline__ int count_mode(const Sched &sc)
+{
+    if (sc.stage != STAGE_ROUNDED) return COUNT_TIED;
+    return sc.shift + sc.bits == 31 ? COUNT_ALL : COUNT_ROUNDED;
+}
+
 // One warp, one pending line: finds the bin that holds the krem-th largest candidate, appends its digit to the
 // line's threshold and decides the line when the bin holds exactly the candidates still to be taken.
-__device__ __forceinline__ void bucket_step(const uint32_t *h, Line &ln, const Sched &sc, int lane, uint32_t *s_long)
+template <int COPIES>
+__device__ __forceinline__ void bucket_step(uint32_t *h, Line &ln, const Sched &sc, int lane, uint32_t *s_long)
 {
-    const uint32_t *mine_bins = h + lane * 65;        // hslot(lane * 64 + i) = lane * 65 + i
+    uint32_t *mine_bins = h + lane * 64;              // this lane's 64 bins (of copy 0)
     uint32_t lane_sum = 0u;
-#pragma unroll 8
-    for (int i = 0; i < 64; ++i) lane_sum += mine_bins[i];
+#pragma unroll 4
+    for (int i = 0; i < 64; ++i) {
+        const int b = (i + lane) & 63;                // rotated start: the 32 lanes hit 32 banks
+        uint32_t c = mine_bins[b];
+        if (COPIES > 1) {                             // fold the copies into copy 0
+#pragma unroll
+            for (int r = 1; r < COPIES; ++r) c += mine_bins[r * HBINS + b];
+            mine_bins[b] = c;
+        }
+        lane_sum += c;
+    }
     uint32_t v = lane_sum;                            // becomes the sum over lanes >= this one
 #pragma unroll
     for (int off = 1; off < 32; off <<= 1) {
@@ -221,13 +259,13 @@ __device__ __forceinline__ void chunk_from(Chunk<BF16> &c, const uint4 *src)    
     }
 }
 
-// keep bit of one element under a decided line's rule
+// keep bit of one element (signed weight a, scale s >= 0) under a decided line's rule
 __device__ __forceinline__ bool keeps(const LineResult &res, float a, float s, long long idx)
 {
-    const uint32_t key = __float_as_uint(__fmul_rn(a, s));
+    const uint32_t key = __float_as_uint(__fmul_rn(a, s)) & 0x7fffffffu;
     if (key != res.tau32) return key > res.tau32;
     if (!res.exact) return true;
-    const unsigned long long k64 = exact_key(a, s);
+    const unsigned long long k64 = exact_key(fabsf(a), s);
     return k64 > res.tau64 || (k64 == res.tau64 && idx <= res.cut);
 }
 
@@ -235,6 +273,7 @@ __device__ __forceinline__ bool keeps(const LineResult &res, float a, float s, l
 // One CTA per row: the row is read once with 16-byte loads into shared memory, selected there and written out
 // (mask bytes and the pruned copy) by the same CTA.
 constexpr int ROW_THREADS = 256;
+constexpr int ROW_COPIES = 1;                   // histogram copies the lanes spread over (2 measured slower: clearing and folding cost more than the conflicts)
 
 template <bool BF16>
 __global__ void __launch_bounds__(ROW_THREADS) select_rows_kernel(const SelectParams p)
@@ -243,7 +282,7 @@ __global__ void __launch_bounds__(ROW_THREADS) select_rows_kernel(const SelectPa
     constexpr int EPV = 16 / sizeof(elem_t);                     // elements per 16-byte vector
     extern __shared__ __align__(16) unsigned char u_smem[];
     elem_t *line_mem = reinterpret_cast<elem_t *>(u_smem);       // [lpad]
-    uint32_t *hist = reinterpret_cast<uint32_t *>(u_smem + (size_t)p.lpad * sizeof(elem_t));   // [HWORDS]
+    uint32_t *hist = reinterpret_cast<uint32_t *>(u_smem + (size_t)p.lpad * sizeof(elem_t));   // [ROW_COPIES][HBINS]
     __shared__ Line st;
     __shared__ uint32_t s_long;
 
@@ -263,12 +302,12 @@ __global__ void __launch_bounds__(ROW_THREADS) select_rows_kernel(const SelectPa
     if (tid == 0) { line_init(st, p.k); s_long = 0u; }
     const float line_scale = p.scale_along_line ? 0.0f : p.scale[row];
 
-    // the 8 magnitudes and scales of chunk q
-    auto fetch = [&](int64_t q, float (&a)[8], float (&sc)[8]) {
+    // the 8 signed weights and scales of chunk q
+    auto fetch = [&](int64_t q, float (&w)[8], float (&sc)[8]) {
         Chunk<BF16> ch;
         chunk_from<BF16>(ch, reinterpret_cast<const uint4 *>(line_mem + q * 8));
 #pragma unroll
-        for (int j = 0; j < 8; ++j) a[j] = chunk_abs<BF16>(ch, j);
+        for (int j = 0; j < 8; ++j) w[j] = chunk_float<BF16>(ch, j);
         if (p.scale_along_line) {
             const float4 s0 = __ldg(reinterpret_cast<const float4 *>(p.scale + q * 8));
             const float4 s1 = __ldg(reinterpret_cast<const float4 *>(p.scale + q * 8) + 1);   // the vector is padded to 8
@@ -278,22 +317,37 @@ __global__ void __launch_bounds__(ROW_THREADS) select_rows_kernel(const SelectPa
             for (int j = 0; j < 8; ++j) sc[j] = line_scale;
         }
     };
+    const int64_t nfull = p.L >> 3;                  // chunks whose 8 elements all exist
+    uint32_t *my_hist = hist + (lane % ROW_COPIES) * HBINS;
+    auto count_pass = [&](auto mode_tag, const Sched &sc, uint32_t t32) {
+        constexpr int MODE = decltype(mode_tag)::value;
+        for (int64_t q = tid; q < nfull; q += ROW_THREADS) {
+            float w[8], s[8];
+            fetch(q, w, s);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) count_element<MODE>(my_hist, st, t32, w[j], s[j], (uint32_t)(q * 8 + j), sc, idx_top);
+        }
+        if (tid == 0 && nfull < nchunks) {           // the ragged last chunk
+            float w[8], s[8];
+            fetch(nfull, w, s);
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+                if (nfull * 8 + j < p.L) count_element<MODE>(my_hist, st, t32, w[j], s[j], (uint32_t)(nfull * 8 + j), sc, idx_top);
+        }
+    };
 
     Sched sc;
     sched_begin(sc, STAGE_ROUNDED, 31, 0);
     for (;;) {
-        for (int i = tid; i < HWORDS; i += ROW_THREADS) hist[i] = 0u;
+        for (int i = tid; i < ROW_COPIES * HBINS; i += ROW_THREADS) hist[i] = 0u;
         __syncthreads();
         const uint32_t t32 = st.tau32;
-        for (int64_t q = tid; q < nchunks; q += ROW_THREADS) {
-            float a[8], s[8];
-            fetch(q, a, s);
-#pragma unroll
-            for (int j = 0; j < 8; ++j)
-                if (q * 8 + j < p.L) count_element(hist, st, t32, a[j], s[j], (uint32_t)(q * 8 + j), sc, idx_top);
-        }
+        const int mode = count_mode(sc);
+        if (mode == COUNT_ALL) count_pass(std::integral_constant<int, COUNT_ALL>{}, sc, t32);
+        else if (mode == COUNT_ROUNDED) count_pass(std::integral_constant<int, COUNT_ROUNDED>{}, sc, t32);
+        else count_pass(std::integral_constant<int, COUNT_TIED>{}, sc, t32);
         __syncthreads();
-        if (warp == 0) bucket_step(hist, st, sc, lane, &s_long);
+        if (warp == 0) bucket_step<ROW_COPIES>(hist, st, sc, lane, &s_long);
         __syncthreads();
         if (!st.pending) break;
         const bool was_rounded = sc.stage == STAGE_ROUNDED;
@@ -330,13 +384,14 @@ __global__ void __launch_bounds__(ROW_THREADS) select_rows_kernel(const SelectPa
 // publishes (tau32, exact, tau64, cut) per column; select_emit_cols_kernel applies them with coalesced rows.
 constexpr int COL_THREADS = 1024;
 constexpr int COL_LINES = 8;
+constexpr int COL_COPIES = 1;                   // histogram copies per column (3 measured slower, as for rows)
 
 template <bool BF16>
 __global__ void __launch_bounds__(COL_THREADS, 1) select_cols_kernel(const SelectParams p)
 {
     using elem_t = typename std::conditional<BF16, uint16_t, uint32_t>::type;
     extern __shared__ __align__(16) unsigned char u_smem[];
-    uint32_t *hist = reinterpret_cast<uint32_t *>(u_smem);       // [COL_LINES][HWORDS]
+    uint32_t *hist = reinterpret_cast<uint32_t *>(u_smem);       // [COL_LINES][COL_COPIES][HBINS]
     __shared__ Line st[COL_LINES];
     __shared__ uint32_t s_long;
 
@@ -352,35 +407,64 @@ __global__ void __launch_bounds__(COL_THREADS, 1) select_cols_kernel(const Selec
 #pragma unroll
     for (int j = 0; j < COL_LINES; ++j) col_scale[j] = (!p.scale_along_line && j < nl) ? p.scale[c0 + j] : 0.0f;
 
+    // One pass over the strip: UNROLL rows per thread are loaded before any is counted, so that several
+    // L2 round trips are in flight per thread.
+    constexpr int UNROLL = BF16 ? 4 : 2;
+    uint32_t *my_hist = hist + (lane % COL_COPIES) * HBINS;
+    auto count_pass = [&](auto mode_tag, const Sched &sc, const uint32_t (&t32)[COL_LINES]) {
+        constexpr int MODE = decltype(mode_tag)::value;
+        for (int64_t r0 = tid; r0 < p.L; r0 += (int64_t)UNROLL * COL_THREADS) {
+            Chunk<BF16> ch[UNROLL];
+            float row_scale[UNROLL];
+#pragma unroll
+            for (int u = 0; u < UNROLL; ++u) {
+                const int64_t r = r0 + (int64_t)u * COL_THREADS;
+                chunk_zero<BF16>(ch[u]);
+                row_scale[u] = 0.0f;
+                if (r < p.L) {
+                    // the row pitch is a multiple of 16 bytes and c0 of 8 elements: aligned vectors inside the row's
+                    // pitch (an f32 row is padded to 4 elements only: its second vector is read when it holds a column)
+                    const uint4 *src = reinterpret_cast<const uint4 *>(strip + r * p.ld);
+                    const uint4 v0 = __ldg(src);
+                    ch[u].w[0] = v0.x; ch[u].w[1] = v0.y; ch[u].w[2] = v0.z; ch[u].w[3] = v0.w;
+                    if constexpr (!BF16) {
+                        if (nl > 4) {
+                            const uint4 v1 = __ldg(src + 1);
+                            ch[u].w[4] = v1.x; ch[u].w[5] = v1.y; ch[u].w[6] = v1.z; ch[u].w[7] = v1.w;
+                        }
+                    }
+                    if (p.scale_along_line) row_scale[u] = __ldg(p.scale + r);
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < UNROLL; ++u) {
+                const int64_t r = r0 + (int64_t)u * COL_THREADS;
+                if (r < p.L) {
+#pragma unroll
+                    for (int j = 0; j < COL_LINES; ++j) {
+                        const float s = p.scale_along_line ? row_scale[u] : col_scale[j];
+                        if (MODE != COUNT_ALL || j < nl)
+                            count_element<MODE>(my_hist + j * (COL_COPIES * HBINS), st[j], t32[j], chunk_float<BF16>(ch[u], j), s, (uint32_t)r, sc, idx_top);
+                    }
+                }
+            }
+        }
+    };
+
     Sched sc;
     sched_begin(sc, STAGE_ROUNDED, 31, 0);
     for (;;) {
-        for (int i = tid; i < COL_LINES * HWORDS; i += COL_THREADS) hist[i] = 0u;
+        for (int i = tid; i < COL_LINES * COL_COPIES * HBINS; i += COL_THREADS) hist[i] = 0u;
         __syncthreads();
         uint32_t t32[COL_LINES];
 #pragma unroll
         for (int j = 0; j < COL_LINES; ++j) t32[j] = (j < nl && st[j].pending) ? st[j].tau32 : 0xffffffffu;
-        for (int64_t r = tid; r < p.L; r += COL_THREADS) {
-            // the row pitch is a multiple of 16 bytes and c0 of 8 elements: aligned vectors inside the row's pitch
-            // (an f32 row is padded to 4 elements only: its second vector is read when it holds a real column)
-            Chunk<BF16> ch;
-            const uint4 *src = reinterpret_cast<const uint4 *>(strip + r * p.ld);
-            const uint4 v0 = __ldg(src);
-            ch.w[0] = v0.x; ch.w[1] = v0.y; ch.w[2] = v0.z; ch.w[3] = v0.w;
-            if constexpr (!BF16) {
-                uint4 v1 = make_uint4(0u, 0u, 0u, 0u);
-                if (nl > 4) v1 = __ldg(src + 1);
-                ch.w[4] = v1.x; ch.w[5] = v1.y; ch.w[6] = v1.z; ch.w[7] = v1.w;
-            }
-            const float row_scale = p.scale_along_line ? __ldg(p.scale + r) : 0.0f;
-#pragma unroll
-            for (int j = 0; j < COL_LINES; ++j) {
-                const float s = p.scale_along_line ? row_scale : col_scale[j];
-                count_element(hist + j * HWORDS, st[j], t32[j], chunk_abs<BF16>(ch, j), s, (uint32_t)r, sc, idx_top);
-            }
-        }
+        const int mode = count_mode(sc);
+        if (mode == COUNT_ALL) count_pass(std::integral_constant<int, COUNT_ALL>{}, sc, t32);
+        else if (mode == COUNT_ROUNDED) count_pass(std::integral_constant<int, COUNT_ROUNDED>{}, sc, t32);
+        else count_pass(std::integral_constant<int, COUNT_TIED>{}, sc, t32);
         __syncthreads();
-        if (warp < nl && st[warp].pending) bucket_step(hist + warp * HWORDS, st[warp], sc, lane, &s_long);
+        if (warp < nl && st[warp].pending) bucket_step<COL_COPIES>(hist + warp * (COL_COPIES * HBINS), st[warp], sc, lane, &s_long);
         __syncthreads();
         uint32_t pending = 0u;
 #pragma unroll
@@ -474,7 +558,7 @@ int device_sm_count();   // dass_abi.cu
 size_t select_row_smem_bytes(int64_t L, bool bf16)
 {
     const int64_t lpad = (L + 7) / 8 * 8;
-    return (size_t)lpad * (bf16 ? 2 : 4) + (size_t)HWORDS * sizeof(uint32_t);
+    return (size_t)lpad * (bf16 ? 2 : 4) + (size_t)ROW_COPIES * HBINS * sizeof(uint32_t);
 }
 
 template <bool BF16>
@@ -490,7 +574,7 @@ static cudaError_t launch_rows(const SelectParams &p, cudaStream_t st)
 template <bool BF16>
 static cudaError_t launch_cols(const SelectParams &p, cudaStream_t st)
 {
-    const size_t smem = (size_t)COL_LINES * HWORDS * sizeof(uint32_t);
+    const size_t smem = (size_t)COL_LINES * COL_COPIES * HBINS * sizeof(uint32_t);
     cudaError_t e = cudaFuncSetAttribute(select_cols_kernel<BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     select_cols_kernel<BF16><<<(unsigned)((p.cols + COL_LINES - 1) / COL_LINES), COL_THREADS, smem, st>>>(p);
