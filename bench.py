@@ -267,6 +267,10 @@ def run_ours(args):
 
     unstructured = unstructured_leg(path, pool, alpha, args.unstructured_iters, peaks) if args.unstructured_iters > 0 else None
 
+    forward = None
+    if args.forward_iters > 0 and cfg.dtype == "bf16":
+        forward = forward_leg(path, X, pool[0], args.forward_tokens, args.forward_iters, peaks)
+
     # end to end: pinned host inputs -> device -> path -> results back to the host, every step
     e2e = None
     if args.e2e_steps > 0:
@@ -299,7 +303,7 @@ def run_ours(args):
                                          peaks, peak_src, traffic.get("score")),
             "roofline_compress": roofline_b("compress_* kernels x3", cb, comp_ms, iso and iso["compress"],
                                             peaks, peak_src, traffic.get("compress")),
-            "unstructured": unstructured,
+            "unstructured": unstructured, "forward": forward,
             "e2e": e2e, "gpu_launches": KERNEL_LAUNCHES_PER_STEP * args.steps, "clocks": clocks,
             "cpu_baseline": cpu,
         }
@@ -379,6 +383,34 @@ def unstructured_leg(path, pool, alpha, iters, peaks, sparsity=0.5):
     return {"sparsity": sparsity, "ms_x3": ms, "achieved": gbs, "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"],
             "kernels": "select_cols_kernel + select_emit_cols_kernel (gate, up), select_rows_kernel (down)",
             "algorithmic_bytes_per_step": nbytes, "timed": "alone, back to back, after the step loop"}
+
+
+def forward_leg(path, X, weights, tokens, iters, peaks):
+    """Forward pass of the layer (Eq. 2 then Eq. 3) with the weights as they are, on a prefix of the calibration
+    tokens, timed alone: two tensor-core launches (GLU projection writing H in bf16, down projection)."""
+    b, cfg = path.b, path.cfg
+    n = min(tokens, cfg.T)
+    Xs = X[:n]
+    Wg, Wu, Wd = weights
+    ws = b.mlp_forward_workspace(b.mlp_forward_workspace_bytes(n, cfg.d, cfg.I, Xs.dtype)[1], path.dev)
+    Z = torch.empty((n, cfg.d), dtype=Xs.dtype, device=path.dev)
+    for _ in range(2):
+        b.mlp_forward(Xs, Wg, Wu, Wd, path.act, Z=Z, workspace=ws)
+    b.calib_status(ws)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(iters):
+        b.mlp_forward(Xs, Wg, Wu, Wd, path.act, Z=Z, workspace=ws)
+    e1.record()
+    torch.cuda.synchronize()
+    b.calib_status(ws)
+    ms = e0.elapsed_time(e1) / iters
+    flops = 6.0 * n * cfg.d * cfg.I
+    tf = flops / (ms * 1e-3) / 1e12
+    return {"tokens": n, "ms": ms, "tokens_per_s": n / (ms * 1e-3), "achieved": tf, "unit": "TFLOP/s",
+            "frac": tf / peaks["bf16_tflops_sustained"], "frac_of_burst_peak": tf / peaks["bf16_tflops"],
+            "kernels": "mlp_forward_tc_kernel<GLU> + mlp_forward_tc_kernel<PLAIN>",
+            "algorithmic_flops": flops, "timed": "alone, back to back, after the step loop"}
 
 
 def run_e2e(cfg, path, X, weights, alpha, steps, world, device):
@@ -517,6 +549,8 @@ def main():
     ap.add_argument("--iso-iters", type=int, default=20, help="iterations of the stage-(b)-only timing loop (0 = skip)")
     ap.add_argument("--unstructured-iters", type=int, default=10,
                     help="iterations of the unstructured-selection timing loop on the same matrices (0 = skip)")
+    ap.add_argument("--forward-iters", type=int, default=5, help="iterations of the forward-pass timing loop (0 = skip)")
+    ap.add_argument("--forward-tokens", type=int, default=32768, help="tokens of the forward-pass timing loop")
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--ref-tokens", type=int, default=64, help="tokens per step of the reference (oracle) arm")
