@@ -59,9 +59,9 @@ def stage_b_bytes(cfg, compress=True):
 
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per launch from one ncu capture of this very
 # command on the default workload; see profiles/.  None where the kernel changed after the capture.
-NCU_DRAM_BYTES = {"llama2_70b": {"calib": 126.73e9 + 24.7e6,                                  # one launch, T = 262144
-                                 "score": (470.3 + 445.1 + 470.3 + 445.5 + 471.0 + 455.8) * 1e6,   # gate + up + down
-                                 "compress": (499.1 + 203.7 + 499.1 + 204.0 + 537.6 + 238.3) * 1e6}}
+NCU_DRAM_BYTES = {"llama2_70b": {"calib": 130.65e9 + 22.2e6,                                  # one launch, T = 262144
+                                 "score": (2 * (470.4 + 444.1) + 471.0 + 455.7) * 1e6,         # gate + up + down
+                                 "compress": (2 * (499.2 + 204.1) + 537.2 + 238.7) * 1e6}}
 
 
 def roofline_b(kernel, algorithmic_bytes, in_step_ms, isolated_ms, peaks, peak_src, traffic):
@@ -545,7 +545,7 @@ def main():
     ap.add_argument("--config", default="llama2_70b", choices=sorted(synth.CONFIGS))
     ap.add_argument("--tokens", type=int, default=0, help="override the number of calibration tokens (debugging)")
     ap.add_argument("--pool", type=int, default=3, help="distinct synthetic layers cycled through the steps")
-    ap.add_argument("--e2e-steps", type=int, default=6)
+    ap.add_argument("--e2e-steps", type=int, default=12)
     ap.add_argument("--iso-iters", type=int, default=20, help="iterations of the stage-(b)-only timing loop (0 = skip)")
     ap.add_argument("--unstructured-iters", type=int, default=10,
                     help="iterations of the unstructured-selection timing loop on the same matrices (0 = skip)")

@@ -108,6 +108,17 @@ def test_forward_of_the_pruned_layer():
     assert 0.05 < rel < 1.0
 
 
+@pytest.mark.parametrize("name,T", [("llama2_70b", 32768), ("gemma_7b", 8192 + 77)])
+def test_forward_full_size_sampled_tokens(name, T):
+    """Full-size layers in the launch configuration the benchmark times (70B shape, 32768 tokens, one pass); the
+    oracle redoes sampled token rows: the first and last lane of both CTAs of a pair, tile borders, the ragged end."""
+    cfg = synth.scaled(synth.CONFIGS[name], T=T)
+    X = synth.make_x(cfg, DEV)
+    Wg, Wu, Wd = synth.make_weights(cfg, DEV)
+    rows = np.array([0, 127, 128, 255, 256, 4095, 4096, T // 2 + 33, T - 257, T - 1])
+    _check_forward(cfg, X, Wg, Wu, Wd, cfg.act, rows=rows)
+
+
 def test_forward_chunked_equals_one_pass():
     cfg = synth.scaled(synth.CONFIGS["llama2_7b"], d=256, I=688, T=1500)
     X = synth.make_x(cfg, DEV)
