@@ -171,13 +171,21 @@ class LayerPath:
                 meta=torch.empty(mshape, dtype=torch.int32, device=device))
         self.ev = {k: [] for k in ("calib", "score", "compress")}
 
-    def step(self, X, Wg, Wu, Wd, alpha, record=False, before_stage_b=None):
+    def step(self, X, Wg, Wu, Wd, alpha, record=False, before_stage_b=None, x_chunks=None):
+        """x_chunks: [(first token, last token + 1, event or None)]: the calibration is then accumulated chunk by
+        chunk (the sums carry over between calls), each call waiting for its chunk's event on the current stream."""
         b, cfg = self.b, self.cfg
         e = [torch.cuda.Event(enable_timing=True) for _ in range(4)] if record else None
         self.sumsq.zero_()
         if record:
             e[0].record()
-        b.calib_accumulate(X, Wg, Wu, self.act, self.sumsq, self.ws)
+        if x_chunks is None:
+            b.calib_accumulate(X, Wg, Wu, self.act, self.sumsq, self.ws)
+        else:
+            for t0, t1, ready in x_chunks:
+                if ready is not None:
+                    torch.cuda.current_stream().wait_event(ready)
+                b.calib_accumulate(X[t0:t1], Wg, Wu, self.act, self.sumsq, self.ws)
         if record:
             e[1].record()
         if before_stage_b is not None:
@@ -428,6 +436,8 @@ def run_e2e(cfg, path, X, weights, alpha, steps, world, device):
     comp = torch.cuda.current_stream()
     copy = torch.cuda.Stream()
 
+    FIRST_CHUNKS = 4          # the very first upload has no step to hide behind: its X goes up in chunks
+
     def run(n):
         uploaded = [torch.cuda.Event() for _ in range(2)]
         computed = [torch.cuda.Event() for _ in range(2)]
@@ -442,13 +452,33 @@ def run_e2e(cfg, path, X, weights, alpha, steps, world, device):
                     dv.copy_(h, non_blocking=True)
                 uploaded[slot].record(copy)
 
+        def upload_first(slot):
+            """Weights first, then X in chunks, an event per chunk: the calibration of chunk c runs while chunk
+            c + 1 is still on its way (the per-neuron sums accumulate across calls)."""
+            chunks = []
+            with torch.cuda.stream(copy):
+                for h, dv in list(zip(host_in, dev_in[slot]))[1:]:
+                    dv.copy_(h, non_blocking=True)
+                T = host_in[0].shape[0]
+                step_t = -(-T // FIRST_CHUNKS)
+                for t0 in range(0, T, step_t):
+                    t1 = min(T, t0 + step_t)
+                    dev_in[slot][0][t0:t1].copy_(host_in[0][t0:t1], non_blocking=True)
+                    ev = torch.cuda.Event()
+                    ev.record(copy)
+                    chunks.append((t0, t1, ev))
+                uploaded[slot].record(copy)
+            return chunks
+
         copy.wait_stream(comp)
-        upload(0)
+        first_chunks = upload_first(0)
         for i in range(n):
             slot = i % 2
-            comp.wait_event(uploaded[slot])
+            if i > 0:
+                comp.wait_event(uploaded[slot])
             wait_dl = (lambda: comp.wait_event(downloaded)) if have_download else None
-            path.step(*dev_in[slot], alpha, before_stage_b=wait_dl)    # outputs are reused: wait for their download
+            path.step(*dev_in[slot], alpha, before_stage_b=wait_dl,             # outputs are reused: wait for their download
+                      x_chunks=first_chunks if i == 0 else None)
             computed[slot].record(comp)
             if i + 1 < n:
                 upload(1 - slot, after=computed[1 - slot] if i >= 1 else None)
@@ -473,7 +503,8 @@ def run_e2e(cfg, path, X, weights, alpha, steps, world, device):
     seconds = max_over_ranks(a.elapsed_time(b) / 1e3, world, device)
     return {"value": aggregate_value(cfg.T, steps, world, seconds), "unit": UNIT, "steps": steps,
             "ms_per_step": seconds * 1e3 / steps, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-            "overlap": "uploads of step i+1 and downloads of step i run on a copy stream beside the kernels"}
+            "overlap": "uploads of step i+1 and downloads of step i run on a copy stream beside the kernels; the first "
+                       "step's X goes up in 4 chunks and is calibrated chunk by chunk"}
 
 
 # --------------------------------------------------------------------------- the oracle legs
