@@ -286,13 +286,9 @@ template <int ACT>
 static cudaError_t launch_tc(const CUtensorMap &mx, const CUtensorMap &mg, const CUtensorMap &mu, const TcParams &p,
                              int grid, cudaStream_t st)
 {
-    static bool configured = false;
-    if (!configured) {
-        const cudaError_t e = cudaFuncSetAttribute(calib_tc_kernel<ACT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                                   (int)TC_SMEM_BYTES);
-        if (e != cudaSuccess) return e;
-        configured = true;
-    }
+    static unsigned long long configured = 0ull;      // per device
+    const cudaError_t ce = ensure_dynamic_smem(calib_tc_kernel<ACT>, (int)TC_SMEM_BYTES, configured);
+    if (ce != cudaSuccess) return ce;
     calib_tc_kernel<ACT><<<grid, TC_THREADS, TC_SMEM_BYTES, st>>>(mx, mg, mu, p);
     return cudaGetLastError();
 }

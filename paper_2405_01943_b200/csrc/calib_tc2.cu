@@ -239,13 +239,9 @@ template <int ACT>
 static cudaError_t launch_tc2(const CUtensorMap &mx, const CUtensorMap &mg, const CUtensorMap &mu, const T2Params &p,
                               int grid, cudaStream_t st)
 {
-    static bool configured = false;
-    if (!configured) {
-        const cudaError_t e = cudaFuncSetAttribute(calib_tc2_kernel<ACT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                                   (int)T2_SMEM_BYTES);
-        if (e != cudaSuccess) return e;
-        configured = true;
-    }
+    static unsigned long long configured = 0ull;      // per device
+    const cudaError_t ce = ensure_dynamic_smem(calib_tc2_kernel<ACT>, (int)T2_SMEM_BYTES, configured);
+    if (ce != cudaSuccess) return ce;
     calib_tc2_kernel<ACT><<<grid, T2_THREADS, T2_SMEM_BYTES, st>>>(mx, mg, mu, p);
     return cudaGetLastError();
 }

@@ -123,6 +123,20 @@ __host__ __device__ constexpr uint32_t idesc_bf16_f32(int m, int n)
     return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
 }
 
+// Raises a kernel's dynamic shared-memory limit once per device (the attribute belongs to the device's copy of
+// the kernel).  `done` holds one bit per device ordinal; ordinals past 63 are configured on every call.
+template <typename Kernel>
+inline cudaError_t ensure_dynamic_smem(Kernel kernel, int bytes, unsigned long long &done)
+{
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 64 && ((done >> dev) & 1ull)) return cudaSuccess;
+    e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    if (e == cudaSuccess && dev < 64) done |= 1ull << dev;
+    return e;
+}
+
 template <int ACT>
 __device__ __forceinline__ float glu_h(float g, float u)
 {
