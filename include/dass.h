@@ -187,8 +187,9 @@ dass_status dass_feature_sumsq(const void *X, int64_t T, int64_t d, int64_t ldx,
  * Score, scale rounding and order are those of dass_score_nm: exact products, higher score first, lower
  * index first.  sparsity in [0, 1).  mask_bits / W_pruned as for dass_score_nm (at least one; mask_bits is
  * written in full, padding bits 0).  workspace: dass_select_workspace_bytes(...) bytes, 16-byte aligned (holds
- * the rounded norm^alpha vector).  A line (in the matrix dtype) must fit twice into shared memory: up to
- * about 50 000 bf16 or 25 000 f32 elements, else DASS_ERR_UNSUPPORTED.
+ * the rounded norm^alpha vector and the per-column thresholds).  A line that is a matrix row is cached in shared
+ * memory: rows of more than about 108 000 bf16 or 54 000 f32 elements are DASS_ERR_UNSUPPORTED; lines that are
+ * matrix columns have no such limit (below 2^31 elements).
  * Errors: NULL / DTYPE / SHAPE (sizes, sparsity outside [0,1)) / ALIGN / UNSUPPORTED / WORKSPACE / CUDA. */
 dass_status dass_select_workspace_bytes(int64_t rows, int64_t cols, dass_axis norm_axis, size_t *bytes /* HOST */);
 dass_status dass_select_unstructured(const void *W, int64_t rows, int64_t cols, int64_t ld, dass_dtype dt,
