@@ -150,56 +150,42 @@ def aggregate_value(tokens_per_step: int, steps: int, world: int, seconds_max: f
 # --------------------------------------------------------------------------- the GPU arm
 
 class LayerPath:
-    """Device buffers and the sequence of C-ABI calls that make one step."""
+    """One step = the library's public per-layer API (paper_2405_01943_b200.layer.LayerPruner: device buffers
+    and the sequence of C-ABI calls), with CUDA events between the stages."""
 
     def __init__(self, cfg, device, binding):
+        from paper_2405_01943_b200.layer import LayerPruner
         self.cfg, self.dev, self.b = cfg, device, binding
-        d, I = cfg.d, cfg.I
-        dt = cfg.torch_dtype
-        self.act = binding.ACT_BY_NAME[cfg.act]
-        self.sumsq = torch.zeros(I, dtype=torch.float64, device=device)
-        self.norm = torch.empty(I, dtype=torch.float32, device=device)
-        self.ws = binding.calib_workspace(cfg.T, d, I, dt, device)
-        self.out = {}
-        for name, (rows, cols, ga) in {"gate": (I, d, binding.AXIS_ROWS), "up": (I, d, binding.AXIS_ROWS),
-                                       "down": (d, I, binding.AXIS_COLS)}.items():
-            vshape, mshape = binding.compress_shapes(rows, cols, cfg.n_keep, cfg.m, ga)
-            self.out[name] = dict(
-                mask=torch.empty((rows, binding.mask_words_per_row(cols)), dtype=torch.int32, device=device),
-                pruned=torch.empty((rows, cols), dtype=dt, device=device),
-                values=torch.empty(vshape, dtype=dt, device=device),
-                meta=torch.empty(mshape, dtype=torch.int32, device=device))
+        self.pruner = LayerPruner(cfg.T, cfg.d, cfg.I, cfg.torch_dtype, act=cfg.act, n_keep=cfg.n_keep, m=cfg.m,
+                                  device=device)
+        self.act = self.pruner.act
+        self.sumsq, self.norm, self.ws, self.out = self.pruner.sumsq, self.pruner.norm, self.pruner.calib_ws, self.pruner.out
         self.ev = {k: [] for k in ("calib", "score", "compress")}
 
     def step(self, X, Wg, Wu, Wd, alpha, record=False, before_stage_b=None, x_chunks=None):
         """x_chunks: [(first token, last token + 1, event or None)]: the calibration is then accumulated chunk by
         chunk (the sums carry over between calls), each call waiting for its chunk's event on the current stream."""
-        b, cfg = self.b, self.cfg
+        pr = self.pruner
         e = [torch.cuda.Event(enable_timing=True) for _ in range(4)] if record else None
-        self.sumsq.zero_()
+        pr.reset()
         if record:
             e[0].record()
         if x_chunks is None:
-            b.calib_accumulate(X, Wg, Wu, self.act, self.sumsq, self.ws)
+            pr.accumulate(X, Wg, Wu)
         else:
             for t0, t1, ready in x_chunks:
                 if ready is not None:
                     torch.cuda.current_stream().wait_event(ready)
-                b.calib_accumulate(X[t0:t1], Wg, Wu, self.act, self.sumsq, self.ws)
+                pr.accumulate(X[t0:t1], Wg, Wu)
         if record:
             e[1].record()
         if before_stage_b is not None:
             before_stage_b()
-        b.norm_finalize(self.sumsq, self.norm)
-        for name, W, na, a, ga in (("gate", Wg, b.AXIS_ROWS, alpha, b.AXIS_ROWS), ("up", Wu, b.AXIS_ROWS, alpha, b.AXIS_ROWS),
-                                   ("down", Wd, b.AXIS_COLS, 1.0, b.AXIS_COLS)):
-            o = self.out[name]
-            b.score_nm(W, self.norm, na, a, cfg.n_keep, cfg.m, ga, mask_bits=o["mask"], W_pruned=o["pruned"])
+        pr.finalize()
+        pr.score_nm(Wg, Wu, Wd, alpha)
         if record:
             e[2].record()
-        for name, W, ga in (("gate", Wg, b.AXIS_ROWS), ("up", Wu, b.AXIS_ROWS), ("down", Wd, b.AXIS_COLS)):
-            o = self.out[name]
-            b.compress_nm(W, o["mask"], cfg.n_keep, cfg.m, ga, values=o["values"], meta=o["meta"])
+        pr.compress_nm(Wg, Wu, Wd)
         if record:
             e[3].record()
             self.ev["calib"].append((e[0], e[1]))
@@ -328,20 +314,11 @@ def run_ours(args):
 
 def isolated_stage_b(path, pool, alpha, iters):
     """Mean ms of the three scoring launches and of the three compression launches, timed alone."""
-    b, cfg = path.b, path.cfg
-
     def score(ws):
-        Wg, Wu, Wd = ws
-        for name, W, na, a, ga in (("gate", Wg, b.AXIS_ROWS, alpha, b.AXIS_ROWS), ("up", Wu, b.AXIS_ROWS, alpha, b.AXIS_ROWS),
-                                   ("down", Wd, b.AXIS_COLS, 1.0, b.AXIS_COLS)):
-            o = path.out[name]
-            b.score_nm(W, path.norm, na, a, cfg.n_keep, cfg.m, ga, mask_bits=o["mask"], W_pruned=o["pruned"])
+        path.pruner.score_nm(*ws, alpha)
 
     def compress(ws):
-        Wg, Wu, Wd = ws
-        for name, W, ga in (("gate", Wg, b.AXIS_ROWS), ("up", Wu, b.AXIS_ROWS), ("down", Wd, b.AXIS_COLS)):
-            o = path.out[name]
-            b.compress_nm(W, o["mask"], cfg.n_keep, cfg.m, ga, values=o["values"], meta=o["meta"])
+        path.pruner.compress_nm(*ws)
 
     out = {}
     time.sleep(0.5)                      # let the clocks recover from the power-capped GEMM
@@ -362,20 +339,11 @@ def isolated_stage_b(path, pool, alpha, iters):
 def unstructured_leg(path, pool, alpha, iters, peaks, sparsity=0.5):
     """The paper's unstructured setting on the same three matrices, timed alone: per input column of gate / up
     (input-balanced) and per output row of down (output-balanced) the floor(s * L) lowest scores are pruned."""
-    b, cfg = path.b, path.cfg
+    cfg = path.cfg
 
     def run(ws):
-        Wg, Wu, Wd = ws
-        for name, W, na, a, ca in (("gate", Wg, b.AXIS_ROWS, alpha, b.AXIS_ROWS), ("up", Wu, b.AXIS_ROWS, alpha, b.AXIS_ROWS),
-                                   ("down", Wd, b.AXIS_COLS, 1.0, b.AXIS_COLS)):
-            o = path.out[name]
-            b.select_unstructured(W, path.norm, na, a, sparsity, ca, mask_bits=o["mask"], W_pruned=o["pruned"],
-                                  workspace=path.select_ws[name])
+        path.pruner.select_unstructured(*ws, sparsity, alpha)
 
-    path.select_ws = {}
-    for name, (rows, cols, na) in {"gate": (cfg.I, cfg.d, b.AXIS_ROWS), "up": (cfg.I, cfg.d, b.AXIS_ROWS),
-                                   "down": (cfg.d, cfg.I, b.AXIS_COLS)}.items():
-        path.select_ws[name] = b.select_workspace(rows, cols, na, path.dev)
     for i in range(3):
         run(pool[i % len(pool)])
     torch.cuda.synchronize()
