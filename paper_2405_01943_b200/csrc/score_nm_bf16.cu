@@ -193,6 +193,45 @@ __device__ __forceinline__ void keep_from_pairs(const uint32_t (&C)[M * (M - 1) 
     }
 }
 
+// Groups of 8: instead of all 28 pairwise comparisons, the rounded products are sorted with a 19-comparator
+// network (min / max pairs) and every element is compared with the n_keep-th largest, t: "p >= t" is the keep
+// rule whenever t is strictly above the next value (monotone rounding then proves the same for the exact
+// products; equal products on one side of the cut need no order).  Shifts "p_q < t" (the sign of p_q - t) into
+// the bit-sliced words D and returns true if the two values at the cut are equal (order not proven).
+__device__ __forceinline__ void cmp_exchange(float &hi, float &lo)
+{
+    const float a = fmaxf(hi, lo), b = fminf(hi, lo);
+    hi = a;
+    lo = b;
+}
+
+__device__ __forceinline__ bool threshold_group8(const float (&pf)[8], int n_keep, uint32_t (&D)[8])
+{
+    float s[8];
+#pragma unroll
+    for (int q = 0; q < 8; ++q) s[q] = pf[q];
+    cmp_exchange(s[0], s[1]); cmp_exchange(s[2], s[3]); cmp_exchange(s[4], s[5]); cmp_exchange(s[6], s[7]);
+    cmp_exchange(s[0], s[2]); cmp_exchange(s[1], s[3]); cmp_exchange(s[4], s[6]); cmp_exchange(s[5], s[7]);
+    cmp_exchange(s[1], s[2]); cmp_exchange(s[5], s[6]); cmp_exchange(s[0], s[4]); cmp_exchange(s[3], s[7]);
+    cmp_exchange(s[1], s[5]); cmp_exchange(s[2], s[6]);
+    cmp_exchange(s[1], s[4]); cmp_exchange(s[3], s[6]);
+    cmp_exchange(s[2], s[4]); cmp_exchange(s[3], s[5]);
+    cmp_exchange(s[3], s[4]);                         // s[0] >= s[1] >= ... >= s[7]
+    float t, next;
+    switch (n_keep) {                                 // n_keep in 1..7, the same for every lane
+    case 1: t = s[0]; next = s[1]; break;
+    case 2: t = s[1]; next = s[2]; break;
+    case 3: t = s[2]; next = s[3]; break;
+    case 4: t = s[3]; next = s[4]; break;
+    case 5: t = s[4]; next = s[5]; break;
+    case 6: t = s[5]; next = s[6]; break;
+    default: t = s[6]; next = s[7]; break;
+    }
+#pragma unroll
+    for (int q = 0; q < 8; ++q) D[q] = __funnelshift_l(__float_as_uint(__fsub_rn(pf[q], t)), D[q], 1);
+    return t == next;
+}
+
 // 16-bit lane masks for the 8 bf16 of a chunk from an 8-bit keep byte, applied in place.
 __device__ __forceinline__ void apply_keep_byte(uint4 &v, uint32_t keep)
 {
@@ -345,19 +384,34 @@ __global__ void __launch_bounds__(F_THREADS, M == 8 ? 2 : F_MIN_BLOCKS) score_ro
             if constexpr (!NORM_COLS) rs[q] = __shfl_sync(FULL_MASK, lane_scale, (int)(r0 & 31) + q);
         }
 
-        uint32_t C[NP];
-#pragma unroll
-        for (int i = 0; i < NP; ++i) C[i] = 0u;
-        bool tie = false;
-#pragma unroll
-        for (int j = 7; j >= 0; --j) {       // column 7 first: after 8 inserts column j sits at bit j
-            float pf[M];
-#pragma unroll
-            for (int q = 0; q < M; ++q) pf[q] = prod_of(word_of(v[q], j >> 1), (j & 1) != 0, NORM_COLS ? sc[j] : rs[q]);
-            tie |= compare_group<M>(pf, C);
-        }
         uint32_t K[M];
-        keep_from_pairs<M>(C, p.n_keep, K);
+        bool tie = false;
+        if constexpr (M == 8) {
+            uint32_t D[M];
+#pragma unroll
+            for (int q = 0; q < M; ++q) D[q] = 0u;
+#pragma unroll
+            for (int j = 7; j >= 0; --j) {   // column 7 first: after 8 inserts column j sits at bit j
+                float pf[M];
+#pragma unroll
+                for (int q = 0; q < M; ++q) pf[q] = prod_of(word_of(v[q], j >> 1), (j & 1) != 0, NORM_COLS ? sc[j] : rs[q]);
+                tie |= threshold_group8(pf, p.n_keep, D);
+            }
+#pragma unroll
+            for (int q = 0; q < M; ++q) K[q] = ~D[q];
+        } else {
+            uint32_t C[NP];
+#pragma unroll
+            for (int i = 0; i < NP; ++i) C[i] = 0u;
+#pragma unroll
+            for (int j = 7; j >= 0; --j) {   // column 7 first: after 8 inserts column j sits at bit j
+                float pf[M];
+#pragma unroll
+                for (int q = 0; q < M; ++q) pf[q] = prod_of(word_of(v[q], j >> 1), (j & 1) != 0, NORM_COLS ? sc[j] : rs[q]);
+                tie |= compare_group<M>(pf, C);
+            }
+            keep_from_pairs<M>(C, p.n_keep, K);
+        }
         if (tie && nvalid > 0) {   // ragged lanes (zero padding ties) also land here; still exact
             TileWords<M> t;
             Scales8 s8;
@@ -451,15 +505,16 @@ __global__ void __launch_bounds__(F_THREADS, M == 8 ? 3 : F_MIN_BLOCKS) score_co
         ++u_pre;
         stage = stage + 1 == STAGES ? 0 : stage + 1;
 
+        // M == 8: C[0][q] collects "p_q < threshold" per row (threshold_group8); else C[g][pair] the pairwise order
         uint32_t C[G][NP];
 #pragma unroll
         for (int g = 0; g < G; ++g)
 #pragma unroll
-            for (int i = 0; i < NP; ++i) C[g][i] = 0u;
+            for (int i = 0; i < (M == 8 ? M : NP); ++i) C[g][i] = 0u;
         bool tie = false;
         float rsv[F_SLAB];
 #pragma unroll
-        for (int i = F_SLAB - 1; i >= 0; --i) {       // row 7 first: after 8 inserts row i sits at bit i
+        for (int i = F_SLAB - 1; i >= 0; --i) {       // last row first: after the inserts row i sits at bit i
             float rs = 0.0f;
             if constexpr (!NORM_COLS) rs = __shfl_sync(FULL_MASK, lane_scale, (int)(r0 & 31) + i);
             rsv[i] = rs;
@@ -471,7 +526,12 @@ __global__ void __launch_bounds__(F_THREADS, M == 8 ? 3 : F_MIN_BLOCKS) score_co
                     const int j = g * M + q;
                     pf[q] = prod_of(word_of(v[i], j >> 1), (j & 1) != 0, NORM_COLS ? sc[j] : rs);
                 }
-                tie |= compare_group<M>(pf, C[g]);
+                if constexpr (M == 8) {
+                    uint32_t (&D)[8] = reinterpret_cast<uint32_t (&)[8]>(C[g]);
+                    tie |= threshold_group8(pf, p.n_keep, D);
+                } else {
+                    tie |= compare_group<M>(pf, C[g]);
+                }
             }
         }
         // Q[h]: byte a = keep bits (bit i = row i) of column 4h + a
@@ -479,7 +539,12 @@ __global__ void __launch_bounds__(F_THREADS, M == 8 ? 3 : F_MIN_BLOCKS) score_co
 #pragma unroll
         for (int g = 0; g < G; ++g) {
             uint32_t K[M];
-            keep_from_pairs<M>(C[g], p.n_keep, K);
+            if constexpr (M == 8) {
+#pragma unroll
+                for (int q = 0; q < M; ++q) K[q] = ~C[g][q];
+            } else {
+                keep_from_pairs<M>(C[g], p.n_keep, K);
+            }
 #pragma unroll
             for (int h = 0; h < M / 4; ++h) {
                 const uint32_t q = (K[4 * h] & 0xffu) | ((K[4 * h + 1] & 0xffu) << 8) | ((K[4 * h + 2] & 0xffu) << 16) |
