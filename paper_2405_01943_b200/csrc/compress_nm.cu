@@ -5,8 +5,8 @@
 // fields are produced in registers and packed into 32-bit words with warp shuffles (groups along the
 // columns: four lanes share a word) or directly per lane (groups along the rows: a lane's 8 columns
 // fill whole words).  Bandwidth-bound: reads W and one mask bit per weight, writes n_keep/m of W plus
-// the fields.  These generic kernels serve fp32 weights and bf16 row groups (4:8 row groups have a kernel of their
-// own below); bf16 column groups take the permute-table kernel of compress_nm_bf16.cu.
+// the fields.  These generic kernels serve fp32 weights and bf16 row groups (2:4 and 4:8 row groups have a kernel
+// of their own below); bf16 column groups take the permute-table kernel of compress_nm_bf16.cu.
 #include "dass_device.cuh"
 
 namespace dass {
@@ -243,13 +243,14 @@ __global__ void __launch_bounds__(C_THREADS) compress_group_rows_kernel(const Co
     }
 }
 
-// ---------------------------------------------------------------- bf16, groups of 8 along the rows, K survivors
-// A lane holds an 8 x 8 tile: 8 rows (one group per column) of its 8 columns, as four words per row, and the 8
-// keep bits of every row.  The survivors of a column keep their row order, so row q goes to output row
-// k = (number of kept rows above q), a 3-bit count kept bit-sliced over the 8 columns.  For every possible
-// (q, k) the byte "kept and count == k" is spread to 16-bit lane masks (one multiply and a sign-replicating
-// byte permute per word pair) and the row is ORed into output k under it: no per-element select chains.
-// The metadata (the 8-bit keep mask of every column) is the 8 x 8 bit transpose of the keep bytes.
+// ---------------------------------------------------------------- bf16, groups along the rows, fast path
+// A lane holds 8 rows of its 8 columns (four words per row) and the 8 keep bits of every row: one group of 8 per
+// column, or two groups of 4.  The survivors of a column keep their row order, so row q of a group goes to output
+// row k = (number of kept rows above q), a small count kept bit-sliced over the 8 columns.  For every possible
+// (q, k) the byte "kept and count == k" is spread to 16-bit lane masks (one multiply and a sign-replicating byte
+// permute per word pair) and the row is ORed into output k under it: no per-element select chains.
+// Metadata: the keep mask of every column is the bit transpose of the keep bytes; the 2:4 nibble
+// pos_lo | pos_hi << 2 is the transpose of the bit-sliced positions sum_q q * [row q goes to output k].
 __device__ __forceinline__ uint32_t prmt_b32(uint32_t a, uint32_t b, uint32_t sel)
 {
     uint32_t d;
@@ -257,10 +258,17 @@ __device__ __forceinline__ uint32_t prmt_b32(uint32_t a, uint32_t b, uint32_t se
     return d;
 }
 
-template <int K>
-__global__ void __launch_bounds__(C_THREADS) compress_rows8_bf16_kernel(const CompressParams p)
+// nibble made of bit j of each of the four bytes of x (byte a -> bit a)
+__device__ __forceinline__ uint32_t gather_bit(uint32_t x, int j)
 {
-    constexpr int M = 8;
+    return (((x >> j) & 0x01010101u) * 0x10204080u) >> 28;
+}
+
+template <int M, int K, bool TWO_FOUR>
+__global__ void __launch_bounds__(C_THREADS) compress_rows_bf16_kernel(const CompressParams p)
+{
+    static_assert((M == 8 && !TWO_FOUR) || (M == 4 && (!TWO_FOUR || K == 2)), "groups of 4 or 8 rows");
+    constexpr int G = 8 / M;         // groups in the 8 rows a lane takes at a time
     const int lane = threadIdx.x & 31;
     const int64_t warp = (int64_t)blockIdx.x * (C_THREADS / 32) + (threadIdx.x >> 5);
     const int64_t nwarps = (int64_t)gridDim.x * (C_THREADS / 32);
@@ -274,64 +282,98 @@ __global__ void __launch_bounds__(C_THREADS) compress_rows8_bf16_kernel(const Co
         const int nvalid = left >= 8 ? 8 : (left > 0 ? (int)left : 0);
         if (nvalid == 0) continue;   // no shuffles in this kernel: lanes are independent
 
-        for (int g = 0; g < C_TILE_ROWS / M; ++g) {
-            const int64_t r0 = rb * C_TILE_ROWS + g * M;
-            if (r0 >= p.rows) break;
-            const int64_t line = r0 / M;
-            Chunk<true> ch[M];
-            uint32_t mb[M];
+        for (int it = 0; it < C_TILE_ROWS / 8; ++it) {
+            const int64_t rbase = rb * C_TILE_ROWS + it * 8;
+            if (rbase >= p.rows) break;
+            Chunk<true> ch[8];
+            uint32_t mb[8];
+            if (M == 8 || rbase + 8 <= p.rows) {     // all 8 rows exist: eight independent loads in flight
 #pragma unroll
-            for (int q = 0; q < M; ++q) {
-                chunk_load<true>(ch[q], p.W, (r0 + q) * p.ld + c0, nvalid);
-                mb[q] = (__ldg(p.mask + (r0 + q) * p.wpr + (c0 >> 5)) >> (8 * (lane & 3))) & 0xffu;
-            }
-            uint32_t out[K][4];
+                for (int q = 0; q < 8; ++q) {
+                    chunk_load<true>(ch[q], p.W, (rbase + q) * p.ld + c0, nvalid);
+                    mb[q] = (__ldg(p.mask + (rbase + q) * p.wpr + (c0 >> 5)) >> (8 * (lane & 3))) & 0xffu;
+                }
+            } else {                                 // rows is a multiple of 4 only: the last group of 4 stands alone
 #pragma unroll
-            for (int k = 0; k < K; ++k)
-#pragma unroll
-                for (int w = 0; w < 4; ++w) out[k][w] = 0u;
-            uint32_t b0 = 0u, b1 = 0u, b2 = 0u;          // bit-sliced count of kept rows above the current one
-#pragma unroll
-            for (int q = 0; q < M; ++q) {
-#pragma unroll
-                for (int k = 0; k < K; ++k) {
-                    if (k <= q && q - k <= M - K) {       // row q can only land in these outputs
-                        const uint32_t eq = ((k & 1) ? b0 : ~b0) & ((k & 2) ? b1 : ~b1) & ((k & 4) ? b2 : ~b2);
-                        const uint32_t e = eq & mb[q];
-                        const uint32_t zlo = (e & 0xfu) * 0x10204080u;    // bit j -> sign bit of byte j
-                        const uint32_t zhi = (e >> 4) * 0x10204080u;
-                        out[k][0] |= ch[q].w[0] & prmt_b32(zlo, 0u, 0x9988u);
-                        out[k][1] |= ch[q].w[1] & prmt_b32(zlo, 0u, 0xbbaau);
-                        out[k][2] |= ch[q].w[2] & prmt_b32(zhi, 0u, 0x9988u);
-                        out[k][3] |= ch[q].w[3] & prmt_b32(zhi, 0u, 0xbbaau);
+                for (int q = 0; q < 8; ++q) {
+                    if (q < 4) {
+                        chunk_load<true>(ch[q], p.W, (rbase + q) * p.ld + c0, nvalid);
+                        mb[q] = (__ldg(p.mask + (rbase + q) * p.wpr + (c0 >> 5)) >> (8 * (lane & 3))) & 0xffu;
+                    } else {
+                        chunk_zero<true>(ch[q]);
+                        mb[q] = 0u;
                     }
                 }
-                const uint32_t c0b = b0 & mb[q];
-                b0 ^= mb[q];
-                const uint32_t c1b = b1 & c0b;
-                b1 ^= c0b;
-                b2 ^= c1b;
             }
-            // metadata: byte j of (lo, hi) = keep mask of column j (bit q = row q): gather bit j of every row's byte
-            const uint32_t x = mb[0] | (mb[1] << 8) | (mb[2] << 16) | (mb[3] << 24);
-            const uint32_t y = mb[4] | (mb[5] << 8) | (mb[6] << 16) | (mb[7] << 24);
-            uint32_t fields_lo = 0u, fields_hi = 0u;
 #pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                const uint32_t lo4 = (((x >> j) & 0x01010101u) * 0x10204080u) >> 28;     // rows 0..3
-                const uint32_t hi4 = (((y >> j) & 0x01010101u) * 0x10204080u) >> 28;     // rows 4..7
-                const uint32_t colmask = lo4 | (hi4 << 4);
-                if (j < 4) fields_lo |= colmask << (8 * j);
-                else fields_hi |= colmask << (8 * (j - 4));
-            }
-            p.meta[line * p.mwpl + (c0 >> 2)] = fields_lo;
-            if (nvalid > 4) p.meta[line * p.mwpl + (c0 >> 2) + 1] = fields_hi;
+            for (int g = 0; g < G; ++g) {
+                const int64_t r0 = rbase + g * M;
+                if (r0 < p.rows) {
+                    const int64_t line = r0 / M;
+                    uint32_t out[K][4];
 #pragma unroll
-            for (int k = 0; k < K; ++k) {
-                Chunk<true> o;
+                    for (int k = 0; k < K; ++k)
 #pragma unroll
-                for (int w = 0; w < 4; ++w) o.w[w] = out[k][w];
-                chunk_store_n<true>(o, p.values, (line * K + k) * p.vcols + c0, nvalid, p.vec_ok != 0);
+                        for (int w = 0; w < 4; ++w) out[k][w] = 0u;
+                    uint32_t b0 = 0u, b1 = 0u, b2 = 0u;          // bit-sliced count of kept rows above the current one
+                    uint32_t pos[2][2] = {{0u, 0u}, {0u, 0u}};   // 2:4: bit-sliced position bits of the two survivors
+#pragma unroll
+                    for (int q = 0; q < M; ++q) {
+                        const uint32_t m = mb[g * M + q];
+#pragma unroll
+                        for (int k = 0; k < K; ++k) {
+                            if (k <= q && q - k <= M - K) {   // row q can only land in these outputs
+                                const uint32_t eq = ((k & 1) ? b0 : ~b0) & ((k & 2) ? b1 : ~b1) & ((k & 4) ? b2 : ~b2);
+                                const uint32_t e = eq & m;
+                                const uint32_t zlo = (e & 0xfu) * 0x10204080u;    // bit j -> sign bit of byte j
+                                const uint32_t zhi = (e >> 4) * 0x10204080u;
+                                const Chunk<true> &row = ch[g * M + q];
+                                out[k][0] |= row.w[0] & prmt_b32(zlo, 0u, 0x9988u);
+                                out[k][1] |= row.w[1] & prmt_b32(zlo, 0u, 0xbbaau);
+                                out[k][2] |= row.w[2] & prmt_b32(zhi, 0u, 0x9988u);
+                                out[k][3] |= row.w[3] & prmt_b32(zhi, 0u, 0xbbaau);
+                                if constexpr (TWO_FOUR) {
+                                    if (q & 1) pos[k][0] |= e;
+                                    if (q & 2) pos[k][1] |= e;
+                                }
+                            }
+                        }
+                        const uint32_t c0b = b0 & m;
+                        b0 ^= m;
+                        const uint32_t c1b = b1 & c0b;
+                        b1 ^= c0b;
+                        b2 ^= c1b;
+                    }
+                    if constexpr (M == 8) {
+                        // byte j of (lo, hi) = keep mask of column j (bit q = row q)
+                        const uint32_t x = mb[0] | (mb[1] << 8) | (mb[2] << 16) | (mb[3] << 24);
+                        const uint32_t y = mb[4] | (mb[5] << 8) | (mb[6] << 16) | (mb[7] << 24);
+                        uint32_t fields_lo = 0u, fields_hi = 0u;
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) {
+                            const uint32_t colmask = gather_bit(x, j) | (gather_bit(y, j) << 4);
+                            if (j < 4) fields_lo |= colmask << (8 * j);
+                            else fields_hi |= colmask << (8 * (j - 4));
+                        }
+                        p.meta[line * p.mwpl + (c0 >> 2)] = fields_lo;
+                        if (nvalid > 4) p.meta[line * p.mwpl + (c0 >> 2) + 1] = fields_hi;
+                    } else {
+                        // nibble j = keep mask of column j, or for 2:4 pos_lo | pos_hi << 2
+                        const uint32_t x = TWO_FOUR ? (pos[0][0] | (pos[0][1] << 8) | (pos[1][0] << 16) | (pos[1][1] << 24))
+                                                    : (mb[g * M] | (mb[g * M + 1] << 8) | (mb[g * M + 2] << 16) | (mb[g * M + 3] << 24));
+                        uint32_t fields = 0u;
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) fields |= gather_bit(x, j) << (4 * j);
+                        p.meta[line * p.mwpl + (c0 >> 3)] = fields;
+                    }
+#pragma unroll
+                    for (int k = 0; k < K; ++k) {
+                        Chunk<true> o;
+#pragma unroll
+                        for (int w = 0; w < 4; ++w) o.w[w] = out[k][w];
+                        chunk_store_n<true>(o, p.values, (line * K + k) * p.vcols + c0, nvalid, p.vec_ok != 0);
+                    }
+                }
             }
         }
     }
@@ -380,8 +422,12 @@ cudaError_t compress_nm_launch(const void *W, const uint32_t *mask_bits, int64_t
     const int64_t cap = (int64_t)device_sm_count() * 8;
     const int grid = (int)(want < cap ? want : cap);
     if (bf16) {
-        if (!group_cols && m == 8 && n_keep == 4) {      // 4:8 on gate / up: the bit-sliced routing kernel
-            compress_rows8_bf16_kernel<4><<<grid, C_THREADS, 0, st>>>(p);
+        if (!group_cols && m == 8 && n_keep == 4) {      // 4:8 and 2:4 on gate / up: the bit-sliced routing kernel
+            compress_rows_bf16_kernel<8, 4, false><<<grid, C_THREADS, 0, st>>>(p);
+            return cudaGetLastError();
+        }
+        if (!group_cols && two_four) {
+            compress_rows_bf16_kernel<4, 2, true><<<grid, C_THREADS, 0, st>>>(p);
             return cudaGetLastError();
         }
         if (two_four) return launch_compress<true, 4, true>(p, group_cols, grid, st);
