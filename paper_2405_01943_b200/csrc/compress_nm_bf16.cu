@@ -17,7 +17,6 @@ struct CompressFastParams {
     uint32_t *meta;
     int64_t rows, cols, ld;
     int64_t wpr, vcols, mwpl;
-    int64_t units_per_strip, units;
     int n_keep, m, log2m;
     int two_four;
     int vec_ok;
@@ -25,7 +24,6 @@ struct CompressFastParams {
 
 constexpr int CF_THREADS = 256;
 constexpr int CF_COLS = 256;
-constexpr int CF_SLAB = 4;
 
 __device__ __forceinline__ uint32_t prmt_c(uint32_t a, uint32_t b, uint32_t sel)
 {
@@ -63,99 +61,55 @@ __device__ __forceinline__ uint32_t make_meta_2of4(uint32_t byte)
     return out;
 }
 
-// 16-byte asynchronous copy global -> shared (src_bytes = 0 writes zeros and reads nothing)
-__device__ __forceinline__ void cf_cp_async16(void *smem_dst, const void *gsrc, int src_bytes)
-{
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;"
-                 ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gsrc), "r"(src_bytes) : "memory");
-}
+// A warp task is 8 rows x 256 columns: a lane issues the loads of its 8 rows (and their mask words) back to back
+// and then works through them, so 16 independent requests per lane are in flight (measured faster than a
+// cp.async slab ring of 4-row units: 151 against 170 us on the 70B-shaped down projection).
+constexpr int CD_ROWS = 8;
 
-constexpr int CF_STAGES = 3;   // prefetch ring: slabs of CF_SLAB rows x 512 bytes per warp
-
-__global__ void __launch_bounds__(CF_THREADS, 4) compress_cols_bf16_kernel(const CompressFastParams p)
+__global__ void __launch_bounds__(CF_THREADS, 3) compress_cols_bf16_kernel(const CompressFastParams p)
 {
     __shared__ uint32_t sel_lut[4][256];
     __shared__ uint8_t meta_lut[256];
-    extern __shared__ uint4 ring_mem[];
-    uint4 (*ring)[CF_STAGES][CF_SLAB][32] = reinterpret_cast<uint4 (*)[CF_STAGES][CF_SLAB][32]>(ring_mem);
     for (int e = threadIdx.x; e < 1024; e += CF_THREADS) sel_lut[e >> 8][e & 255] = make_selectors(e & 255, e >> 8);
     if (threadIdx.x < 256) meta_lut[threadIdx.x] = (uint8_t)(p.two_four ? make_meta_2of4(threadIdx.x) : threadIdx.x);
     __syncthreads();
 
     const int lane = threadIdx.x & 31;
-    const int wib = threadIdx.x >> 5;
-    const int64_t warp = (int64_t)blockIdx.x * (CF_THREADS / 32) + wib;
+    const int64_t warp = (int64_t)blockIdx.x * (CF_THREADS / 32) + (threadIdx.x >> 5);
     const int64_t nwarps = (int64_t)gridDim.x * (CF_THREADS / 32);
-    const int64_t u_begin = p.units * warp / nwarps;
-    const int64_t u_end = p.units * (warp + 1) / nwarps;
-    const int ups = (int)p.units_per_strip;
+    const int64_t strips = (p.cols + CF_COLS - 1) / CF_COLS;
+    const int64_t row_blocks = (p.rows + CD_ROWS - 1) / CD_ROWS;
+    const int64_t ntasks = strips * row_blocks;
 
-    // unit position (strip, slab) advanced incrementally; `pre` runs CF_STAGES-1 units ahead for the prefetch
-    int strip = (int)(u_begin / p.units_per_strip), g = (int)(u_begin - (int64_t)strip * p.units_per_strip);
-    int pstrip = strip, pg = g;
-    int64_t u_pre = u_begin;
-    auto issue = [&](int stage) {
-        if (u_pre < u_end) {
-            const int64_t r0 = (int64_t)pg * CF_SLAB;
-            const int64_t c0 = (int64_t)pstrip * CF_COLS + lane * 8;
-            const uint16_t *src = p.W + r0 * p.ld + c0;
-#pragma unroll
-            for (int i = 0; i < CF_SLAB; ++i) {
-                const bool ok = c0 < p.cols && r0 + i < p.rows;
-                cf_cp_async16(&ring[wib][stage][i][lane], ok ? (const void *)src : (const void *)p.W, ok ? 16 : 0);
-                src += p.ld;
-            }
-        }
-        asm volatile("cp.async.commit_group;" ::: "memory");
-        ++u_pre;
-        if (++pg == ups) { pg = 0; ++pstrip; }
-    };
-#pragma unroll
-    for (int s = 0; s < CF_STAGES - 1; ++s) issue(s);
-
-    // mask words of a unit (one per row; the lane's byte is cut out later), fetched one unit ahead
-    auto load_mask_words = [&](int st_, int g_, uint32_t (&mw)[CF_SLAB]) {
-        const int64_t r0 = (int64_t)g_ * CF_SLAB;
-        const int64_t c0 = (int64_t)st_ * CF_COLS + lane * 8;
-#pragma unroll
-        for (int i = 0; i < CF_SLAB; ++i)
-            mw[i] = (c0 < p.cols && r0 + i < p.rows) ? __ldg(p.mask + (r0 + i) * p.wpr + (c0 >> 5)) : 0u;
-    };
-    uint32_t mw_next[CF_SLAB];
-    if (u_begin < u_end) load_mask_words(strip, g, mw_next);
-
-    int stage = 0;
-    for (int64_t u = u_begin; u < u_end; ++u) {
-        const int64_t r0 = (int64_t)g * CF_SLAB;
-        const int64_t c0 = (int64_t)strip * CF_COLS + lane * 8;
-        if (++g == ups) { g = 0; ++strip; }
+    for (int64_t task = warp; task < ntasks; task += nwarps) {
+        const int64_t strip = task % strips, rb = task / strips;
+        const int64_t r0 = rb * CD_ROWS;
+        const int64_t c0 = strip * CF_COLS + lane * 8;
         const int64_t left = p.cols - c0;
         const int nvalid = left >= 8 ? 8 : (left > 0 ? (int)left : 0);     // a multiple of m
         const int nout = (nvalid >> p.log2m) * p.n_keep;
-
-        uint32_t mb[CF_SLAB];
+        uint4 v[CD_ROWS];
+        uint32_t mw[CD_ROWS];
 #pragma unroll
-        for (int i = 0; i < CF_SLAB; ++i) mb[i] = (mw_next[i] >> (8 * (lane & 3))) & 0xffu;
-        if (u + 1 < u_end) load_mask_words(strip, g, mw_next);              // (strip, g) already point at unit u + 1
-        asm volatile("cp.async.wait_group %0;" ::"n"(CF_STAGES - 2) : "memory");
-        uint4 v[CF_SLAB];
-#pragma unroll
-        for (int i = 0; i < CF_SLAB; ++i) v[i] = ring[wib][stage][i][lane];
-        issue(stage == 0 ? CF_STAGES - 1 : stage - 1);
-        stage = stage + 1 == CF_STAGES ? 0 : stage + 1;
-
+        for (int i = 0; i < CD_ROWS; ++i) {
+            const bool ok = nvalid > 0 && r0 + i < p.rows;
+            // the row pitch is a multiple of 8 elements: a whole vector stays inside the row's pitch
+            v[i] = ok ? __ldcs(reinterpret_cast<const uint4 *>(p.W + (r0 + i) * p.ld + c0)) : make_uint4(0u, 0u, 0u, 0u);
+            mw[i] = ok ? __ldg(p.mask + (r0 + i) * p.wpr + (c0 >> 5)) : 0u;
+        }
         uint16_t *dst = p.values + r0 * p.vcols + (c0 >> p.log2m) * p.n_keep;
         uint32_t *mdst = p.meta + r0 * p.mwpl + (c0 >> 5);
 #pragma unroll
-        for (int i = 0; i < CF_SLAB; ++i, dst += p.vcols, mdst += p.mwpl) {
-            const uint32_t word = quad_pack_bytes((uint32_t)meta_lut[mb[i]], lane);
+        for (int i = 0; i < CD_ROWS; ++i, dst += p.vcols, mdst += p.mwpl) {
+            const uint32_t mb = (mw[i] >> (8 * (lane & 3))) & 0xffu;
+            const uint32_t word = quad_pack_bytes((uint32_t)meta_lut[mb], lane);
             if (nvalid == 0 || r0 + i >= p.rows) continue;
             if ((lane & 3) == 0) *mdst = word;
             uint32_t out[4];
 #pragma unroll
             for (int w = 0; w < 4; ++w) {
                 if (2 * w < nout) {
-                    const uint32_t s = sel_lut[w][mb[i]];
+                    const uint32_t s = sel_lut[w][mb];
                     const uint32_t t_lo = prmt_c(v[i].x, v[i].y, s & 0xffffu);
                     const uint32_t t_hi = prmt_c(v[i].z, v[i].w, s & 0xffffu);
                     out[w] = prmt_c(t_lo, t_hi, s >> 16);
@@ -193,16 +147,12 @@ cudaError_t compress_cols_bf16_launch(const void *W, const uint32_t *mask_bits, 
     p.two_four = (n_keep == 2 && m == 4) ? 1 : 0;
     p.vec_ok = ((p.vcols * 2) % 16 == 0) && ((reinterpret_cast<uintptr_t>(values) & 15u) == 0);
     const int64_t strips = (cols + CF_COLS - 1) / CF_COLS;
-    p.units_per_strip = (rows + CF_SLAB - 1) / CF_SLAB;
-    p.units = strips * p.units_per_strip;
+    const int64_t tasks = strips * ((rows + CD_ROWS - 1) / CD_ROWS);
     const int64_t wpb = CF_THREADS / 32;
-    const int64_t want = (p.units + wpb - 1) / wpb;
+    const int64_t want = (tasks + wpb - 1) / wpb;
     const int64_t cap = (int64_t)device_sm_count() * 8;
     const int grid = (int)(want < cap ? want : cap);
-    constexpr int ring_bytes = (CF_THREADS / 32) * CF_STAGES * CF_SLAB * 512;
-    const cudaError_t e = cudaFuncSetAttribute(compress_cols_bf16_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, ring_bytes);
-    if (e != cudaSuccess) return e;
-    compress_cols_bf16_kernel<<<grid, CF_THREADS, ring_bytes, st>>>(p);
+    compress_cols_bf16_kernel<<<grid, CF_THREADS, 0, st>>>(p);
     return cudaGetLastError();
 }
 
