@@ -99,6 +99,23 @@ __global__ void __launch_bounds__(CF_THREADS, 3) compress_cols_bf16_kernel(const
         }
         uint16_t *dst = p.values + r0 * p.vcols + (c0 >> p.log2m) * p.n_keep;
         uint32_t *mdst = p.meta + r0 * p.mwpl + (c0 >> 5);
+        // whole tiles of a half-density pattern (2:4, 4:8: four survivors per lane and row, one 8-byte store):
+        // the common case, decided once per task for the whole warp
+        const bool whole = p.vec_ok && nout == 4 && r0 + CD_ROWS <= p.rows &&
+                           (strip + 1) * CF_COLS <= p.cols;
+        if (whole) {
+#pragma unroll
+            for (int i = 0; i < CD_ROWS; ++i, dst += p.vcols, mdst += p.mwpl) {
+                const uint32_t mb = (mw[i] >> (8 * (lane & 3))) & 0xffu;
+                const uint32_t word = quad_pack_bytes((uint32_t)meta_lut[mb], lane);
+                if ((lane & 3) == 0) *mdst = word;
+                const uint32_t s0 = sel_lut[0][mb], s1 = sel_lut[1][mb];
+                const uint32_t o0 = prmt_c(prmt_c(v[i].x, v[i].y, s0 & 0xffffu), prmt_c(v[i].z, v[i].w, s0 & 0xffffu), s0 >> 16);
+                const uint32_t o1 = prmt_c(prmt_c(v[i].x, v[i].y, s1 & 0xffffu), prmt_c(v[i].z, v[i].w, s1 & 0xffffu), s1 >> 16);
+                __stcs(reinterpret_cast<uint2 *>(dst), make_uint2(o0, o1));
+            }
+            continue;
+        }
 #pragma unroll
         for (int i = 0; i < CD_ROWS; ++i, dst += p.vcols, mdst += p.mwpl) {
             const uint32_t mb = (mw[i] >> (8 * (lane & 3))) & 0xffu;
