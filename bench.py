@@ -59,9 +59,9 @@ def stage_b_bytes(cfg, compress=True):
 
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per launch from one ncu capture of this very
 # command on the default workload; see profiles/.  None where the kernel changed after the capture.
-NCU_DRAM_BYTES = {"llama2_70b": {"calib": 130.65e9 + 22.2e6,                                  # one launch, T = 262144
-                                 "score": (2 * (470.4 + 444.1) + 471.0 + 455.7) * 1e6,         # gate + up + down
-                                 "compress": (2 * (499.2 + 204.1) + 537.2 + 238.7) * 1e6}}
+NCU_DRAM_BYTES = {"llama2_70b": {"calib": 126.74e9 + 22.0e6,                                  # one launch, T = 262144
+                                 "score": (2 * (470.3 + 443.9) + 471.0 + 455.6) * 1e6,         # gate + up + down
+                                 "compress": (2 * (499.2 + 207.0) + 499.2 + 212.1) * 1e6}}
 
 
 def roofline_b(kernel, algorithmic_bytes, in_step_ms, isolated_ms, peaks, peak_src, traffic):
@@ -295,7 +295,7 @@ def run_ours(args):
                          "algorithmic_flops_per_launch": flops, "traffic": traffic.get("calib")},
             "roofline_score": roofline_b("score_{rows,cols}_bf16_kernel x3 (gate, up, down)", sb, score_ms, iso and iso["score"],
                                          peaks, peak_src, traffic.get("score")),
-            "roofline_compress": roofline_b("compress_* kernels x3", cb, comp_ms, iso and iso["compress"],
+            "roofline_compress": roofline_b("compress_rows_bf16_kernel x2 (gate, up) + compress_cols_bf16_kernel (down)", cb, comp_ms, iso and iso["compress"],
                                             peaks, peak_src, traffic.get("compress")),
             "unstructured": unstructured, "forward": forward,
             "e2e": e2e, "gpu_launches": KERNEL_LAUNCHES_PER_STEP * args.steps, "clocks": clocks,
