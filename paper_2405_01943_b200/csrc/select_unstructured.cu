@@ -491,6 +491,14 @@ struct EmitParams {
     int scale_per_row;           // 1: scale[r] (the norm runs along the lines), 0: scale[c]
 };
 
+// Rare path of the emit pass, kept out of line so that the streaming loop stays small enough to unroll: the
+// element's rounded product equals a threshold that the exact stage had to split.
+__device__ __noinline__ bool exact_tie_keeps(const LineResult *res, float a, float s, int64_t r)
+{
+    const unsigned long long k64 = (unsigned long long)__double_as_longlong((double)a * (double)s);
+    return k64 > res->tau64 || (k64 == res->tau64 && (long long)r <= res->cut);
+}
+
 template <bool BF16>
 __global__ void __launch_bounds__(256) select_emit_cols_kernel(const EmitParams p)
 {
@@ -516,36 +524,85 @@ __global__ void __launch_bounds__(256) select_emit_cols_kernel(const EmitParams 
                 if (!p.scale_per_row) sc[j] = p.scale[c0 + j];
             }
         }
-        for (int i = 0; i < 32; ++i) {
-            const int64_t r = rb * 32 + i;
-            if (r >= p.rows) break;                     // warp-uniform
-            Chunk<BF16> ch;
-            if (nvalid > 0) chunk_load<BF16>(ch, p.W, r * p.ld + c0, nvalid);
-            else chunk_zero<BF16>(ch);
-            const float rs = p.scale_per_row ? __ldg(p.scale + r) : 0.0f;
-            uint32_t keep = 0u;
+        if ((cb + 1) * 256 > p.cols) {
+            // the ragged last strip: row by row
+            for (int i = 0; i < 32; ++i) {
+                const int64_t r = rb * 32 + i;
+                if (r >= p.rows) break;                     // warp-uniform
+                Chunk<BF16> ch;
+                if (nvalid > 0) chunk_load<BF16>(ch, p.W, r * p.ld + c0, nvalid);
+                else chunk_zero<BF16>(ch);
+                const float rs = p.scale_per_row ? __ldg(p.scale + r) : 0.0f;
+                uint32_t keep = 0u;
 #pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                const float a = chunk_abs<BF16>(ch, j);
-                const float s = p.scale_per_row ? rs : sc[j];
-                const uint32_t key = __float_as_uint(__fmul_rn(a, s));
-                bool k = key > tau[j];
-                if (key == tau[j] && j < nvalid) {
-                    k = true;                           // products equal to the threshold stay ...
-                    if ((exact_cols >> j) & 1u) {       // ... unless the exact stage had to split them
-                        const LineResult res = p.results[c0 + j];
-                        const unsigned long long k64 = (unsigned long long)__double_as_longlong((double)a * (double)s);
-                        k = k64 > res.tau64 || (k64 == res.tau64 && (long long)r <= res.cut);
+                for (int j = 0; j < 8; ++j) {
+                    const float a = chunk_abs<BF16>(ch, j);
+                    const float s = p.scale_per_row ? rs : sc[j];
+                    const uint32_t key = __float_as_uint(__fmul_rn(a, s));
+                    bool k = key > tau[j];
+                    if (key == tau[j] && j < nvalid) {
+                        k = true;                           // products equal to the threshold stay ...
+                        if ((exact_cols >> j) & 1u) {       // ... unless the exact stage had to split them
+                            const LineResult res = p.results[c0 + j];
+                            const unsigned long long k64 = (unsigned long long)__double_as_longlong((double)a * (double)s);
+                            k = k64 > res.tau64 || (k64 == res.tau64 && (long long)r <= res.cut);
+                        }
+                    }
+                    keep |= (k && j < nvalid ? 1u : 0u) << j;
+                }
+                const uint32_t word = quad_pack_bytes(keep, lane);
+                if (nvalid > 0) {
+                    if (p.mask && (lane & 3) == 0) p.mask[r * p.wpr + (c0 >> 5)] = word;
+                    if (p.Wp) {
+                        chunk_apply_mask<BF16>(ch, keep);
+                        chunk_store<BF16>(ch, p.Wp, r * p.ld + c0, nvalid);
                     }
                 }
-                keep |= (k && j < nvalid ? 1u : 0u) << j;
             }
-            const uint32_t word = quad_pack_bytes(keep, lane);
-            if (nvalid > 0) {
-                if (p.mask && (lane & 3) == 0) p.mask[r * p.wpr + (c0 >> 5)] = word;
-                if (p.Wp) {
-                    chunk_apply_mask<BF16>(ch, keep);
-                    chunk_store<BF16>(ch, p.Wp, r * p.ld + c0, nvalid);
+            continue;
+        }
+        // whole strips, 8 rows at a time: all their loads are issued before any row is processed
+#pragma unroll 1
+        for (int i0 = 0; i0 < 32; i0 += 8) {
+            const int64_t rbase = rb * 32 + i0;
+            if (rbase >= p.rows) break;                     // warp-uniform
+            Chunk<BF16> chs[8];
+            float rss[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const int64_t r = rbase + u;
+                if (r < p.rows) chunk_load<BF16>(chs[u], p.W, r * p.ld + c0, 8);
+                else chunk_zero<BF16>(chs[u]);
+                rss[u] = (p.scale_per_row && r < p.rows) ? __ldg(p.scale + r) : 0.0f;
+            }
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const int64_t r = rbase + u;
+                uint32_t keep = 0u;
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    const float a = chunk_abs<BF16>(chs[u], j);
+                    const float s = p.scale_per_row ? rss[u] : sc[j];
+                    const uint32_t key = __float_as_uint(__fmul_rn(a, s));
+                    bool k = key >= tau[j];                 // products equal to the threshold stay ...
+                    if (key == tau[j] && ((exact_cols >> j) & 1u))
+                        k = exact_tie_keeps(p.results + c0 + j, a, s, r);   // ... unless the exact stage split them
+                    keep |= (k ? 1u : 0u) << j;
+                }
+                const uint32_t word = quad_pack_bytes(keep, lane);
+                if (r < p.rows) {
+                    if (p.mask && (lane & 3) == 0) p.mask[r * p.wpr + (c0 >> 5)] = word;
+                    if (p.Wp) {
+                        chunk_apply_mask<BF16>(chs[u], keep);
+                        if constexpr (BF16) {
+                            __stcs(reinterpret_cast<uint4 *>(static_cast<uint16_t *>(p.Wp) + r * p.ld + c0),
+                                   make_uint4(chs[u].w[0], chs[u].w[1], chs[u].w[2], chs[u].w[3]));
+                        } else {
+                            uint4 *dst = reinterpret_cast<uint4 *>(static_cast<uint32_t *>(p.Wp) + r * p.ld + c0);
+                            __stcs(dst, make_uint4(chs[u].w[0], chs[u].w[1], chs[u].w[2], chs[u].w[3]));
+                            __stcs(dst + 1, make_uint4(chs[u].w[4], chs[u].w[5], chs[u].w[6], chs[u].w[7]));
+                        }
+                    }
                 }
             }
         }
