@@ -205,28 +205,46 @@ __device__ __forceinline__ void cmp_exchange(float &hi, float &lo)
     lo = b;
 }
 
+// The n_keep-th and (n_keep+1)-th largest of M rounded products (M = 4: 5-comparator network, M = 8: 19).
+template <int M>
+__device__ __forceinline__ void cut_values(const float (&pf)[M], int n_keep, float &t, float &next)
+{
+    float s[M];
+#pragma unroll
+    for (int q = 0; q < M; ++q) s[q] = pf[q];
+    if constexpr (M == 4) {
+        cmp_exchange(s[0], s[1]); cmp_exchange(s[2], s[3]);
+        cmp_exchange(s[0], s[2]); cmp_exchange(s[1], s[3]);
+        cmp_exchange(s[1], s[2]);                         // s[0] >= s[1] >= s[2] >= s[3]
+        switch (n_keep) {                                 // n_keep in 1..3, the same for every lane
+        case 1: t = s[0]; next = s[1]; break;
+        case 2: t = s[1]; next = s[2]; break;
+        default: t = s[2]; next = s[3]; break;
+        }
+    } else {
+        cmp_exchange(s[0], s[1]); cmp_exchange(s[2], s[3]); cmp_exchange(s[4], s[5]); cmp_exchange(s[6], s[7]);
+        cmp_exchange(s[0], s[2]); cmp_exchange(s[1], s[3]); cmp_exchange(s[4], s[6]); cmp_exchange(s[5], s[7]);
+        cmp_exchange(s[1], s[2]); cmp_exchange(s[5], s[6]); cmp_exchange(s[0], s[4]); cmp_exchange(s[3], s[7]);
+        cmp_exchange(s[1], s[5]); cmp_exchange(s[2], s[6]);
+        cmp_exchange(s[1], s[4]); cmp_exchange(s[3], s[6]);
+        cmp_exchange(s[2], s[4]); cmp_exchange(s[3], s[5]);
+        cmp_exchange(s[3], s[4]);                         // s[0] >= s[1] >= ... >= s[7]
+        switch (n_keep) {                                 // n_keep in 1..7, the same for every lane
+        case 1: t = s[0]; next = s[1]; break;
+        case 2: t = s[1]; next = s[2]; break;
+        case 3: t = s[2]; next = s[3]; break;
+        case 4: t = s[3]; next = s[4]; break;
+        case 5: t = s[4]; next = s[5]; break;
+        case 6: t = s[5]; next = s[6]; break;
+        default: t = s[6]; next = s[7]; break;
+        }
+    }
+}
+
 __device__ __forceinline__ bool threshold_group8(const float (&pf)[8], int n_keep, uint32_t (&D)[8])
 {
-    float s[8];
-#pragma unroll
-    for (int q = 0; q < 8; ++q) s[q] = pf[q];
-    cmp_exchange(s[0], s[1]); cmp_exchange(s[2], s[3]); cmp_exchange(s[4], s[5]); cmp_exchange(s[6], s[7]);
-    cmp_exchange(s[0], s[2]); cmp_exchange(s[1], s[3]); cmp_exchange(s[4], s[6]); cmp_exchange(s[5], s[7]);
-    cmp_exchange(s[1], s[2]); cmp_exchange(s[5], s[6]); cmp_exchange(s[0], s[4]); cmp_exchange(s[3], s[7]);
-    cmp_exchange(s[1], s[5]); cmp_exchange(s[2], s[6]);
-    cmp_exchange(s[1], s[4]); cmp_exchange(s[3], s[6]);
-    cmp_exchange(s[2], s[4]); cmp_exchange(s[3], s[5]);
-    cmp_exchange(s[3], s[4]);                         // s[0] >= s[1] >= ... >= s[7]
     float t, next;
-    switch (n_keep) {                                 // n_keep in 1..7, the same for every lane
-    case 1: t = s[0]; next = s[1]; break;
-    case 2: t = s[1]; next = s[2]; break;
-    case 3: t = s[2]; next = s[3]; break;
-    case 4: t = s[3]; next = s[4]; break;
-    case 5: t = s[4]; next = s[5]; break;
-    case 6: t = s[5]; next = s[6]; break;
-    default: t = s[6]; next = s[7]; break;
-    }
+    cut_values<8>(pf, n_keep, t, next);
 #pragma unroll
     for (int q = 0; q < 8; ++q) D[q] = __funnelshift_l(__float_as_uint(__fsub_rn(pf[q], t)), D[q], 1);
     return t == next;
@@ -441,7 +459,6 @@ __global__ void __launch_bounds__(F_THREADS, M == 8 ? 2 : F_MIN_BLOCKS) score_ro
 template <int M, bool NORM_COLS>
 __global__ void __launch_bounds__(F_THREADS, M == 8 ? 3 : F_MIN_BLOCKS) score_cols_bf16_kernel(const ScoreFastParams p)
 {
-    constexpr int NP = M * (M - 1) / 2;
     constexpr int G = 8 / M;             // groups inside a lane's 8 columns
     constexpr int STAGES = ring_stages(F_SLAB);
     extern __shared__ uint4 ring_mem[];
@@ -505,60 +522,33 @@ __global__ void __launch_bounds__(F_THREADS, M == 8 ? 3 : F_MIN_BLOCKS) score_co
         ++u_pre;
         stage = stage + 1 == STAGES ? 0 : stage + 1;
 
-        // M == 8: C[0][q] collects "p_q < threshold" per row (threshold_group8); else C[g][pair] the pairwise order
-        uint32_t C[G][NP];
-#pragma unroll
-        for (int g = 0; g < G; ++g)
-#pragma unroll
-            for (int i = 0; i < (M == 8 ? M : NP); ++i) C[g][i] = 0u;
+        // Every group is compared with its own cut value t (the n_keep-th largest rounded product): the sign of
+        // p - t is shifted straight into the row's byte, column 7 first, so that bit j ends up as "column j pruned".
+        // The rule is proven unless t equals the next value (a tie across the cut): then the slab goes the exact way.
+        uint32_t row_keep[F_SLAB];
         bool tie = false;
         float rsv[F_SLAB];
 #pragma unroll
-        for (int i = F_SLAB - 1; i >= 0; --i) {       // last row first: after the inserts row i sits at bit i
+        for (int i = 0; i < F_SLAB; ++i) {
             float rs = 0.0f;
             if constexpr (!NORM_COLS) rs = __shfl_sync(FULL_MASK, lane_scale, (int)(r0 & 31) + i);
             rsv[i] = rs;
+            uint32_t pruned = 0u;
 #pragma unroll
-            for (int g = 0; g < G; ++g) {
+            for (int g = G - 1; g >= 0; --g) {
                 float pf[M];
 #pragma unroll
                 for (int q = 0; q < M; ++q) {
                     const int j = g * M + q;
                     pf[q] = prod_of(word_of(v[i], j >> 1), (j & 1) != 0, NORM_COLS ? sc[j] : rs);
                 }
-                if constexpr (M == 8) {
-                    uint32_t (&D)[8] = reinterpret_cast<uint32_t (&)[8]>(C[g]);
-                    tie |= threshold_group8(pf, p.n_keep, D);
-                } else {
-                    tie |= compare_group<M>(pf, C[g]);
-                }
+                float t, next;
+                cut_values<M>(pf, p.n_keep, t, next);
+                tie |= t == next;
+#pragma unroll
+                for (int q = M - 1; q >= 0; --q) pruned = __funnelshift_l(__float_as_uint(__fsub_rn(pf[q], t)), pruned, 1);
             }
-        }
-        // Q[h]: byte a = keep bits (bit i = row i) of column 4h + a
-        uint32_t Q[2];
-#pragma unroll
-        for (int g = 0; g < G; ++g) {
-            uint32_t K[M];
-            if constexpr (M == 8) {
-#pragma unroll
-                for (int q = 0; q < M; ++q) K[q] = ~C[g][q];
-            } else {
-                keep_from_pairs<M>(C[g], p.n_keep, K);
-            }
-#pragma unroll
-            for (int h = 0; h < M / 4; ++h) {
-                const uint32_t q = (K[4 * h] & 0xffu) | ((K[4 * h + 1] & 0xffu) << 8) | ((K[4 * h + 2] & 0xffu) << 16) |
-                                   (K[4 * h + 3] << 24);
-                Q[g * (M / 4) + h] = q;
-            }
-        }
-        uint32_t row_keep[F_SLAB];
-#pragma unroll
-        for (int i = 0; i < F_SLAB; ++i) {
-            // gather bit i of each byte of Q[h] into a nibble (columns 4h .. 4h+3)
-            const uint32_t n0 = (((Q[0] >> i) & 0x01010101u) * 0x10204080u) >> 28;
-            const uint32_t n1 = (((Q[1] >> i) & 0x01010101u) * 0x10204080u) >> 28;
-            row_keep[i] = n0 | (n1 << 4);
+            row_keep[i] = ~pruned & 0xffu;
         }
         if (tie && nvalid > 0) {   // ragged slabs (zero padding ties) also land here; still exact
             TileWords<F_SLAB> t;
