@@ -4,13 +4,13 @@
 // vector; a warp row is one contiguous 512-byte segment), but the selection is done with 32-bit
 // integer and bit-sliced logic instead of per-element double arithmetic:
 //
-//   * p = fl32(|w| * scale).  Rounding is monotone, so p_b > p_a proves score_b > score_a for the
-//     exact products; the comparison is the sign of the float difference p_a - p_b (never wrong), shifted
-//     into a bit-sliced word with one funnel shift (bit j of a word = column j, or row j, of the lane's tile).
-//   * ranks are counted with full adders on those words (one LOP3 each) and compared with n_keep, which
-//     yields the keep bits of 8 groups at once;
-//   * only when two rounded products of a group are EQUAL is the order not proven; the lane then
-//     recomputes its tile's keep bits with exact double products (rare on real data, always correct).
+//   * p = fl32(|w| * scale).  Rounding is monotone, so p_b > p_a proves score_b > score_a for the exact
+//     products.  A group's products are sorted with a min / max network, which gives the cut value t (the
+//     n_keep-th largest) and the value below it; every element is then compared with t by the sign of the float
+//     difference p - t (never wrong), shifted into a bit-sliced word with one funnel shift (bit j of a word =
+//     column j of the lane's tile).
+//   * only when the two values at the cut are EQUAL is the order not proven; the lane then recomputes its
+//     tile's keep bits with exact double products (rare on real data, always correct).
 //   * pruned weights: keep bits are spread to byte sign bits with one multiply and expanded to 16-bit
 //     masks with the sign-replicating byte permute.
 //
@@ -107,97 +107,12 @@ __device__ __forceinline__ float prod_of(uint32_t word, bool hi, float scale)
     return fabsf(__uint_as_float(fb)) * scale;
 }
 
-// Pair index of (a, b), a < b, in the order (0,1),(0,2),...,(0,M-1),(1,2),...
-template <int M>
-__host__ __device__ constexpr int pair_index(int a, int b) { return a * M - a * (a + 1) / 2 + (b - a - 1); }
-
-// Pairwise comparisons of one group of M rounded products: shifts "p_b > p_a" (the sign of p_a - p_b, which
-// floating-point subtraction never gets wrong) into the bit-sliced words C and returns true if two products may
-// be equal.  Equality is found with a running product of the differences (FMA pipe): it is 0 -- or NaN after an
-// overflow -- exactly when some difference is 0, and it can only err towards "maybe" (underflow), which sends
-// the lane to the exact path.
-template <int M>
-__device__ __forceinline__ bool compare_group(const float (&pf)[M], uint32_t (&C)[M * (M - 1) / 2])
-{
-    bool maybe_tie = false;
-    if constexpr (M == 4) {
-        float t = 1.2676506e30f;   // 2^100: head-room against underflow of six small differences
-#pragma unroll
-        for (int a = 0; a < M; ++a)
-#pragma unroll
-            for (int b = a + 1; b < M; ++b) {
-                const float dlt = __fsub_rn(pf[a], pf[b]);
-                C[pair_index<M>(a, b)] = __funnelshift_l(__float_as_uint(dlt), C[pair_index<M>(a, b)], 1);
-                t = __fmul_rn(t, dlt);
-            }
-        maybe_tie = !(fabsf(t) > 0.0f);
-    } else {
-#pragma unroll
-        for (int a = 0; a < M - 1; ++a) {
-            float t = 1.8446744e19f;   // 2^64 per chain of at most 7 differences
-#pragma unroll
-            for (int b = a + 1; b < M; ++b) {
-                const float dlt = __fsub_rn(pf[a], pf[b]);
-                C[pair_index<M>(a, b)] = __funnelshift_l(__float_as_uint(dlt), C[pair_index<M>(a, b)], 1);
-                t = __fmul_rn(t, dlt);
-            }
-            maybe_tie |= !(fabsf(t) > 0.0f);
-        }
-    }
-    return maybe_tie;
-}
-
-// full adder on bit-sliced words
-__device__ __forceinline__ uint32_t xor3(uint32_t a, uint32_t b, uint32_t c) { return a ^ b ^ c; }
-__device__ __forceinline__ uint32_t maj3(uint32_t a, uint32_t b, uint32_t c) { return (a & b) | (a & c) | (b & c); }
-
-// rank < n_keep for a bit-sliced 3-bit rank (b2 b1 b0), n_keep in 1..7
-__device__ __forceinline__ uint32_t rank_below(uint32_t b2, uint32_t b1, uint32_t b0, int n_keep)
-{
-    switch (n_keep) {
-    case 1: return ~(b2 | b1 | b0);
-    case 2: return ~(b2 | b1);
-    case 3: return ~(b2 | (b1 & b0));
-    case 4: return ~b2;
-    case 5: return ~(b2 & (b1 | b0));
-    case 6: return ~(b2 & b1);
-    default: return ~(b2 & b1 & b0);
-    }
-}
-
-
-// Keep words from the bit-sliced comparison words C[pair] (bit set: the later element b beats a).
-// Element a is preceded by every earlier k that b-beats... i.e. rank_a = sum_{k<a} !C[k,a] + sum_{k>a} C[a,k].
-template <int M>
-__device__ __forceinline__ void keep_from_pairs(const uint32_t (&C)[M * (M - 1) / 2], int n_keep, uint32_t (&K)[M])
-{
-#pragma unroll
-    for (int a = 0; a < M; ++a) {
-        uint32_t in[M - 1];
-#pragma unroll
-        for (int k = 0; k < M; ++k) {
-            if (k < a) in[k] = ~C[pair_index<M>(k, a)];
-            else if (k > a) in[k - 1] = C[pair_index<M>(a, k)];
-        }
-        if constexpr (M == 4) {
-            const uint32_t b0 = xor3(in[0], in[1], in[2]);
-            const uint32_t b1 = maj3(in[0], in[1], in[2]);
-            K[a] = rank_below(0u, b1, b0, n_keep);
-        } else {
-            const uint32_t s1 = xor3(in[0], in[1], in[2]), c1 = maj3(in[0], in[1], in[2]);
-            const uint32_t s2 = xor3(in[3], in[4], in[5]), c2 = maj3(in[3], in[4], in[5]);
-            const uint32_t b0 = xor3(s1, s2, in[6]), c3 = maj3(s1, s2, in[6]);
-            const uint32_t b1 = xor3(c1, c2, c3), b2 = maj3(c1, c2, c3);
-            K[a] = rank_below(b2, b1, b0, n_keep);
-        }
-    }
-}
-
-// Groups of 8: instead of all 28 pairwise comparisons, the rounded products are sorted with a 19-comparator
-// network (min / max pairs) and every element is compared with the n_keep-th largest, t: "p >= t" is the keep
-// rule whenever t is strictly above the next value (monotone rounding then proves the same for the exact
-// products; equal products on one side of the cut need no order).  Shifts "p_q < t" (the sign of p_q - t) into
-// the bit-sliced words D and returns true if the two values at the cut are equal (order not proven).
+// Selection inside a group of M rounded products: the products are sorted with a small min / max network (5
+// comparators for M = 4, 19 for M = 8) and every element is compared with the n_keep-th largest, t.  "p >= t" is
+// the keep rule whenever t is strictly above the next value: monotone rounding then proves the same for the exact
+// products, and equal products on one side of the cut need no order.  threshold_group shifts "p_q < t" (the sign
+// of p_q - t, which floating-point subtraction never gets wrong) into the bit-sliced words D and returns true if
+// the two values at the cut are equal (order not proven: the lane then takes the exact path).
 __device__ __forceinline__ void cmp_exchange(float &hi, float &lo)
 {
     const float a = fmaxf(hi, lo), b = fminf(hi, lo);
@@ -241,12 +156,13 @@ __device__ __forceinline__ void cut_values(const float (&pf)[M], int n_keep, flo
     }
 }
 
-__device__ __forceinline__ bool threshold_group8(const float (&pf)[8], int n_keep, uint32_t (&D)[8])
+template <int M>
+__device__ __forceinline__ bool threshold_group(const float (&pf)[M], int n_keep, uint32_t (&D)[M])
 {
     float t, next;
-    cut_values<8>(pf, n_keep, t, next);
+    cut_values<M>(pf, n_keep, t, next);
 #pragma unroll
-    for (int q = 0; q < 8; ++q) D[q] = __funnelshift_l(__float_as_uint(__fsub_rn(pf[q], t)), D[q], 1);
+    for (int q = 0; q < M; ++q) D[q] = __funnelshift_l(__float_as_uint(__fsub_rn(pf[q], t)), D[q], 1);
     return t == next;
 }
 
@@ -331,7 +247,6 @@ __device__ __noinline__ KeepWords<F_SLAB> exact_keep_cols(TileWords<F_SLAB> t, S
 template <int M, bool NORM_COLS>
 __global__ void __launch_bounds__(F_THREADS, M == 8 ? 2 : F_MIN_BLOCKS) score_rows_bf16_kernel(const ScoreFastParams p)
 {
-    constexpr int NP = M * (M - 1) / 2;
     constexpr int STAGES = ring_stages(M);
     extern __shared__ uint4 ring_mem[];
     const int lane = threadIdx.x & 31;
@@ -402,34 +317,21 @@ __global__ void __launch_bounds__(F_THREADS, M == 8 ? 2 : F_MIN_BLOCKS) score_ro
             if constexpr (!NORM_COLS) rs[q] = __shfl_sync(FULL_MASK, lane_scale, (int)(r0 & 31) + q);
         }
 
-        uint32_t K[M];
+        // D[q]: bit j = "row q is pruned at column j" (the sign of p - t, t the column group's cut value)
+        uint32_t D[M];
+#pragma unroll
+        for (int q = 0; q < M; ++q) D[q] = 0u;
         bool tie = false;
-        if constexpr (M == 8) {
-            uint32_t D[M];
 #pragma unroll
-            for (int q = 0; q < M; ++q) D[q] = 0u;
+        for (int j = 7; j >= 0; --j) {       // column 7 first: after 8 inserts column j sits at bit j
+            float pf[M];
 #pragma unroll
-            for (int j = 7; j >= 0; --j) {   // column 7 first: after 8 inserts column j sits at bit j
-                float pf[M];
-#pragma unroll
-                for (int q = 0; q < M; ++q) pf[q] = prod_of(word_of(v[q], j >> 1), (j & 1) != 0, NORM_COLS ? sc[j] : rs[q]);
-                tie |= threshold_group8(pf, p.n_keep, D);
-            }
-#pragma unroll
-            for (int q = 0; q < M; ++q) K[q] = ~D[q];
-        } else {
-            uint32_t C[NP];
-#pragma unroll
-            for (int i = 0; i < NP; ++i) C[i] = 0u;
-#pragma unroll
-            for (int j = 7; j >= 0; --j) {   // column 7 first: after 8 inserts column j sits at bit j
-                float pf[M];
-#pragma unroll
-                for (int q = 0; q < M; ++q) pf[q] = prod_of(word_of(v[q], j >> 1), (j & 1) != 0, NORM_COLS ? sc[j] : rs[q]);
-                tie |= compare_group<M>(pf, C);
-            }
-            keep_from_pairs<M>(C, p.n_keep, K);
+            for (int q = 0; q < M; ++q) pf[q] = prod_of(word_of(v[q], j >> 1), (j & 1) != 0, NORM_COLS ? sc[j] : rs[q]);
+            tie |= threshold_group<M>(pf, p.n_keep, D);
         }
+        uint32_t K[M];
+#pragma unroll
+        for (int q = 0; q < M; ++q) K[q] = ~D[q];
         if (tie && nvalid > 0) {   // ragged lanes (zero padding ties) also land here; still exact
             TileWords<M> t;
             Scales8 s8;
