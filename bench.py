@@ -59,9 +59,9 @@ def stage_b_bytes(cfg, compress=True):
 
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per launch from one ncu capture of this very
 # command on the default workload; see profiles/.  None where the kernel changed after the capture.
-NCU_DRAM_BYTES = {"llama2_70b": {"calib": 126.74e9 + 22.0e6,                                  # one launch, T = 262144
-                                 "score": (2 * (470.3 + 443.9) + 471.0 + 455.6) * 1e6,         # gate + up + down
-                                 "compress": (2 * (499.2 + 207.0) + 499.2 + 212.1) * 1e6}}
+NCU_DRAM_BYTES = {"llama2_70b": {"calib": 122.00e9 + 20.8e6,                                  # one launch, T = 262144
+                                 "score": (2 * (470.4 + 443.6) + 471.4 + 454.4) * 1e6,         # gate + up + down
+                                 "compress": (2 * (499.1 + 206.7) + 499.2 + 214.1) * 1e6}}
 
 
 def roofline_b(kernel, algorithmic_bytes, in_step_ms, isolated_ms, peaks, peak_src, traffic):
