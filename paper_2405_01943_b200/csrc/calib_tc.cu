@@ -31,7 +31,7 @@ constexpr int TC_BN = 256;         // tokens per tile (MMA N)
 constexpr int TC_BK = 64;          // k per ring slot: 64 bf16 = one 128-byte swizzle row
 constexpr int TC_UMMA_K = 16;      // k per tcgen05.mma for 16-bit inputs
 constexpr int TC_STAGES = 3;
-constexpr int TC_BAND_TILES = 16;    // token tiles per band (one partial per band and neuron)
+constexpr int TC_MAX_BAND_TILES = 16;   // token tiles per band (one partial per band and neuron) at most
 constexpr int TC_SUPER_BANDS = 16;   // bands interleaved in the item order for L2 sharing
 constexpr unsigned long long TC_ALIGN_NS = 20000ull;   // longest a CTA waits for the others at a tile boundary
 constexpr int TC_THREADS = 192;
@@ -47,6 +47,7 @@ struct TcParams {
     int *align_counter;  // arrivals of the tile-boundary alignment barrier (zeroed before the launch)
     int64_t T, I, d;
     int64_t neuron_tiles, token_tiles, bands, items, k_blocks;
+    int band_tiles;      // token tiles per band (calib_tc_band_tiles)
 };
 
 struct ItemCoord { int64_t nt, band; };
@@ -116,8 +117,8 @@ calib_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
             int64_t round = 0;
             for (int64_t idx = blockIdx.x; idx < p.items && ok; idx += gridDim.x, ++round) {
                 const ItemCoord c = decode_item(p, idx);
-                const int64_t tt0 = c.band * TC_BAND_TILES;
-                const int64_t tt1 = tt0 + TC_BAND_TILES < p.token_tiles ? tt0 + TC_BAND_TILES : p.token_tiles;
+                const int64_t tt0 = c.band * p.band_tiles;
+                const int64_t tt1 = tt0 + p.band_tiles < p.token_tiles ? tt0 + p.band_tiles : p.token_tiles;
                 const int64_t left = p.items - round * gridDim.x;
                 const int round_ctas = (int)(left < (int64_t)gridDim.x ? left : (int64_t)gridDim.x);   // CTAs with an item in this round
                 for (int64_t tt = tt0; tt < tt1 && ok; ++tt) {
@@ -127,7 +128,7 @@ calib_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
                     // longer than TC_ALIGN_NS (a late or absent CTA just is not waited for).
                     {
                         const int t_in_item = (int)(tt - tt0);
-                        const int target = (int)(round * gridDim.x) * TC_BAND_TILES + round_ctas * (t_in_item + 1);
+                        const int target = (int)(round * gridDim.x) * p.band_tiles + round_ctas * (t_in_item + 1);
                         atomicAdd(p.align_counter, 1);
                         const unsigned long long t0 = global_ns();
                         while (*reinterpret_cast<volatile int *>(p.align_counter) < target && global_ns() - t0 < TC_ALIGN_NS) { }
@@ -143,8 +144,8 @@ calib_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
                         if (++stage == TC_STAGES) { stage = 0; phase ^= 1u; }
                     }
                 }
-                // a short last band still counts TC_BAND_TILES arrivals, so later rounds' targets hold
-                if (tt1 - tt0 < TC_BAND_TILES) atomicAdd(p.align_counter, (int)(TC_BAND_TILES - (tt1 - tt0)));
+                // a short last band still counts p.band_tiles arrivals, so later rounds' targets hold
+                if (tt1 - tt0 < p.band_tiles) atomicAdd(p.align_counter, (int)(p.band_tiles - (tt1 - tt0)));
             }
             if (!ok) { *abort_flag = 1; atomicExch(p.status, (int)DASS_ERR_TIMEOUT); }
         }
@@ -157,8 +158,8 @@ calib_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
             bool ok = true;
             for (int64_t idx = blockIdx.x; idx < p.items && ok; idx += gridDim.x) {
                 const ItemCoord c = decode_item(p, idx);
-                const int64_t tt0 = c.band * TC_BAND_TILES;
-                const int64_t tt1 = tt0 + TC_BAND_TILES < p.token_tiles ? tt0 + TC_BAND_TILES : p.token_tiles;
+                const int64_t tt0 = c.band * p.band_tiles;
+                const int64_t tt1 = tt0 + p.band_tiles < p.token_tiles ? tt0 + p.band_tiles : p.token_tiles;
                 for (int64_t tt = tt0; tt < tt1 && ok; ++tt, ++tile) {
                     // the epilogue must have drained the previous tile's accumulators
                     if (!mbar_wait(bar_acc_empty, (tile & 1u) ^ 1u, abort_flag)) { ok = false; break; }
@@ -194,8 +195,8 @@ calib_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
         bool ok = true;
         for (int64_t idx = blockIdx.x; idx < p.items && ok; idx += gridDim.x) {
             const ItemCoord c = decode_item(p, idx);
-            const int64_t tt0 = c.band * TC_BAND_TILES;
-            const int64_t tt1 = tt0 + TC_BAND_TILES < p.token_tiles ? tt0 + TC_BAND_TILES : p.token_tiles;
+            const int64_t tt0 = c.band * p.band_tiles;
+            const int64_t tt1 = tt0 + p.band_tiles < p.token_tiles ? tt0 + p.band_tiles : p.token_tiles;
             double acc = 0.0;
             for (int64_t tt = tt0; tt < tt1 && ok; ++tt, ++tile) {
                 if (!mbar_wait(bar_acc_full, tile & 1u, abort_flag)) { ok = false; break; }
@@ -273,11 +274,32 @@ bool tc_make_map(CUtensorMap *map, const void *ptr, int64_t rows, int64_t cols, 
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Token tiles per band.  16 keeps a W tile in L2 for 16 token tiles; with few tokens that leaves the persistent
+// grid (148 CTAs, which this library is written for) with a part-filled last round, so a shorter band is taken
+// when it saves at least 1 % of the tile steps and the partial sums (one double per band and neuron) stay within
+// 14 MiB.  A function of (T, I) only: the workspace query, both tensor-core kernels and the scratch-free entry
+// point must agree on it.
+int calib_tc_band_tiles(int64_t T, int64_t I)
+{
+    const int64_t tiles = (I + TC_BM - 1) / TC_BM;
+    const int64_t token_tiles = (T + TC_BN - 1) / TC_BN;
+    auto bands = [&](int bt) { return (token_tiles + bt - 1) / bt; };
+    auto steps = [&](int bt) { return ((tiles * bands(bt) + 147) / 148) * bt; };
+    int best = TC_MAX_BAND_TILES;
+    int64_t best_steps = steps(best);
+    for (int bt = TC_MAX_BAND_TILES / 2; bt >= 1; bt >>= 1) {
+        const int64_t st = steps(bt);
+        if (bands(bt) * I * (int64_t)sizeof(double) > ((int64_t)14 << 20)) break;
+        if (st * 100 < best_steps * 99) { best = bt; best_steps = st; }
+    }
+    return best;
+}
+
 int64_t calib_tc_parts(int64_t T, int64_t I)
 {
-    (void)I;
     const int64_t token_tiles = (T + TC_BN - 1) / TC_BN;
-    return (token_tiles + TC_BAND_TILES - 1) / TC_BAND_TILES;
+    const int bt = calib_tc_band_tiles(T, I);
+    return (token_tiles + bt - 1) / bt;
 }
 
 int device_sm_count();   // dass_abi.cu
@@ -333,6 +355,7 @@ dass_status calib_tc_launch(const void *X, int64_t T, int64_t ldx, const void *W
     p.T = T; p.I = I; p.d = d;
     p.neuron_tiles = (I + TC_BM - 1) / TC_BM;
     p.token_tiles = (T + TC_BN - 1) / TC_BN;
+    p.band_tiles = calib_tc_band_tiles(T, I);
     p.bands = calib_tc_parts(T, I);
     p.items = p.neuron_tiles * p.bands;
     p.k_blocks = (d + TC_BK - 1) / TC_BK;

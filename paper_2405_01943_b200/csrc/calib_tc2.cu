@@ -22,7 +22,6 @@ constexpr int T2_BN = 256;          // tokens per tile (each CTA loads 128 of th
 constexpr int T2_BK = 64;
 constexpr int T2_UMMA_K = 16;
 constexpr int T2_STAGES = 4;
-constexpr int T2_BAND_TILES = 16;
 constexpr int T2_SUPER_BANDS = 16;
 constexpr unsigned long long T2_ALIGN_NS = 20000ull;
 constexpr int T2_THREADS = 192;
@@ -37,6 +36,7 @@ struct T2Params {
     int *align_counter;
     int64_t T, I, d;
     int64_t neuron_pairs, token_tiles, bands, items, k_blocks;   // items = neuron_pairs * bands (one per CTA pair)
+    int band_tiles;      // token tiles per band (calib_tc_band_tiles)
 };
 
 struct T2Item { int64_t np, band; };
@@ -109,15 +109,15 @@ calib_tc2_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
             int64_t round = 0;
             for (int64_t idx = cluster_id; idx < p.items && ok; idx += nclusters, ++round) {
                 const T2Item c = t2_decode(p, idx);
-                const int64_t tt0 = c.band * T2_BAND_TILES;
-                const int64_t tt1 = tt0 + T2_BAND_TILES < p.token_tiles ? tt0 + T2_BAND_TILES : p.token_tiles;
+                const int64_t tt0 = c.band * p.band_tiles;
+                const int64_t tt1 = tt0 + p.band_tiles < p.token_tiles ? tt0 + p.band_tiles : p.token_tiles;
                 const int64_t left = p.items - round * nclusters;
                 const int round_ctas = 2 * (int)(left < nclusters ? left : nclusters);
                 const int w_row = (int)(c.np * 2 * T2_BM + rank * T2_BM);
                 for (int64_t tt = tt0; tt < tt1 && ok; ++tt) {
                     {   // tile-boundary alignment of all CTAs of the round (bounded wait), see calib_tc.cu
                         const int t_in_item = (int)(tt - tt0);
-                        const int target = (int)(round * gridDim.x) * T2_BAND_TILES + round_ctas * (t_in_item + 1);
+                        const int target = (int)(round * gridDim.x) * p.band_tiles + round_ctas * (t_in_item + 1);
                         atomicAdd(p.align_counter, 1);
                         const unsigned long long t0 = global_ns();
                         while (*reinterpret_cast<volatile int *>(p.align_counter) < target && global_ns() - t0 < T2_ALIGN_NS) { }
@@ -134,7 +134,7 @@ calib_tc2_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                         if (++stage == T2_STAGES) { stage = 0; phase ^= 1u; }
                     }
                 }
-                if (tt1 - tt0 < T2_BAND_TILES) atomicAdd(p.align_counter, (int)(T2_BAND_TILES - (tt1 - tt0)));
+                if (tt1 - tt0 < p.band_tiles) atomicAdd(p.align_counter, (int)(p.band_tiles - (tt1 - tt0)));
             }
             if (!ok) { *abort_flag = 1; atomicExch(p.status, (int)DASS_ERR_TIMEOUT); }
         }
@@ -147,8 +147,8 @@ calib_tc2_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
             bool ok = true;
             for (int64_t idx = cluster_id; idx < p.items && ok; idx += nclusters) {
                 const T2Item c = t2_decode(p, idx);
-                const int64_t tt0 = c.band * T2_BAND_TILES;
-                const int64_t tt1 = tt0 + T2_BAND_TILES < p.token_tiles ? tt0 + T2_BAND_TILES : p.token_tiles;
+                const int64_t tt0 = c.band * p.band_tiles;
+                const int64_t tt1 = tt0 + p.band_tiles < p.token_tiles ? tt0 + p.band_tiles : p.token_tiles;
                 for (int64_t tt = tt0; tt < tt1 && ok; ++tt, ++tile) {
                     if (!mbar_wait(bar_acc_empty, (tile & 1u) ^ 1u, abort_flag)) { ok = false; break; }
                     tc_fence_after();
@@ -184,8 +184,8 @@ calib_tc2_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
         bool ok = true;
         for (int64_t idx = cluster_id; idx < p.items && ok; idx += nclusters) {
             const T2Item c = t2_decode(p, idx);
-            const int64_t tt0 = c.band * T2_BAND_TILES;
-            const int64_t tt1 = tt0 + T2_BAND_TILES < p.token_tiles ? tt0 + T2_BAND_TILES : p.token_tiles;
+            const int64_t tt0 = c.band * p.band_tiles;
+            const int64_t tt1 = tt0 + p.band_tiles < p.token_tiles ? tt0 + p.band_tiles : p.token_tiles;
             double acc = 0.0;
             for (int64_t tt = tt0; tt < tt1 && ok; ++tt, ++tile) {
                 if (!mbar_wait(bar_acc_full, tile & 1u, abort_flag)) { ok = false; break; }
@@ -233,6 +233,7 @@ calib_tc2_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
 // ------------------------------------------------------------------ host side
 bool tc_make_map(CUtensorMap *map, const void *ptr, int64_t rows, int64_t cols, int64_t ld, int box_rows);   // calib_tc.cu
 int64_t calib_tc_parts(int64_t T, int64_t I);                                                                 // calib_tc.cu
+int calib_tc_band_tiles(int64_t T, int64_t I);                                                                // calib_tc.cu
 int device_sm_count();                                                                                        // dass_abi.cu
 
 template <int ACT>
@@ -261,6 +262,7 @@ dass_status calib_tc2_launch(const void *X, int64_t T, int64_t ldx, const void *
     p.T = T; p.I = I; p.d = d;
     p.neuron_pairs = (I + 2 * T2_BM - 1) / (2 * T2_BM);
     p.token_tiles = (T + T2_BN - 1) / T2_BN;
+    p.band_tiles = calib_tc_band_tiles(T, I);
     p.bands = calib_tc_parts(T, I);
     p.items = p.neuron_pairs * p.bands;
     p.k_blocks = (d + T2_BK - 1) / T2_BK;
