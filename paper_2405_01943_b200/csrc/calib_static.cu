@@ -20,7 +20,7 @@ cudaError_t calib_simt_launch(const float *X, int64_t T, int64_t ldx, const floa
                               int64_t I, int64_t d, int64_t ldw, int act, double *partial, cudaStream_t st);
 cudaError_t calib_reduce_launch(const double *partial, int64_t parts, int64_t I, double *sumsq, cudaStream_t st);
 cudaError_t status_clear_launch(int *status, cudaStream_t st);
-int64_t calib_tc_parts(int64_t T, int64_t I);
+int64_t calib_tc_parts(int64_t T, int64_t I, int64_t d);
 dass_status calib_tc_launch(const void *X, int64_t T, int64_t ldx, const void *Wg, const void *Wu,
                             int64_t I, int64_t d, int64_t ldw, int act, double *partial, int *status,
                             cudaStream_t st);
@@ -82,7 +82,7 @@ extern "C" dass_status dass_calib_accumulate_static(const void *X, int64_t T, in
     if (status_clear_launch(status, st) != cudaSuccess) return DASS_ERR_CUDA;
     int64_t parts;
     if (bf16) {
-        parts = calib_tc_parts(T, I);
+        parts = calib_tc_parts(T, I, d);
         const dass_status ts = calib_tc_launch(X, T, ldx, Wg, Wu, I, d, ldw, (int)act, partial, status, st);
         if (ts != DASS_OK) return ts;
     } else {

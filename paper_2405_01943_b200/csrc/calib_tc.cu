@@ -32,7 +32,7 @@ constexpr int TC_BK = 64;          // k per ring slot: 64 bf16 = one 128-byte sw
 constexpr int TC_UMMA_K = 16;      // k per tcgen05.mma for 16-bit inputs
 constexpr int TC_STAGES = 3;
 constexpr int TC_MAX_BAND_TILES = 16;   // token tiles per band (one partial per band and neuron) at most
-constexpr int TC_SUPER_BANDS = 16;   // bands interleaved in the item order for L2 sharing
+constexpr int TC_SUPER_BANDS = 16;   // bands interleaved in the item order for L2 sharing, at most
 constexpr unsigned long long TC_ALIGN_NS = 20000ull;   // longest a CTA waits for the others at a tile boundary
 constexpr int TC_THREADS = 192;
 constexpr uint32_t TC_W_BYTES = TC_BM * TC_BK * 2;                 // 16 KB
@@ -48,20 +48,21 @@ struct TcParams {
     int64_t T, I, d;
     int64_t neuron_tiles, token_tiles, bands, items, k_blocks;
     int band_tiles;      // token tiles per band (calib_tc_band_tiles)
+    int super_bands;     // bands interleaved in the item order (calib_tc_super_bands)
 };
 
 struct ItemCoord { int64_t nt, band; };
 
 __device__ __forceinline__ ItemCoord decode_item(const TcParams &p, int64_t idx)
 {
-    const int64_t per_super = p.neuron_tiles * TC_SUPER_BANDS;
+    const int64_t per_super = p.neuron_tiles * p.super_bands;
     const int64_t sb = idx / per_super;
     const int64_t rem = idx - sb * per_super;
-    const int64_t left = p.bands - sb * TC_SUPER_BANDS;
-    const int64_t nb = left < TC_SUPER_BANDS ? left : TC_SUPER_BANDS;
+    const int64_t left = p.bands - sb * p.super_bands;
+    const int64_t nb = left < p.super_bands ? left : p.super_bands;
     ItemCoord c;
     c.nt = rem / nb;
-    c.band = sb * TC_SUPER_BANDS + (rem - c.nt * nb);
+    c.band = sb * p.super_bands + (rem - c.nt * nb);
     return c;
 }
 
@@ -276,30 +277,40 @@ bool tc_make_map(CUtensorMap *map, const void *ptr, int64_t rows, int64_t cols, 
 
 // Token tiles per band.  16 keeps a W tile in L2 for 16 token tiles; with few tokens that leaves the persistent
 // grid (148 CTAs, which this library is written for) with a part-filled last round, so a shorter band is taken
-// when it saves at least 1 % of the tile steps and the partial sums (one double per band and neuron) stay within
-// 14 MiB.  A function of (T, I) only: the workspace query, both tensor-core kernels and the scratch-free entry
-// point must agree on it.
-int calib_tc_band_tiles(int64_t T, int64_t I)
+// when it saves at least 1 % of the modelled time -- rounds x (band's k-blocks + a per-item cost of about 29
+// k-blocks: new W tiles and the re-alignment of the CTAs, fitted to measurements) -- and the partial sums (one
+// double per band and neuron) stay within 14 MiB.  A function of (T, I, d) only: the workspace query, both
+// tensor-core kernels and the scratch-free entry point must agree on it.
+int calib_tc_band_tiles(int64_t T, int64_t I, int64_t d)
 {
     const int64_t tiles = (I + TC_BM - 1) / TC_BM;
     const int64_t token_tiles = (T + TC_BN - 1) / TC_BN;
+    const int64_t k_blocks = (d + TC_BK - 1) / TC_BK;
     auto bands = [&](int bt) { return (token_tiles + bt - 1) / bt; };
-    auto steps = [&](int bt) { return ((tiles * bands(bt) + 147) / 148) * bt; };
+    auto cost = [&](int bt) { return ((tiles * bands(bt) + 147) / 148) * (bt * k_blocks + 29); };
     int best = TC_MAX_BAND_TILES;
-    int64_t best_steps = steps(best);
+    int64_t best_cost = cost(best);
     for (int bt = TC_MAX_BAND_TILES / 2; bt >= 1; bt >>= 1) {
-        const int64_t st = steps(bt);
         if (bands(bt) * I * (int64_t)sizeof(double) > ((int64_t)14 << 20)) break;
-        if (st * 100 < best_steps * 99) { best = bt; best_steps = st; }
+        const int64_t ct = cost(bt);
+        if (ct * 100 < best_cost * 99) { best = bt; best_cost = ct; }
     }
     return best;
 }
 
-int64_t calib_tc_parts(int64_t T, int64_t I)
+int64_t calib_tc_parts(int64_t T, int64_t I, int64_t d)
 {
     const int64_t token_tiles = (T + TC_BN - 1) / TC_BN;
-    const int bt = calib_tc_band_tiles(T, I);
+    const int bt = calib_tc_band_tiles(T, I, d);
     return (token_tiles + bt - 1) / bt;
+}
+
+// Bands interleaved in the item order: at most 16, and near-equal groups (25 bands run as 13 + 12, not 16 + 9:
+// a short last group would spread the CTAs over too many W tiles for L2).
+int calib_tc_super_bands(int64_t bands)
+{
+    const int64_t groups = (bands + TC_SUPER_BANDS - 1) / TC_SUPER_BANDS;
+    return (int)((bands + groups - 1) / groups);
 }
 
 int device_sm_count();   // dass_abi.cu
@@ -355,8 +366,9 @@ dass_status calib_tc_launch(const void *X, int64_t T, int64_t ldx, const void *W
     p.T = T; p.I = I; p.d = d;
     p.neuron_tiles = (I + TC_BM - 1) / TC_BM;
     p.token_tiles = (T + TC_BN - 1) / TC_BN;
-    p.band_tiles = calib_tc_band_tiles(T, I);
-    p.bands = calib_tc_parts(T, I);
+    p.band_tiles = calib_tc_band_tiles(T, I, d);
+    p.bands = calib_tc_parts(T, I, d);
+    p.super_bands = calib_tc_super_bands(p.bands);
     p.items = p.neuron_tiles * p.bands;
     p.k_blocks = (d + TC_BK - 1) / TC_BK;
     const int sms = device_sm_count();

@@ -22,7 +22,6 @@ constexpr int T2_BN = 256;          // tokens per tile (each CTA loads 128 of th
 constexpr int T2_BK = 64;
 constexpr int T2_UMMA_K = 16;
 constexpr int T2_STAGES = 4;
-constexpr int T2_SUPER_BANDS = 16;
 constexpr unsigned long long T2_ALIGN_NS = 20000ull;
 constexpr int T2_THREADS = 192;
 constexpr uint32_t T2_TILE_BYTES = 128 * T2_BK * 2;                 // 16 KB: a 128-row, 64-column bf16 tile
@@ -37,20 +36,21 @@ struct T2Params {
     int64_t T, I, d;
     int64_t neuron_pairs, token_tiles, bands, items, k_blocks;   // items = neuron_pairs * bands (one per CTA pair)
     int band_tiles;      // token tiles per band (calib_tc_band_tiles)
+    int super_bands;     // bands interleaved in the item order (calib_tc_super_bands)
 };
 
 struct T2Item { int64_t np, band; };
 
 __device__ __forceinline__ T2Item t2_decode(const T2Params &p, int64_t idx)
 {
-    const int64_t per_super = p.neuron_pairs * T2_SUPER_BANDS;
+    const int64_t per_super = p.neuron_pairs * p.super_bands;
     const int64_t sb = idx / per_super;
     const int64_t rem = idx - sb * per_super;
-    const int64_t left = p.bands - sb * T2_SUPER_BANDS;
-    const int64_t nb = left < T2_SUPER_BANDS ? left : T2_SUPER_BANDS;
+    const int64_t left = p.bands - sb * p.super_bands;
+    const int64_t nb = left < p.super_bands ? left : p.super_bands;
     T2Item c;
     c.np = rem / nb;
-    c.band = sb * T2_SUPER_BANDS + (rem - c.np * nb);
+    c.band = sb * p.super_bands + (rem - c.np * nb);
     return c;
 }
 
@@ -232,8 +232,9 @@ calib_tc2_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
 
 // ------------------------------------------------------------------ host side
 bool tc_make_map(CUtensorMap *map, const void *ptr, int64_t rows, int64_t cols, int64_t ld, int box_rows);   // calib_tc.cu
-int64_t calib_tc_parts(int64_t T, int64_t I);                                                                 // calib_tc.cu
-int calib_tc_band_tiles(int64_t T, int64_t I);                                                                // calib_tc.cu
+int64_t calib_tc_parts(int64_t T, int64_t I, int64_t d);                                                      // calib_tc.cu
+int calib_tc_band_tiles(int64_t T, int64_t I, int64_t d);                                                     // calib_tc.cu
+int calib_tc_super_bands(int64_t bands);                                                                      // calib_tc.cu
 int device_sm_count();                                                                                        // dass_abi.cu
 
 template <int ACT>
@@ -262,8 +263,9 @@ dass_status calib_tc2_launch(const void *X, int64_t T, int64_t ldx, const void *
     p.T = T; p.I = I; p.d = d;
     p.neuron_pairs = (I + 2 * T2_BM - 1) / (2 * T2_BM);
     p.token_tiles = (T + T2_BN - 1) / T2_BN;
-    p.band_tiles = calib_tc_band_tiles(T, I);
-    p.bands = calib_tc_parts(T, I);
+    p.band_tiles = calib_tc_band_tiles(T, I, d);
+    p.bands = calib_tc_parts(T, I, d);
+    p.super_bands = calib_tc_super_bands(p.bands);
     p.items = p.neuron_pairs * p.bands;
     p.k_blocks = (d + T2_BK - 1) / T2_BK;
     const int64_t max_pairs = device_sm_count() / 2;

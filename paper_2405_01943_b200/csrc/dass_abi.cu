@@ -19,7 +19,7 @@ cudaError_t calib_simt_launch(const float *X, int64_t T, int64_t ldx, const floa
 cudaError_t calib_reduce_launch(const double *partial, int64_t parts, int64_t I, double *sumsq, cudaStream_t st);
 cudaError_t norm_finalize_launch(const double *sumsq, int64_t I, float *norm, cudaStream_t st);
 cudaError_t status_clear_launch(int *status, cudaStream_t st);
-int64_t calib_tc_parts(int64_t T, int64_t I);
+int64_t calib_tc_parts(int64_t T, int64_t I, int64_t d);
 dass_status calib_tc_launch(const void *X, int64_t T, int64_t ldx, const void *Wg, const void *Wu,
                             int64_t I, int64_t d, int64_t ldw, int act, double *partial, int *status,
                             cudaStream_t st);
@@ -87,7 +87,7 @@ dass_status dass_calib_workspace_bytes(int64_t T, int64_t d, int64_t I, dass_dty
     if (!bytes) return DASS_ERR_NULL;
     if (dt != DASS_BF16 && dt != DASS_F32) return DASS_ERR_DTYPE;
     if (T < 1 || d < 1 || I < 1) return DASS_ERR_SHAPE;
-    const int64_t parts = dt == DASS_BF16 ? calib_tc_parts(T, I) : calib_simt_parts(T);
+    const int64_t parts = dt == DASS_BF16 ? calib_tc_parts(T, I, d) : calib_simt_parts(T);
     *bytes = WS_HEADER + (size_t)parts * (size_t)I * sizeof(double);
     return DASS_OK;
 }
@@ -116,7 +116,7 @@ dass_status dass_calib_accumulate(const void *X, int64_t T, int64_t ldx,
     if (status_clear_launch(status, st) != cudaSuccess) return DASS_ERR_CUDA;
     int64_t parts;
     if (bf16) {
-        parts = calib_tc_parts(T, I);
+        parts = calib_tc_parts(T, I, d);
         const dass_status ts = calib_tc_launch(X, T, ldx, Wg, Wu, I, d, ldw, (int)act, partial, status, st);
         if (ts != DASS_OK) return ts;
     } else {
