@@ -51,6 +51,25 @@ def test_workspace_query_validation(lib):
     assert out.value < (1 << 30)
 
 
+def test_calib_workspace_of_short_batches_stays_within_the_static_scratch(lib):
+    """The band length of the tensor-core calibration depends on (T, I, d): shorter bands for short batches mean
+    more partial sums.  Whatever it picks, a problem that bands of 16 token tiles (256 tokens each) would have kept
+    within the fixed scratch of dass_calib_accumulate_static must still fit there, the full-size call keeps bands
+    of 16, and no choice needs more partial rows than one per token tile."""
+    limit = 16 << 20
+    out = ctypes.c_size_t(0)
+    for d, I in ((4096, 11008), (5120, 13824), (4096, 14336), (3072, 24576), (8192, 28672), (256, 688), (8192, 57344)):
+        for T in (1, 255, 256, 2048, 8192, 16384, 32768, 65536, 98304, 100000, 131072, 262144, 300000):
+            assert lib.dass_calib_workspace_bytes(T, d, I, binding.BF16, ctypes.byref(out)) == 0
+            token_tiles = -(-T // 256)
+            with_16 = 256 + (-(-token_tiles // 16)) * I * 8
+            assert with_16 <= out.value <= 256 + token_tiles * I * 8
+            if with_16 <= limit:
+                assert out.value <= limit, (T, d, I, out.value)
+    assert lib.dass_calib_workspace_bytes(262144, 8192, 28672, binding.BF16, ctypes.byref(out)) == 0
+    assert out.value == 256 + 64 * 28672 * 8
+
+
 FAKE = 0x10000  # a 16-byte aligned non-NULL address; validation must fail before it is ever dereferenced
 
 
