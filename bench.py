@@ -284,6 +284,7 @@ def run_ours(args):
                                    f"{cfg.n_keep}:{cfg.m} on gate/up (Eq. 4, alpha={alpha}, input-balanced) and down (Eq. 5); "
                                    "mask + pruned weights + compressed values/metadata",
                        "layers_per_rank": args.steps, "weight_sets_cycled": len(pool),
+                       "input_checksums": {n: synth.checksum(t) for n, t in zip(("X", "Wg", "Wu", "Wd"), (X,) + tuple(pool[0]))},
                        "l2": "inputs exceed L2 (X and each weight set are far larger than 126 MB); no flush",
                        "parallelism": "independent layers per GPU, no collective" if world > 1 else "single GPU"},
             "stage_ms": {"calib": calib_ms, "score_x3": score_ms, "compress_x3": comp_ms},

@@ -143,9 +143,14 @@ def make_weights(cfg: LayerConfig, device="cpu", layer: int = 0):
     return wg, wu, wd
 
 
-def checksum(t: torch.Tensor) -> int:
-    """Order-dependent 64-bit checksum of a tensor's raw bytes (for run-to-run comparison)."""
-    raw = t.contiguous().view(torch.uint8).to(torch.int64)
+def checksum(t: torch.Tensor, chunk: int = 1 << 26) -> int:
+    """Order-dependent 64-bit checksum of a tensor's raw bytes (for run-to-run comparison):
+    sum of byte[i] * (i % 65521 + 1) modulo 2^64, evaluated in chunks so that large tensors need little scratch."""
+    raw = t.contiguous().view(-1).view(torch.uint8)
     n = raw.numel()
-    weights = (torch.arange(n, device=raw.device, dtype=torch.int64) % 65521) + 1
-    return int((raw * weights).sum().item() & 0xFFFFFFFFFFFFFFFF)
+    total = 0
+    for lo in range(0, n, chunk):
+        hi = min(n, lo + chunk)
+        weights = (torch.arange(lo, hi, device=raw.device, dtype=torch.int64) % 65521) + 1
+        total = (total + int((raw[lo:hi].to(torch.int64) * weights).sum().item())) & 0xFFFFFFFFFFFFFFFF
+    return total
