@@ -35,7 +35,7 @@ struct ScoreFastParams {
 };
 
 constexpr int F_THREADS = 256;
-constexpr int F_MIN_BLOCKS = 4;      // CTAs per SM the 2:4 kernels are compiled for (64 registers: measured best)
+constexpr int F_MIN_BLOCKS = 4;      // CTAs per SM the 2:4 row-group kernel is compiled for (64 registers: measured best)
 constexpr int F_COLS = 256;          // columns per warp strip
 // prefetch depth of the shared-memory slab ring (slabs of R rows x 512 bytes per warp)
 __host__ __device__ constexpr int ring_stages(int rows_per_unit) { return rows_per_unit >= 8 ? 2 : 3; }
@@ -358,8 +358,9 @@ __global__ void __launch_bounds__(F_THREADS, M == 8 ? 2 : F_MIN_BLOCKS) score_ro
 }
 
 // ---------------------------------------------------------------- groups along the columns (down)
+// 3 CTAs per SM (85 registers): with 4 the 2:4 kernel spills a few words and runs 4 % slower
 template <int M, bool NORM_COLS>
-__global__ void __launch_bounds__(F_THREADS, M == 8 ? 3 : F_MIN_BLOCKS) score_cols_bf16_kernel(const ScoreFastParams p)
+__global__ void __launch_bounds__(F_THREADS, 3) score_cols_bf16_kernel(const ScoreFastParams p)
 {
     constexpr int G = 8 / M;             // groups inside a lane's 8 columns
     constexpr int STAGES = ring_stages(F_SLAB);
