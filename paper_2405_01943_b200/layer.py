@@ -42,6 +42,7 @@ class LayerPruner:
             self.out[name] = o
         self.compressed = compressed
         self._select_ws: Optional[Dict[str, torch.Tensor]] = None
+        self._forward_ws: Optional[torch.Tensor] = None
 
     # ------------------------------------------------------------------ stage (a)
     def reset(self) -> None:
@@ -98,3 +99,17 @@ class LayerPruner:
         else:
             self.select_unstructured(Wg, Wu, Wd, sparsity, alpha)
         return self.out
+
+    # ------------------------------------------------------------------ the pruned layer's output
+    def forward_pruned(self, X: torch.Tensor, Z: Optional[torch.Tensor] = None,
+                       workspace_bytes: Optional[int] = None) -> torch.Tensor:
+        """Z = (act(X Wg'^T) * (X Wu'^T)) Wd'^T (Eq. 2 then Eq. 3) with the pruned copies the last prune() /
+        score_nm() / select_unstructured() wrote, e.g. to feed the next layer's calibration.  `workspace_bytes`
+        bounds the scratch that holds the intermediate activations (default: all tokens in one pass)."""
+        T = X.shape[0]
+        lo, full = b.mlp_forward_workspace_bytes(T, self.d, self.I, self.dtype)
+        nbytes = full if workspace_bytes is None else max(lo, min(full, int(workspace_bytes)))
+        if self._forward_ws is None or self._forward_ws.numel() != nbytes:
+            self._forward_ws = b.mlp_forward_workspace(nbytes, self.device)
+        return b.mlp_forward(X, self.out["gate"]["pruned"], self.out["up"]["pruned"], self.out["down"]["pruned"],
+                             self.act, Z=Z, workspace=self._forward_ws)

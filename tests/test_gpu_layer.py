@@ -58,3 +58,21 @@ def test_prune_unstructured_and_batched_calibration():
     pruner.finalize()
     pruner.check()
     assert np.max(np.abs(to_np32(pruner.norm) - norm_one_call) / norm_one_call) <= 1e-6
+
+
+def test_forward_of_the_pruned_layer_matches_oracle_forward_of_the_same_weights():
+    """prune() then forward_pruned(): the oracle's forward pass of the very weights the GPU pruned (bf16 rounding
+    of the intermediate on both sides), in one pass and in token chunks."""
+    cfg, X, Wg, Wu, Wd = _layer("llama2_7b", d=256, I=688, T=700)
+    pruner = LayerPruner(cfg.T, cfg.d, cfg.I, X.dtype, act=cfg.act, device=DEV, compressed=False)
+    out = pruner.prune(X, Wg, Wu, Wd, alpha=0.5)
+    Z = pruner.forward_pruned(X)
+    pruner.check()
+    Zc = pruner.forward_pruned(X, workspace_bytes=1)            # smallest workspace: 256-token chunks
+    assert np.array_equal(bits_of(Z), bits_of(Zc))
+    Z_ref, _ = oracle.mlp_forward(to_np32(X), to_np32(out["gate"]["pruned"]), to_np32(out["up"]["pruned"]),
+                                  to_np32(out["down"]["pruned"]), ORACLE_ACT[cfg.act], True, want_h=True)
+    z = to_np32(Z).astype(np.float64)
+    err = np.sqrt(np.mean((z - Z_ref) ** 2)) / (np.sqrt(np.mean(Z_ref ** 2)) + 1e-30)
+    assert err <= 6e-3                                          # the bound test_gpu_forward.py derives for bf16
+    assert float((out["gate"]["pruned"] == 0).float().mean()) >= 0.5
