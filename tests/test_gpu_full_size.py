@@ -129,3 +129,27 @@ def test_70b_stream_other_layers_sampled_neurons(layer_id):
         oracle.calib_sumsq(to_np32(X[t0:t0 + 32768]), wg, wu, ORACLE_ACT[cfg.act], ref)
     rel = np.abs(np.sqrt(got[idx]) - np.sqrt(ref)) / np.sqrt(ref)
     assert rel.max() <= 2e-3, f"layer {layer_id}: sampled-neuron norm error {rel.max():.3e}"
+
+
+@pytest.mark.parametrize("name,T", [("llama2_70b", 32768), ("llama2_7b", 8192 + 300), ("gemma_7b", 16384), ("llama2_13b", 2048)])
+def test_stage_a_short_batches_sampled_neurons(name, T):
+    """Short calibration batches of the full-width layers: the tensor-core kernels pick shorter bands of token tiles
+    for them (other item counts, other partial-sum layouts than the full 262144-token call), and two such batches
+    accumulate.  Sampled neurons over all tokens against the oracle."""
+    cfg = synth.scaled(synth.CONFIGS[name], T=T)
+    X = synth.make_x(cfg, DEV)
+    Wg, Wu, _ = synth.make_weights(cfg, DEV)
+    sumsq = torch.zeros(cfg.I, dtype=torch.float64, device=DEV)
+    ws = binding.calib_workspace(T, cfg.d, cfg.I, X.dtype, DEV)
+    act = binding.ACT_BY_NAME[cfg.act]
+    binding.calib_accumulate(X, Wg, Wu, act, sumsq, ws)
+    once = sumsq.clone()
+    binding.calib_accumulate(X, Wg, Wu, act, sumsq, ws)            # a second batch (the same tokens) adds the same sums
+    binding.calib_status(ws)
+    got = once.cpu().numpy()
+    assert np.array_equal(sumsq.cpu().numpy(), 2.0 * got)          # doubling is exact: the kernel is deterministic
+    idx = np.unique(np.concatenate([np.argsort(-got)[:8], np.linspace(0, cfg.I - 1, 24).astype(np.int64)]))
+    sel = torch.from_numpy(idx).to(DEV)
+    ref = oracle.calib_sumsq(to_np32(X), to_np32(Wg[sel]), to_np32(Wu[sel]), ORACLE_ACT[cfg.act])
+    rel = np.abs(np.sqrt(got[idx]) - np.sqrt(ref)) / np.sqrt(ref)
+    assert rel.max() <= 2e-3, f"{name} T={T}: sampled-neuron norm error {rel.max():.3e}"
