@@ -58,6 +58,22 @@ def test_random_shapes_bit_exact(dtype, n_keep, m, norm_axis, group_axis):
                 assert np.all(mk.reshape(rows // m, m, cols).sum(1) == n_keep)
 
 
+@pytest.mark.parametrize("n_keep", [1, 2, 3])
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32], ids=["bf16", "f32"])
+def test_row_groups_of_four_with_an_odd_number_of_groups(dtype, n_keep):
+    """Row counts that are a multiple of 4 but not of 8 (the row-group kernels take 8 rows at a time, so the last
+    group of 4 stands alone), down to a single group, with ragged column counts."""
+    gen = torch.Generator(device=DEV)
+    gen.manual_seed(4242 + n_keep)
+    for rows, cols, ld in [(4, 8, 8), (12, 40, 40), (44, 344, 352), (36, 1032, 1040), (100, 24, 24)]:
+        for ties in (False, True):
+            base, W = _padded(rows, cols, ld, dtype, gen, ties=ties)
+            norm = _norm(rows, gen, ties=ties)
+            ref = oracle_stage_b(W, to_np32(norm), AXIS_ROWS, 0.5, n_keep, 4, AXIS_ROWS)
+            assert_stage_b_equal(gpu_stage_b(W, norm, AXIS_ROWS, 0.5, n_keep, 4, AXIS_ROWS), ref)
+            assert torch.all(base[:, cols:] == 7.0)                # the padding of the input is never touched
+
+
 def test_generic_alpha_uses_pow():
     gen = torch.Generator(device=DEV)
     gen.manual_seed(5)
