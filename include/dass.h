@@ -68,11 +68,12 @@ typedef enum { DASS_AXIS_ROWS = 0, DASS_AXIS_COLS = 1 } dass_axis;
  * sumsq [I] doubles, in/out: the call ADDS this batch's contribution, so a
  * calibration set may be fed in any number of batches; the caller zeroes it
  * before the first batch.  The per-batch contribution is reduced in a fixed
- * order, so equal inputs give bit-equal results.
- * workspace: scratch of at least dass_calib_workspace_bytes(...) bytes, 256-byte
- * aligned, contents irrelevant on entry; it must not be shared by calls that
- * may overlap on the device.  Its first word receives a device status that
- * dass_calib_status reads.
+ * order, so equal inputs (and an equal workspace size) give bit-equal results.
+ * workspace: scratch of dass_calib_workspace_bytes(...) bytes, 256-byte aligned,
+ * contents irrelevant on entry; it must not be shared by calls that may overlap
+ * on the device.  A workspace sized by the query for T tokens also serves every
+ * call with fewer tokens (the call then uses coarser partial sums if it has to).
+ * Its first word receives a device status that dass_calib_status reads.
  * Errors: NULL / SHAPE (T, d, I < 1) / ALIGN / DTYPE / WORKSPACE / CUDA. */
 dass_status dass_calib_workspace_bytes(int64_t T, int64_t d, int64_t I, dass_dtype dt, size_t *bytes /* HOST */);
 dass_status dass_calib_accumulate(const void *X, int64_t T, int64_t ldx,
@@ -102,9 +103,9 @@ dass_status dass_selftest_wait_timeout(void *status_word, int64_t limit_us, void
  * fixed reduction order, same arguments and error codes), but its scratch is a fixed array of
  * DASS_STATIC_SCRATCH_BYTES inside the library's device image, which every GPU that loads the library
  * holds until the process exits.  It calls no cudaMalloc / cudaFree and no allocating routine.
- *  - Limit: a problem whose dass_calib_workspace_bytes(T, d, I, dt) exceeds DASS_STATIC_SCRATCH_BYTES is
- *    refused with DASS_ERR_WORKSPACE and nothing is touched (16 MiB covers a 28672-neuron bf16 layer
- *    at 262144 tokens per call; feed larger token counts in several calls).
+ *  - Limit: a problem whose partial sums do not fit into DASS_STATIC_SCRATCH_BYTES even at their coarsest (bf16:
+ *    one double per neuron and 4096 tokens) is refused with DASS_ERR_WORKSPACE and nothing is touched (16 MiB
+ *    covers a 28672-neuron bf16 layer at 262144 tokens per call; feed larger token counts in several calls).
  *  - The first call on each device (made with that device current) looks up the scratch's device
  *    address once; make that first call before any stream capture begins.
  *  - All calls on a device share the one array, which keeps the previous call's contents; the call

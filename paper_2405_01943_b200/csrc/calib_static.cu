@@ -20,9 +20,10 @@ cudaError_t calib_simt_launch(const float *X, int64_t T, int64_t ldx, const floa
                               int64_t I, int64_t d, int64_t ldw, int act, double *partial, cudaStream_t st);
 cudaError_t calib_reduce_launch(const double *partial, int64_t parts, int64_t I, double *sumsq, cudaStream_t st);
 cudaError_t status_clear_launch(int *status, cudaStream_t st);
-int64_t calib_tc_parts(int64_t T, int64_t I, int64_t d);
+int calib_tc_band_tiles(int64_t T, int64_t I, int64_t d, int64_t partial_budget_bytes);
+int64_t calib_tc_parts_for(int64_t T, int band_tiles);
 dass_status calib_tc_launch(const void *X, int64_t T, int64_t ldx, const void *Wg, const void *Wu,
-                            int64_t I, int64_t d, int64_t ldw, int act, double *partial, int *status,
+                            int64_t I, int64_t d, int64_t ldw, int act, int band_tiles, double *partial, int *status,
                             cudaStream_t st);
 
 // Held by every GPU that loads this library, until the process exits.
@@ -65,9 +66,9 @@ extern "C" dass_status dass_calib_accumulate_static(const void *X, int64_t T, in
         (reinterpret_cast<uintptr_t>(Wu) & 15u) || ldx % ldmul || ldw % ldmul ||
         (reinterpret_cast<uintptr_t>(sumsq) & 7u))
         return DASS_ERR_ALIGN;
-    size_t need = 0;
-    const dass_status qs = dass_calib_workspace_bytes(T, d, I, dt, &need);
-    if (qs != DASS_OK) return qs;
+    // room for the status header and the partial sums of bands of 16 token tiles (bf16) is the least the call needs
+    const int64_t parts_min = bf16 ? calib_tc_parts_for(T, 16) : calib_simt_parts(T);
+    const size_t need = 256 + (size_t)parts_min * (size_t)I * sizeof(double);
     if (need > (size_t)DASS_STATIC_SCRATCH_BYTES) return DASS_ERR_WORKSPACE;   // too large for the fixed scratch
 
     void *scratch = nullptr;
@@ -82,8 +83,9 @@ extern "C" dass_status dass_calib_accumulate_static(const void *X, int64_t T, in
     if (status_clear_launch(status, st) != cudaSuccess) return DASS_ERR_CUDA;
     int64_t parts;
     if (bf16) {
-        parts = calib_tc_parts(T, I, d);
-        const dass_status ts = calib_tc_launch(X, T, ldx, Wg, Wu, I, d, ldw, (int)act, partial, status, st);
+        const int band_tiles = calib_tc_band_tiles(T, I, d, (int64_t)DASS_STATIC_SCRATCH_BYTES - 256);
+        parts = calib_tc_parts_for(T, band_tiles);
+        const dass_status ts = calib_tc_launch(X, T, ldx, Wg, Wu, I, d, ldw, (int)act, band_tiles, partial, status, st);
         if (ts != DASS_OK) return ts;
     } else {
         parts = calib_simt_parts(T);

@@ -279,9 +279,10 @@ bool tc_make_map(CUtensorMap *map, const void *ptr, int64_t rows, int64_t cols, 
 // grid (148 CTAs, which this library is written for) with a part-filled last round, so a shorter band is taken
 // when it saves at least 1 % of the modelled time -- rounds x (band's k-blocks + a per-item cost of about 29
 // k-blocks: new W tiles and the re-alignment of the CTAs, fitted to measurements) -- and the partial sums (one
-// double per band and neuron) stay within 14 MiB.  A function of (T, I, d) only: the workspace query, both
-// tensor-core kernels and the scratch-free entry point must agree on it.
-int calib_tc_band_tiles(int64_t T, int64_t I, int64_t d)
+// double per band and neuron) stay within 14 MiB and within `partial_budget_bytes`, what the caller's scratch has
+// room for.  Bands of 16 are the fallback, so a scratch sized by the query for some token count also serves every
+// shorter batch.  The entry points choose the band length and hand it to the launchers and to the reduction.
+int calib_tc_band_tiles(int64_t T, int64_t I, int64_t d, int64_t partial_budget_bytes)
 {
     const int64_t tiles = (I + TC_BM - 1) / TC_BM;
     const int64_t token_tiles = (T + TC_BN - 1) / TC_BN;
@@ -291,18 +292,25 @@ int calib_tc_band_tiles(int64_t T, int64_t I, int64_t d)
     int best = TC_MAX_BAND_TILES;
     int64_t best_cost = cost(best);
     for (int bt = TC_MAX_BAND_TILES / 2; bt >= 1; bt >>= 1) {
-        if (bands(bt) * I * (int64_t)sizeof(double) > ((int64_t)14 << 20)) break;
+        const int64_t bytes = bands(bt) * I * (int64_t)sizeof(double);
+        if (bytes > ((int64_t)14 << 20) || bytes > partial_budget_bytes) break;
         const int64_t ct = cost(bt);
         if (ct * 100 < best_cost * 99) { best = bt; best_cost = ct; }
     }
     return best;
 }
 
-int64_t calib_tc_parts(int64_t T, int64_t I, int64_t d)
+// Partial sums per neuron (= bands) for a band length.
+int64_t calib_tc_parts_for(int64_t T, int band_tiles)
 {
     const int64_t token_tiles = (T + TC_BN - 1) / TC_BN;
-    const int bt = calib_tc_band_tiles(T, I, d);
-    return (token_tiles + bt - 1) / bt;
+    return (token_tiles + band_tiles - 1) / band_tiles;
+}
+
+// The workspace query's answer: the preferred band length with no limit from the caller.
+int64_t calib_tc_parts(int64_t T, int64_t I, int64_t d)
+{
+    return calib_tc_parts_for(T, calib_tc_band_tiles(T, I, d, INT64_MAX));
 }
 
 // Bands interleaved in the item order: at most 16, and near-equal groups (25 bands run as 13 + 12, not 16 + 9:
@@ -349,14 +357,16 @@ cudaError_t bounded_wait_selftest_launch(int *status, unsigned long long limit_n
 
 constexpr bool TC_USE_PAIR_KERNEL = true;   // layers with more than one neuron tile take the CTA-pair kernel (calib_tc2.cu)
 dass_status calib_tc2_launch(const void *X, int64_t T, int64_t ldx, const void *Wg, const void *Wu,
-                             int64_t I, int64_t d, int64_t ldw, int act, double *partial, int *status,
+                             int64_t I, int64_t d, int64_t ldw, int act, int band_tiles, double *partial, int *status,
                              cudaStream_t st);   // calib_tc2.cu
 
 dass_status calib_tc_launch(const void *X, int64_t T, int64_t ldx, const void *Wg, const void *Wu,
-                            int64_t I, int64_t d, int64_t ldw, int act, double *partial, int *status,
+                            int64_t I, int64_t d, int64_t ldw, int act, int band_tiles, double *partial, int *status,
                             cudaStream_t st)
 {
-    if (TC_USE_PAIR_KERNEL && I > TC_BM) return calib_tc2_launch(X, T, ldx, Wg, Wu, I, d, ldw, act, partial, status, st);
+    if (band_tiles < 1 || band_tiles > TC_MAX_BAND_TILES) return DASS_ERR_UNSUPPORTED;
+    if (TC_USE_PAIR_KERNEL && I > TC_BM)
+        return calib_tc2_launch(X, T, ldx, Wg, Wu, I, d, ldw, act, band_tiles, partial, status, st);
     if (d > 0x7fffffffll - TC_BK || T > 0x7fffffffll - TC_BN || I > 0x7fffffffll - TC_BM) return DASS_ERR_UNSUPPORTED;
     CUtensorMap mx, mg, mu;
     if (!tc_make_map(&mx, X, T, d, ldx, TC_BN) || !tc_make_map(&mg, Wg, I, d, ldw, TC_BM) || !tc_make_map(&mu, Wu, I, d, ldw, TC_BM))
@@ -366,8 +376,8 @@ dass_status calib_tc_launch(const void *X, int64_t T, int64_t ldx, const void *W
     p.T = T; p.I = I; p.d = d;
     p.neuron_tiles = (I + TC_BM - 1) / TC_BM;
     p.token_tiles = (T + TC_BN - 1) / TC_BN;
-    p.band_tiles = calib_tc_band_tiles(T, I, d);
-    p.bands = calib_tc_parts(T, I, d);
+    p.band_tiles = band_tiles;
+    p.bands = calib_tc_parts_for(T, band_tiles);
     p.super_bands = calib_tc_super_bands(p.bands);
     p.items = p.neuron_tiles * p.bands;
     p.k_blocks = (d + TC_BK - 1) / TC_BK;

@@ -232,8 +232,7 @@ calib_tc2_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
 
 // ------------------------------------------------------------------ host side
 bool tc_make_map(CUtensorMap *map, const void *ptr, int64_t rows, int64_t cols, int64_t ld, int box_rows);   // calib_tc.cu
-int64_t calib_tc_parts(int64_t T, int64_t I, int64_t d);                                                      // calib_tc.cu
-int calib_tc_band_tiles(int64_t T, int64_t I, int64_t d);                                                     // calib_tc.cu
+int64_t calib_tc_parts_for(int64_t T, int band_tiles);                                                        // calib_tc.cu
 int calib_tc_super_bands(int64_t bands);                                                                      // calib_tc.cu
 int device_sm_count();                                                                                        // dass_abi.cu
 
@@ -250,7 +249,7 @@ static cudaError_t launch_tc2(const CUtensorMap &mx, const CUtensorMap &mg, cons
 
 // CTA-pair launch; same contract as calib_tc_launch (partials per band, status word, alignment counter behind it).
 dass_status calib_tc2_launch(const void *X, int64_t T, int64_t ldx, const void *Wg, const void *Wu,
-                             int64_t I, int64_t d, int64_t ldw, int act, double *partial, int *status,
+                             int64_t I, int64_t d, int64_t ldw, int act, int band_tiles, double *partial, int *status,
                              cudaStream_t st)
 {
     if (d > 0x7fffffffll - T2_BK || T > 0x7fffffffll - T2_BN || I > 0x7fffffffll - 2 * T2_BM) return DASS_ERR_UNSUPPORTED;
@@ -263,8 +262,8 @@ dass_status calib_tc2_launch(const void *X, int64_t T, int64_t ldx, const void *
     p.T = T; p.I = I; p.d = d;
     p.neuron_pairs = (I + 2 * T2_BM - 1) / (2 * T2_BM);
     p.token_tiles = (T + T2_BN - 1) / T2_BN;
-    p.band_tiles = calib_tc_band_tiles(T, I, d);
-    p.bands = calib_tc_parts(T, I, d);
+    p.band_tiles = band_tiles;
+    p.bands = calib_tc_parts_for(T, band_tiles);
     p.super_bands = calib_tc_super_bands(p.bands);
     p.items = p.neuron_pairs * p.bands;
     p.k_blocks = (d + T2_BK - 1) / T2_BK;

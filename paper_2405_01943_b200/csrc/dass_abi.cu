@@ -20,8 +20,10 @@ cudaError_t calib_reduce_launch(const double *partial, int64_t parts, int64_t I,
 cudaError_t norm_finalize_launch(const double *sumsq, int64_t I, float *norm, cudaStream_t st);
 cudaError_t status_clear_launch(int *status, cudaStream_t st);
 int64_t calib_tc_parts(int64_t T, int64_t I, int64_t d);
+int calib_tc_band_tiles(int64_t T, int64_t I, int64_t d, int64_t partial_budget_bytes);
+int64_t calib_tc_parts_for(int64_t T, int band_tiles);
 dass_status calib_tc_launch(const void *X, int64_t T, int64_t ldx, const void *Wg, const void *Wu,
-                            int64_t I, int64_t d, int64_t ldw, int act, double *partial, int *status,
+                            int64_t I, int64_t d, int64_t ldw, int act, int band_tiles, double *partial, int *status,
                             cudaStream_t st);
 
 cudaError_t bounded_wait_selftest_launch(int *status, unsigned long long limit_ns, cudaStream_t st);
@@ -104,9 +106,10 @@ dass_status dass_calib_accumulate(const void *X, int64_t T, int64_t ldx,
     const bool bf16 = dt == DASS_BF16;
     if (!aligned16(X) || !aligned16(Wg) || !aligned16(Wu) || !ld_ok(ldx, bf16) || !ld_ok(ldw, bf16)) return DASS_ERR_ALIGN;
     if ((reinterpret_cast<uintptr_t>(sumsq) & 7u) != 0) return DASS_ERR_ALIGN;
-    size_t need = 0;
-    const dass_status qs = dass_calib_workspace_bytes(T, d, I, dt, &need);
-    if (qs != DASS_OK) return qs;
+    // The query's size is what the call would like; what it needs is room for bands of 16 token tiles (bf16), so
+    // a workspace sized by the query for some token count also serves every shorter batch.
+    const int64_t parts_min = bf16 ? calib_tc_parts_for(T, 16) : calib_simt_parts(T);
+    const size_t need = WS_HEADER + (size_t)parts_min * (size_t)I * sizeof(double);
     if (!workspace || workspace_bytes < need) return DASS_ERR_WORKSPACE;
     if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return DASS_ERR_ALIGN;
 
@@ -116,8 +119,9 @@ dass_status dass_calib_accumulate(const void *X, int64_t T, int64_t ldx,
     if (status_clear_launch(status, st) != cudaSuccess) return DASS_ERR_CUDA;
     int64_t parts;
     if (bf16) {
-        parts = calib_tc_parts(T, I, d);
-        const dass_status ts = calib_tc_launch(X, T, ldx, Wg, Wu, I, d, ldw, (int)act, partial, status, st);
+        const int band_tiles = calib_tc_band_tiles(T, I, d, (int64_t)(workspace_bytes - WS_HEADER));
+        parts = calib_tc_parts_for(T, band_tiles);
+        const dass_status ts = calib_tc_launch(X, T, ldx, Wg, Wu, I, d, ldw, (int)act, band_tiles, partial, status, st);
         if (ts != DASS_OK) return ts;
     } else {
         parts = calib_simt_parts(T);

@@ -153,3 +153,26 @@ def test_stage_a_short_batches_sampled_neurons(name, T):
     ref = oracle.calib_sumsq(to_np32(X), to_np32(Wg[sel]), to_np32(Wu[sel]), ORACLE_ACT[cfg.act])
     rel = np.abs(np.sqrt(got[idx]) - np.sqrt(ref)) / np.sqrt(ref)
     assert rel.max() <= 2e-3, f"{name} T={T}: sampled-neuron norm error {rel.max():.3e}"
+
+
+def test_workspace_sized_for_more_tokens_serves_shorter_batches():
+    """A workspace obtained for a long batch is accepted for shorter ones even where the short batch alone would have
+    asked for more room (finer partial sums): the call then falls back to coarser bands; results agree to rounding."""
+    cfg = synth.scaled(synth.CONFIGS["llama2_70b"], T=65536)
+    X = synth.make_x(cfg, DEV)
+    Wg, Wu, _ = synth.make_weights(cfg, DEV)
+    act = binding.ACT_BY_NAME[cfg.act]
+    big = binding.calib_workspace_bytes(cfg.T, cfg.d, cfg.I, X.dtype)
+    sizes = {T: binding.calib_workspace_bytes(T, cfg.d, cfg.I, X.dtype) for T in (49152, 32768, 300)}
+    assert max(sizes.values()) > big                      # the case this test is about exists at these shapes
+    ws_big = binding.calib_workspace(cfg.T, cfg.d, cfg.I, X.dtype, DEV)
+    for T in sizes:
+        a = torch.zeros(cfg.I, dtype=torch.float64, device=DEV)
+        b_ = torch.zeros(cfg.I, dtype=torch.float64, device=DEV)
+        binding.calib_accumulate(X[:T], Wg, Wu, act, a, ws_big)
+        binding.calib_status(ws_big)
+        ws_own = binding.calib_workspace(T, cfg.d, cfg.I, X.dtype, DEV)
+        binding.calib_accumulate(X[:T], Wg, Wu, act, b_, ws_own)
+        binding.calib_status(ws_own)
+        a, b_ = a.cpu().numpy(), b_.cpu().numpy()
+        assert np.all(a > 0) and np.max(np.abs(a - b_) / b_) <= 1e-12
