@@ -138,8 +138,8 @@ dass_status dass_norm_finalize(const double *sumsq, int64_t I, float *norm, void
  *                        alpha = 1
  *     Wanda, Eq. 1:      any W [out x in] with input-feature norms: norm_axis = COLS, group_axis = COLS
  * norm: rows (ROWS) or cols (COLS) floats.  alpha: finite, >= 0.
- * Supported patterns: m in {4, 8}, 1 <= n_keep < m; the group-axis extent must be a multiple of m,
- * and for group_axis = ROWS with bf16 data `cols` ... any value; see alignment rules above.
+ * Supported patterns: m in {4, 8}, 1 <= n_keep < m; the group-axis extent must be a multiple of m (the other
+ * extent may be any positive value; see the alignment rules above).
  * mask_bits (nullable): rows * ceil(cols/32) words; bit (c % 32) of word r * ceil(cols/32) + c / 32
  *     is 1 iff W[r,c] is kept; padding bits are written as 0.
  * W_pruned (nullable): same dtype and ld as W; survivors are copied bit for bit, the others become +0
@@ -167,6 +167,27 @@ dass_status dass_compress_nm(const void *W, const uint32_t *mask_bits,
                              int64_t rows, int64_t cols, int64_t ld, dass_dtype dt,
                              int n_keep, int m, dass_axis group_axis,
                              void *values, uint32_t *meta, void *cuda_stream);
+
+/* Stage (b) in one pass: dass_score_nm and dass_compress_nm of the same selection from a single read of W.
+ * The mask and the compressed form describe one and the same choice of survivors (Section 3, "Extension to N:M
+ * Sparsity": every group of m consecutive weights of a comparison line keeps n of them, by the score of Eq. 4 /
+ * Eq. 5), so nothing but memory traffic separates the two calls: this entry point reads each weight once and writes
+ * whichever of the outputs are asked for -- per bf16 weight 2 bytes in, 2 (pruned copy) + 0.125 (mask) + 1 (values)
+ * + 0.125 (metadata) out, against 7.375 bytes for the two calls in sequence.
+ * All arguments, layouts, the score, the order and the tie rule are those of dass_score_nm (W, norm, alpha, n_keep, m,
+ * axes, mask_bits, W_pruned) and dass_compress_nm (values, meta); the results are bit-identical to theirs.
+ * Outputs: mask_bits, W_pruned (may be W itself), values + meta -- each nullable, at least one group required;
+ * values and meta are given together or not at all.  values / meta must not overlap W.
+ * Errors: NULL (no output, or values without meta) / SHAPE / ALIGN / DTYPE / UNSUPPORTED as for dass_score_nm. */
+dass_status dass_prune_nm(const void *W, int64_t rows, int64_t cols, int64_t ld, dass_dtype dt,
+                          const float *norm, dass_axis norm_axis, float alpha,
+                          int n_keep, int m, dass_axis group_axis,
+                          uint32_t *mask_bits, void *W_pruned, void *values, uint32_t *meta, void *cuda_stream);
+/* The tuned kernels behind dass_prune_nm (bf16, 2:4 and 4:8) receive their tiles through bulk tensor copies and
+ * wait for each on a barrier; every such wait is bounded (2 s).  Waits for `cuda_stream`, then returns DASS_OK, or
+ * DASS_ERR_TIMEOUT if a wait of any dass_prune_nm call on the current device ran out since the last query (that
+ * call's outputs are then incomplete; the context stays usable) and clears the record.  CUDA failure: DASS_ERR_CUDA. */
+dass_status dass_prune_status(void *cuda_stream);
 
 /* Eq. 1's input-feature norms (Wanda; the paper prunes the attention projections with it, Section 4.1 "Sparsity"):
  *     sumsq[j] += sum_{t < T} X[t,j]^2      for j in [0, d)

@@ -26,7 +26,7 @@ ACT_BY_NAME = {"silu": ACT_SILU, "gelu_tanh": ACT_GELU_TANH, "relu": ACT_RELU}
 EXPORTS = (
     "dass_calib_workspace_bytes", "dass_calib_accumulate", "dass_calib_accumulate_static", "dass_calib_status",
     "dass_norm_finalize",
-    "dass_score_nm", "dass_compress_nm", "dass_select_workspace_bytes", "dass_select_unstructured",
+    "dass_score_nm", "dass_compress_nm", "dass_prune_nm", "dass_prune_status", "dass_select_workspace_bytes", "dass_select_unstructured",
     "dass_selftest_wait_timeout", "dass_feature_workspace_bytes", "dass_feature_sumsq",
     "dass_mlp_forward_workspace_bytes", "dass_mlp_forward",
     "dass_status_string", "dass_version",
@@ -70,6 +70,11 @@ def load() -> ctypes.CDLL:
     lib.dass_compress_nm.restype = ctypes.c_int
     lib.dass_compress_nm.argtypes = [vp, vp, i64, i64, i64, ctypes.c_int, ctypes.c_int, ctypes.c_int,
                                      ctypes.c_int, vp, vp, vp]
+    lib.dass_prune_nm.restype = ctypes.c_int
+    lib.dass_prune_nm.argtypes = [vp, i64, i64, i64, ctypes.c_int, vp, ctypes.c_int, ctypes.c_float,
+                                  ctypes.c_int, ctypes.c_int, ctypes.c_int, vp, vp, vp, vp, vp]
+    lib.dass_prune_status.restype = ctypes.c_int
+    lib.dass_prune_status.argtypes = [vp]
     lib.dass_select_workspace_bytes.restype = ctypes.c_int
     lib.dass_select_workspace_bytes.argtypes = [i64, i64, ctypes.c_int, ctypes.POINTER(sz)]
     lib.dass_select_unstructured.restype = ctypes.c_int
@@ -273,6 +278,51 @@ def compress_nm(W: torch.Tensor, mask_bits: torch.Tensor, n_keep: int, m: int, g
                                    _stream(stream))
     _check(code, "dass_compress_nm")
     return values, meta
+
+
+def prune_nm(W: torch.Tensor, norm: torch.Tensor, norm_axis: int, alpha: float, n_keep: int, m: int,
+             group_axis: int, mask_bits: Optional[torch.Tensor] = None, W_pruned: Optional[torch.Tensor] = None,
+             values: Optional[torch.Tensor] = None, meta: Optional[torch.Tensor] = None,
+             want_mask: bool = True, want_pruned: bool = True, want_compressed: bool = True,
+             stream: Optional[torch.cuda.Stream] = None):
+    """score_nm and compress_nm of the same selection in one pass over W.
+    Returns (mask_bits or None, W_pruned or None, values or None, meta or None)."""
+    rows, cols, ld = _matrix(W, "W")
+    if norm.dtype != torch.float32 or not norm.is_cuda or not norm.is_contiguous():
+        raise ValueError("norm must be a contiguous CUDA float32 tensor")
+    if norm.numel() != (rows if norm_axis == AXIS_ROWS else cols):
+        raise ValueError("norm has the wrong length for norm_axis")
+    if mask_bits is None and want_mask:
+        mask_bits = torch.empty((rows, mask_words_per_row(cols)), dtype=torch.int32, device=W.device)
+    if W_pruned is None and want_pruned:
+        W_pruned = torch.empty_strided((rows, cols), (ld, 1), dtype=W.dtype, device=W.device)
+    if W_pruned is not None:
+        prow, pcol, pld = _matrix(W_pruned, "W_pruned")
+        if (prow, pcol, pld) != (rows, cols, ld) or W_pruned.dtype != W.dtype:
+            raise ValueError("W_pruned must have W's shape, dtype and row pitch")
+    if mask_bits is not None and (mask_bits.dtype != torch.int32 or not mask_bits.is_contiguous() or
+                                  tuple(mask_bits.shape) != (rows, mask_words_per_row(cols))):
+        raise ValueError("mask_bits must be a contiguous int32 [rows x ceil(cols/32)] tensor")
+    if want_compressed or values is not None or meta is not None:
+        vshape, mshape = compress_shapes(rows, cols, n_keep, m, group_axis)
+        if values is None:
+            values = torch.empty(vshape, dtype=W.dtype, device=W.device)
+        if meta is None:
+            meta = torch.empty(mshape, dtype=torch.int32, device=W.device)
+        if tuple(values.shape) != vshape or not values.is_contiguous() or values.dtype != W.dtype:
+            raise ValueError(f"values must be a contiguous {vshape} tensor of W's dtype")
+        if tuple(meta.shape) != mshape or not meta.is_contiguous() or meta.dtype != torch.int32:
+            raise ValueError(f"meta must be a contiguous int32 {mshape} tensor")
+    code = load().dass_prune_nm(W.data_ptr(), rows, cols, ld, _dtype_code(W), norm.data_ptr(), int(norm_axis),
+                                float(alpha), int(n_keep), int(m), int(group_axis),
+                                _ptr(mask_bits), _ptr(W_pruned), _ptr(values), _ptr(meta), _stream(stream))
+    _check(code, "dass_prune_nm")
+    return mask_bits, W_pruned, values, meta
+
+
+def prune_status(stream: Optional[torch.cuda.Stream] = None) -> None:
+    """Waits for the stream and raises if a bounded wait inside a prune_nm kernel ran out since the last query."""
+    _check(load().dass_prune_status(_stream(stream)), "dass_prune_status")
 
 
 def select_workspace(rows: int, cols: int, norm_axis: int, device="cuda") -> torch.Tensor:

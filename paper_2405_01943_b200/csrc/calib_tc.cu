@@ -275,6 +275,21 @@ bool tc_make_map(CUtensorMap *map, const void *ptr, int64_t rows, int64_t cols, 
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Row-major bf16 matrix [rows x cols] with pitch ld, plain (un-swizzled) boxes of box_cols x box_rows elements;
+// out-of-range elements read as zero.  Used by the streaming stage-(b) kernels.
+bool tile_map_bf16(CUtensorMap *map, const void *ptr, int64_t rows, int64_t cols, int64_t ld, int box_cols, int box_rows)
+{
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)box_cols, (cuuint32_t)box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(ptr), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 // Token tiles per band.  16 keeps a W tile in L2 for 16 token tiles; with few tokens that leaves the persistent
 // grid (148 CTAs, which this library is written for) with a part-filled last round, so a shorter band is taken
 // when it saves at least 1 % of the modelled time -- rounds x (band's k-blocks + a per-item cost of about 29

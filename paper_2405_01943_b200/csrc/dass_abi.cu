@@ -10,6 +10,10 @@ namespace dass {
 cudaError_t score_nm_launch(const void *W, int64_t rows, int64_t cols, int64_t ld, bool bf16,
                             const float *norm, bool norm_cols, float alpha, int n_keep, int m, bool group_cols,
                             uint32_t *mask_bits, void *W_pruned, cudaStream_t st);
+cudaError_t prune_nm_launch(const void *W, int64_t rows, int64_t cols, int64_t ld, bool bf16,
+                            const float *norm, bool norm_cols, float alpha, int n_keep, int m, bool group_cols,
+                            uint32_t *mask_bits, void *W_pruned, void *values, uint32_t *meta, cudaStream_t st);
+cudaError_t prune_status_read(int *host_value, cudaStream_t st);
 cudaError_t compress_nm_launch(const void *W, const uint32_t *mask_bits, int64_t rows, int64_t cols, int64_t ld,
                                bool bf16, int n_keep, int m, bool group_cols,
                                void *values, uint32_t *meta, cudaStream_t st);
@@ -179,6 +183,36 @@ dass_status dass_score_nm(const void *W, int64_t rows, int64_t cols, int64_t ld,
                         static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
         return DASS_ERR_CUDA;
     return DASS_OK;
+}
+
+dass_status dass_prune_nm(const void *W, int64_t rows, int64_t cols, int64_t ld, dass_dtype dt,
+                          const float *norm, dass_axis norm_axis, float alpha,
+                          int n_keep, int m, dass_axis group_axis,
+                          uint32_t *mask_bits, void *W_pruned, void *values, uint32_t *meta, void *cuda_stream)
+{
+    if (!W || !norm || (!mask_bits && !W_pruned && !values)) return DASS_ERR_NULL;
+    if ((values == nullptr) != (meta == nullptr)) return DASS_ERR_NULL;      // the compressed form is both or neither
+    if (norm_axis != DASS_AXIS_ROWS && norm_axis != DASS_AXIS_COLS) return DASS_ERR_DTYPE;
+    const dass_status cs = check_nm(rows, cols, ld, (int)dt, n_keep, m, (int)group_axis);
+    if (cs != DASS_OK) return cs;
+    if (!std::isfinite(alpha) || alpha < 0.0f) return DASS_ERR_UNSUPPORTED;
+    if (!aligned16(W) || (W_pruned && !aligned16(W_pruned))) return DASS_ERR_ALIGN;
+    if ((reinterpret_cast<uintptr_t>(norm) & 3u) || (reinterpret_cast<uintptr_t>(mask_bits) & 3u) ||
+        (reinterpret_cast<uintptr_t>(meta) & 3u))
+        return DASS_ERR_ALIGN;
+    if (reinterpret_cast<uintptr_t>(values) & (dt == DASS_BF16 ? 1u : 3u)) return DASS_ERR_ALIGN;
+    if (prune_nm_launch(W, rows, cols, ld, dt == DASS_BF16, norm, norm_axis == DASS_AXIS_COLS, alpha, n_keep, m,
+                        group_axis == DASS_AXIS_COLS, mask_bits, W_pruned, values, meta,
+                        static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
+        return DASS_ERR_CUDA;
+    return DASS_OK;
+}
+
+dass_status dass_prune_status(void *cuda_stream)
+{
+    int value = 0;
+    if (prune_status_read(&value, static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) return DASS_ERR_CUDA;
+    return value == 0 ? DASS_OK : DASS_ERR_TIMEOUT;
 }
 
 dass_status dass_compress_nm(const void *W, const uint32_t *mask_bits,

@@ -1,6 +1,8 @@
 // Stage (b): Eq. 4 / Eq. 5 score and N:M selection in one streaming pass -- the plain formulation with
-// exact double products, used for fp32 weights (bf16 weights take the tuned kernels of score_nm_bf16.cu,
-// which fall back to the same exact selection on ties).
+// exact double products, used for fp32 weights and for bf16 patterns without a tuned kernel (bf16 weights otherwise
+// take the kernels of score_nm_bf16.cu / prune_nm_bf16.cu, which fall back to the same exact selection on ties).
+// When the caller asks for them, the compressed values and metadata of the same selection are emitted by the same
+// pass (Section 3, "Extension to N:M Sparsity"), so W is read once for every output.
 //
 // Bandwidth-bound: every weight is read once (128-bit loads), the pruned copy and one mask bit per
 // weight are written once; no score matrix and no sort exist.  A warp owns a tile of 32 rows by 256
@@ -14,6 +16,7 @@
 // (24 bits) fits a double without rounding.  The scale ||y||^alpha is evaluated once per tile edge
 // (per lane for column norms, per row via a shuffle for row norms), not per weight.
 #include "dass_device.cuh"
+#include "nm_compact.cuh"
 
 namespace dass {
 
@@ -21,9 +24,14 @@ struct ScoreParams {
     const void *W;
     void *Wp;            // nullable
     uint32_t *mask;      // nullable
+    void *values;        // nullable (then meta is null too)
+    uint32_t *meta;
     const float *norm;
     int64_t rows, cols, ld;
     int64_t wpr;         // mask words per row
+    int64_t vcols;       // columns of the values matrix
+    int64_t mwpl;        // metadata words per line
+    int vec_ok;          // values rows are 16-byte aligned: vector stores allowed
     int64_t col_blocks, row_blocks;
     int n_keep;
     int scale_mode;
@@ -89,6 +97,20 @@ __global__ void __launch_bounds__(SCORE_THREADS) score_group_cols_kernel(const S
                     keep |= (g * M < nvalid ? kg : 0u) << (g * M);
                 }
                 const uint32_t word = quad_pack_bytes(keep, lane);
+                if (p.values) {   // compressed form of the same selection (every lane takes part in the shuffles)
+                    Chunk<BF16> out;
+                    const int nout = nvalid / M * p.n_keep;
+                    uint32_t fb;
+                    bool two_four = false;
+                    if constexpr (M == 4) two_four = p.n_keep == 2;
+                    if (two_four) fb = compact_cols<BF16, 4, true>(ch[u], keep, 2, nout, out);
+                    else fb = compact_cols<BF16, M, false>(ch[u], keep, p.n_keep, nout, out);
+                    const uint32_t mword = quad_pack_bytes(fb, lane);
+                    if (r < p.rows && nvalid > 0) {
+                        if ((lane & 3) == 0) p.meta[r * p.mwpl + (c0 >> 5)] = mword;
+                        chunk_store_n<BF16>(out, p.values, r * p.vcols + c0 / M * p.n_keep, nout, p.vec_ok != 0);
+                    }
+                }
                 if (r < p.rows) {
                     if (p.mask && (lane & 3) == 0 && nvalid > 0) p.mask[r * p.wpr + (c0 >> 5)] = word;
                     if (p.Wp && nvalid > 0) {
@@ -102,6 +124,28 @@ __global__ void __launch_bounds__(SCORE_THREADS) score_group_cols_kernel(const S
 }
 
 // ---------------------------------------------------------------- groups along the rows
+// Compressed values and metadata of one row group at a lane's 8 columns (lanes are independent here).
+template <bool BF16, int M, bool TWO_FOUR>
+__device__ __forceinline__ void emit_rows(const ScoreParams &p, const Chunk<BF16> (&ch)[M], const uint32_t (&keep_row)[M],
+                                          int64_t line, int64_t c0, int nvalid)
+{
+    static_assert(!TWO_FOUR || M == 4, "2:4 has groups of four");
+    constexpr int MAXK = TWO_FOUR ? 2 : M - 1;
+    Chunk<BF16> out[MAXK];
+    uint32_t fields_lo, fields_hi;
+    compact_rows<BF16, M, TWO_FOUR, MAXK>(ch, keep_row, p.n_keep, out, fields_lo, fields_hi);
+    if constexpr (M == 4) {
+        p.meta[line * p.mwpl + (c0 >> 3)] = fields_lo;
+    } else {
+        p.meta[line * p.mwpl + (c0 >> 2)] = fields_lo;
+        if (nvalid > 4) p.meta[line * p.mwpl + (c0 >> 2) + 1] = fields_hi;
+    }
+#pragma unroll
+    for (int k = 0; k < MAXK; ++k)
+        if (k < p.n_keep)
+            chunk_store_n<BF16>(out[k], p.values, (line * p.n_keep + k) * p.vcols + c0, nvalid, p.vec_ok != 0);
+}
+
 template <bool BF16, int M, bool NORM_COLS>
 __global__ void __launch_bounds__(SCORE_THREADS) score_group_rows_kernel(const ScoreParams p)
 {
@@ -155,6 +199,16 @@ __global__ void __launch_bounds__(SCORE_THREADS) score_group_rows_kernel(const S
 #pragma unroll
                 for (int q = 0; q < M; ++q) keep_row[q] |= ((kg >> q) & 1u) << j;
             }
+            if (p.values && nvalid > 0) {
+                bool done = false;
+                if constexpr (M == 4) {
+                    if (p.n_keep == 2) {
+                        emit_rows<BF16, 4, true>(p, ch, keep_row, r0 / M, c0, nvalid);
+                        done = true;
+                    }
+                }
+                if (!done) emit_rows<BF16, M, false>(p, ch, keep_row, r0 / M, c0, nvalid);
+            }
 #pragma unroll
             for (int q = 0; q < M; ++q) {
                 const uint32_t word = quad_pack_bytes(keep_row[q], lane);
@@ -186,17 +240,53 @@ cudaError_t score_nm_bf16_launch(const void *W, int64_t rows, int64_t cols, int6
                                  const float *norm, bool norm_cols, float alpha, int n_keep, int m, bool group_cols,
                                  uint32_t *mask_bits, void *W_pruned, cudaStream_t st);   // score_nm_bf16.cu
 
-// Host entry used by the C ABI (arguments already validated there).
+cudaError_t prune_nm_bf16_launch(const void *W, int64_t rows, int64_t cols, int64_t ld,
+                                 const float *norm, bool norm_cols, float alpha, int m, bool group_cols,
+                                 uint32_t *mask_bits, void *W_pruned, void *values, uint32_t *meta, cudaStream_t st);   // prune_nm_bf16.cu
+
+static cudaError_t generic_launch(const void *W, int64_t rows, int64_t cols, int64_t ld, bool bf16,
+                                  const float *norm, bool norm_cols, float alpha, int n_keep, int m, bool group_cols,
+                                  uint32_t *mask_bits, void *W_pruned, void *values, uint32_t *meta, cudaStream_t st);
+
+// Host entry of dass_score_nm (arguments already validated by the C ABI).
 cudaError_t score_nm_launch(const void *W, int64_t rows, int64_t cols, int64_t ld, bool bf16,
                             const float *norm, bool norm_cols, float alpha, int n_keep, int m, bool group_cols,
                             uint32_t *mask_bits, void *W_pruned, cudaStream_t st)
 {
     if (bf16)   // bf16 weights take the integer / bit-sliced kernels of score_nm_bf16.cu
         return score_nm_bf16_launch(W, rows, cols, ld, norm, norm_cols, alpha, n_keep, m, group_cols, mask_bits, W_pruned, st);
+    return generic_launch(W, rows, cols, ld, false, norm, norm_cols, alpha, n_keep, m, group_cols, mask_bits, W_pruned,
+                          nullptr, nullptr, st);
+}
+
+// Host entry of dass_prune_nm: every requested output of the selection from one read of W.
+cudaError_t prune_nm_launch(const void *W, int64_t rows, int64_t cols, int64_t ld, bool bf16,
+                            const float *norm, bool norm_cols, float alpha, int n_keep, int m, bool group_cols,
+                            uint32_t *mask_bits, void *W_pruned, void *values, uint32_t *meta, cudaStream_t st)
+{
+    if (bf16 && 2 * n_keep == m)   // 2:4 and 4:8 on bf16: the tuned one-pass kernels
+        return prune_nm_bf16_launch(W, rows, cols, ld, norm, norm_cols, alpha, m, group_cols, mask_bits, W_pruned, values, meta, st);
+    return generic_launch(W, rows, cols, ld, bf16, norm, norm_cols, alpha, n_keep, m, group_cols, mask_bits, W_pruned,
+                          values, meta, st);
+}
+
+static cudaError_t generic_launch(const void *W, int64_t rows, int64_t cols, int64_t ld, bool bf16,
+                                  const float *norm, bool norm_cols, float alpha, int n_keep, int m, bool group_cols,
+                                  uint32_t *mask_bits, void *W_pruned, void *values, uint32_t *meta, cudaStream_t st)
+{
     ScoreParams p;
     p.W = W; p.Wp = W_pruned; p.mask = mask_bits; p.norm = norm;
+    p.values = values; p.meta = meta;
     p.rows = rows; p.cols = cols; p.ld = ld;
     p.wpr = (cols + 31) / 32;
+    {
+        const int field_bits = (n_keep == 2 && m == 4) ? 4 : m;
+        const int fpw = 32 / field_bits;
+        p.vcols = group_cols ? cols / m * n_keep : cols;
+        p.mwpl = group_cols ? (cols / m + fpw - 1) / fpw : (cols + fpw - 1) / fpw;
+        const int esz = bf16 ? 2 : 4;
+        p.vec_ok = ((p.vcols * esz) % 16 == 0) && ((reinterpret_cast<uintptr_t>(values) & 15u) == 0);
+    }
     p.col_blocks = (cols + TILE_COLS - 1) / TILE_COLS;
     p.row_blocks = (rows + TILE_ROWS - 1) / TILE_ROWS;
     p.n_keep = n_keep;
@@ -207,6 +297,9 @@ cudaError_t score_nm_launch(const void *W, int64_t rows, int64_t cols, int64_t l
     const int64_t want = (ntasks + warps_per_block - 1) / warps_per_block;
     const int64_t cap = (int64_t)device_sm_count() * 8;   // 8 blocks of 256 threads fill an SM
     const int grid = (int)(want < cap ? want : cap);
+    if (bf16)
+        return m == 4 ? launch_score<true, 4>(p, norm_cols, group_cols, grid, st)
+                      : launch_score<true, 8>(p, norm_cols, group_cols, grid, st);
     return m == 4 ? launch_score<false, 4>(p, norm_cols, group_cols, grid, st)
                   : launch_score<false, 8>(p, norm_cols, group_cols, grid, st);
 }

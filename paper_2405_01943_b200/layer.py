@@ -67,6 +67,15 @@ class LayerPruner:
             b.score_nm(W, self.norm, axis, alpha if name != "down" else 1.0, self.n_keep, self.m, axis,
                        mask_bits=o["mask"], W_pruned=o["pruned"])
 
+    def prune_nm(self, Wg: torch.Tensor, Wu: torch.Tensor, Wd: torch.Tensor, alpha: float = 0.5) -> None:
+        """score_nm and compress_nm in one pass per projection: each weight is read once for all of its outputs."""
+        for name, W in zip(_PROJECTIONS, (Wg, Wu, Wd)):
+            _, _, axis = self.geometry[name]
+            o = self.out[name]
+            b.prune_nm(W, self.norm, axis, alpha if name != "down" else 1.0, self.n_keep, self.m, axis,
+                       mask_bits=o["mask"], W_pruned=o["pruned"], values=o.get("values"), meta=o.get("meta"),
+                       want_compressed=self.compressed)
+
     def compress_nm(self, Wg: torch.Tensor, Wu: torch.Tensor, Wd: torch.Tensor) -> None:
         for name, W in zip(_PROJECTIONS, (Wg, Wu, Wd)):
             _, _, axis = self.geometry[name]
@@ -93,9 +102,7 @@ class LayerPruner:
         self.accumulate(X, Wg, Wu)
         self.finalize()
         if sparsity is None:
-            self.score_nm(Wg, Wu, Wd, alpha)
-            if self.compressed:
-                self.compress_nm(Wg, Wu, Wd)
+            self.prune_nm(Wg, Wu, Wd, alpha)
         else:
             self.select_unstructured(Wg, Wu, Wd, sparsity, alpha)
         return self.out

@@ -99,6 +99,28 @@ def test_score_nm_argument_errors(lib):
     assert call(ga=0, rows=6) == 2         # rows not a multiple of m for row groups
 
 
+def test_prune_nm_argument_errors(lib):
+    f = lib.dass_prune_nm
+    ok_args = dict(W=FAKE, rows=8, cols=64, ld=64, dt=binding.BF16, norm=FAKE, na=1, alpha=1.0, n=2, m=4, ga=1,
+                   mask=FAKE, wp=FAKE, values=FAKE, meta=FAKE, st=None)
+
+    def call(**kw):
+        a = dict(ok_args, **kw)
+        return f(a["W"], a["rows"], a["cols"], a["ld"], a["dt"], a["norm"], a["na"], a["alpha"], a["n"], a["m"],
+                 a["ga"], a["mask"], a["wp"], a["values"], a["meta"], a["st"])
+
+    assert call(W=None) == 1 and call(norm=None) == 1
+    assert call(mask=None, wp=None, values=None, meta=None) == 1      # no output at all
+    assert call(values=None) == 1 and call(meta=None) == 1           # the compressed form is both or neither
+    assert call(rows=0) == 2 and call(cols=62) == 2 and call(ld=32) == 2
+    assert call(n=4) == 2 and call(n=0) == 2 and call(ga=0, rows=6) == 2
+    assert call(m=16, n=2) == 5
+    assert call(ld=68) == 3 and call(W=FAKE + 2) == 3 and call(wp=FAKE + 4) == 3
+    assert call(meta=FAKE + 2) == 3 and call(values=FAKE + 1) == 3 and call(mask=FAKE + 1) == 3
+    assert call(dt=9) == 4 and call(na=3) == 4 and call(ga=-1) == 4
+    assert call(alpha=-0.5) == 5 and call(alpha=float("nan")) == 5
+
+
 def test_compress_nm_argument_errors(lib):
     f = lib.dass_compress_nm
     assert f(None, FAKE, 8, 64, 64, 0, 2, 4, 1, FAKE, FAKE, None) == 1
