@@ -1,19 +1,23 @@
 #!/usr/bin/env python
 """Throughput of the DaSS hot path on B200: one step = one MLP layer through the whole path
-(fused GLU calibration norms -> norm finalize -> N:M scoring of gate / up / down -> compression)
-on synthetic inputs shaped like the paper's models and its 128 x 2048-token calibration set.
+(fused GLU calibration norms -> norm finalize -> one-pass N:M scoring + selection + compression of
+gate / up / down) on synthetic inputs shaped like the paper's models and its 128 x 2048-token calibration set.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--config llama2_70b] [--impl ours|reference]
 
 Prints ONE JSON line (rank 0).  `--impl reference` times the fp64 CPU oracle on a bounded sample of
-the same workload instead.  With N > 1 (launched by torch.distributed.run) every rank prunes its own
-independent layers -- the path has no cross-GPU exchange -- and the value is the aggregate.
+the same workload instead.  `--gpus N` means N ranks: started under torch.distributed.run the script checks that
+WORLD_SIZE is N, started plainly with N > 1 it launches the N ranks itself.  Every rank prunes its own independent
+layers -- the path has no cross-GPU exchange -- and the value is the aggregate.
 """
 from __future__ import annotations
 
 import argparse
+import hashlib
 import json
+import math
 import os
+import socket
 import statistics
 import subprocess
 import sys
@@ -30,8 +34,10 @@ from paper_2405_01943_b200 import synth  # noqa: E402
 
 METRIC = "calib tokens/s (fused GLU-norm pass + N:M scoring + compression, per layer step)"
 UNIT = "tokens/s"
-KERNEL_LAUNCHES_PER_STEP = 10   # status clear, calib GEMM, partial reduce, finalize, 3 x score, 3 x compress
+KERNEL_LAUNCHES_PER_STEP = 7    # status clear, calib GEMM, partial reduce, finalize, 3 x one-pass prune
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+NOMINAL = {"hbm_gbs": 8000.0, "bf16_tflops": 2250.0}     # data-sheet figures (HBM3e, dense bf16), for context
+PER_CONFIG = ("tiny", "llama2_7b", "mistral_7b", "gemma_7b")   # reported beside the headline shape
 
 
 # --------------------------------------------------------------------------- small helpers
@@ -47,32 +53,55 @@ def load_peaks():
 
 
 def stage_b_bytes(cfg, compress=True):
-    """Algorithmic bytes of stage (b) for the three projections of one layer."""
+    """Algorithmic bytes of stage (b) for the three projections of one layer: (score pass, compress pass, one pass)."""
     esz = 2 if cfg.dtype == "bf16" else 4
     elems = 3 * cfg.d * cfg.I
     score = elems * (esz + esz + 0.125)                                   # read W, write pruned + mask bit
     frac = cfg.n_keep / cfg.m
     meta_bits = 4 / 4 if (cfg.n_keep == 2 and cfg.m == 4) else 1.0        # field bits per weight
     comp = elems * (esz + 0.125 + esz * frac + meta_bits / 8.0) if compress else 0.0
-    return score, comp
+    fused = elems * (esz + esz + 0.125 + esz * frac + meta_bits / 8.0)    # one read of W for all four outputs
+    return score, comp, fused
 
 
-# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per launch from one ncu capture of this very
-# command on the default workload; see profiles/.  None where the kernel changed after the capture.
-NCU_DRAM_BYTES = {"llama2_70b": {"calib": 122.00e9 + 20.8e6,                                  # one launch, T = 262144
-                                 "score": (2 * (470.4 + 443.6) + 471.4 + 454.4) * 1e6,         # gate + up + down
-                                 "compress": (2 * (499.1 + 206.7) + 499.2 + 214.1) * 1e6}}
+def _git_blob_sha(path):
+    """The id git gives the file's content: ties a stored counter to the kernel source it was captured from."""
+    try:
+        data = open(os.path.join(ROOT, path), "rb").read()
+    except OSError:
+        return None
+    return hashlib.sha1(b"blob %d\0" % len(data) + data).hexdigest()
 
 
-def roofline_b(kernel, algorithmic_bytes, in_step_ms, isolated_ms, peaks, peak_src, traffic):
-    """HBM roofline entry of a group of stage-(b) launches (bytes are per step: three matrices)."""
-    ms = isolated_ms if isolated_ms else in_step_ms
-    gbs = algorithmic_bytes / (ms * 1e-3) / 1e9
-    return {"bound": "hbm", "kernel": kernel, "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-            "frac": gbs / peaks["hbm_gbs"], "peak_source": peak_src,
-            "timed": "alone, back to back, after the step loop" if isolated_ms else "inside the step",
-            "in_step_gbs": algorithmic_bytes / (in_step_ms * 1e-3) / 1e9,
-            "algorithmic_bytes_per_step": algorithmic_bytes, "traffic": traffic}
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per launch, from ncu captures summarised under profiles/.
+# Each entry names its summary and the git blob id of the kernel source it was captured from; when the source has
+# changed since, the number is withheld (reported as null) instead of going stale.
+NCU_DRAM_BYTES = {}
+
+
+def ncu_traffic(cfg_name, key):
+    rec = NCU_DRAM_BYTES.get(cfg_name, {}).get(key)
+    if rec is None:
+        return None, None
+    if _git_blob_sha(rec["source"]) != rec["blob"]:
+        return None, {"withheld": f"{rec['source']} changed since {rec['profile']} was captured"}
+    return rec["bytes"], {"profile": rec["profile"], "source": rec["source"], "blob": rec["blob"], "how": rec["how"]}
+
+
+def roofline_b(kernel, algorithmic_bytes, in_step_ms, isolated_ms, peaks, peak_src, traffic, provenance):
+    """HBM roofline entry of the stage-(b) launches of one step (three matrices).  The headline fraction is the one
+    measured where the kernels run, inside the step right after the power-capped GEMM; the same launches timed
+    alone are reported beside it."""
+    gbs = algorithmic_bytes / (in_step_ms * 1e-3) / 1e9
+    out = {"bound": "hbm", "kernel": kernel, "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+           "frac": gbs / peaks["hbm_gbs"], "frac_of_nominal": gbs / NOMINAL["hbm_gbs"], "peak_source": peak_src,
+           "timed": "inside the step", "ms": in_step_ms,
+           "algorithmic_bytes_per_step": algorithmic_bytes, "traffic": traffic, "traffic_provenance": provenance}
+    if isolated_ms:
+        alone = algorithmic_bytes / (isolated_ms * 1e-3) / 1e9
+        out.update({"alone_gbs": alone, "alone_frac": alone / peaks["hbm_gbs"], "alone_ms": isolated_ms,
+                    "alone_timed": "the same launches back to back after the step loop"})
+    return out
 
 
 class ClockSampler:
@@ -160,13 +189,13 @@ class LayerPath:
                                   device=device)
         self.act = self.pruner.act
         self.sumsq, self.norm, self.ws, self.out = self.pruner.sumsq, self.pruner.norm, self.pruner.calib_ws, self.pruner.out
-        self.ev = {k: [] for k in ("calib", "score", "compress")}
+        self.ev = {k: [] for k in ("calib", "prune")}
 
     def step(self, X, Wg, Wu, Wd, alpha, record=False, before_stage_b=None, x_chunks=None):
         """x_chunks: [(first token, last token + 1, event or None)]: the calibration is then accumulated chunk by
         chunk (the sums carry over between calls), each call waiting for its chunk's event on the current stream."""
         pr = self.pruner
-        e = [torch.cuda.Event(enable_timing=True) for _ in range(4)] if record else None
+        e = [torch.cuda.Event(enable_timing=True) for _ in range(3)] if record else None
         pr.reset()
         if record:
             e[0].record()
@@ -182,19 +211,88 @@ class LayerPath:
         if before_stage_b is not None:
             before_stage_b()
         pr.finalize()
-        pr.score_nm(Wg, Wu, Wd, alpha)
+        pr.prune_nm(Wg, Wu, Wd, alpha)
         if record:
             e[2].record()
-        pr.compress_nm(Wg, Wu, Wd)
-        if record:
-            e[3].record()
             self.ev["calib"].append((e[0], e[1]))
-            self.ev["score"].append((e[1], e[2]))
-            self.ev["compress"].append((e[2], e[3]))
+            self.ev["prune"].append((e[1], e[2]))
 
     def mean_ms(self, key):
         v = [a.elapsed_time(b) for a, b in self.ev[key]]
         return sum(v) / len(v) if v else None
+
+    def check(self):
+        self.b.calib_status(self.ws)
+        self.b.prune_status()
+
+
+class PinnedArena:
+    """One pinned host allocation carved into tensors, so that the end-to-end legs of several shapes pay for page
+    locking once."""
+
+    def __init__(self, nbytes):
+        self.buf = torch.empty(int(nbytes), dtype=torch.uint8, pin_memory=True)
+        self.off = 0
+
+    def reset(self):
+        self.off = 0
+
+    def take(self, like):
+        n = like.numel() * like.element_size()
+        start = (self.off + 255) // 256 * 256
+        if start + n > self.buf.numel():
+            raise RuntimeError("pinned arena too small")
+        self.off = start + n
+        return self.buf[start:start + n].view(like.dtype).view(like.shape)
+
+
+def e2e_bytes(cfg):
+    esz = 2 if cfg.dtype == "bf16" else 4
+    up = (cfg.T * cfg.d + 3 * cfg.d * cfg.I) * esz
+    down = cfg.I * 4 + 3 * cfg.d * cfg.I * (0.125 + esz * cfg.n_keep / cfg.m + 0.125) + 4096
+    return int(up + down) + (1 << 20)
+
+
+def timed_steps(path, X, pool, alpha, steps, warmup, world, device, rank, local_rank):
+    """W untimed steps, then K timed ones between barriers; the clock of this GPU is sampled meanwhile."""
+    def barrier():
+        if world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for i in range(warmup):
+        path.step(X, *pool[i % len(pool)], alpha)
+    path.check()
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    barrier()
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0.record()
+    for i in range(steps):
+        path.step(X, *pool[(warmup + i) % len(pool)], alpha, record=True)
+    t1.record()
+    barrier()
+    clocks = sampler.stop() if rank == 0 else None
+    path.check()
+    seconds = max_over_ranks(t0.elapsed_time(t1) / 1e3, world, device)
+    return seconds, clocks
+
+
+def calib_roofline(cfg, calib_ms, peaks, peak_src, traffic, provenance):
+    flops = 4.0 * cfg.T * cfg.d * cfg.I
+    tf = flops / (calib_ms * 1e-3) / 1e12
+    out = {"bound": "tensor", "kernel": "calib_tc2_kernel", "achieved": tf, "peak": peaks["bf16_tflops_sustained"],
+           "unit": "TFLOP/s", "frac": tf / peaks["bf16_tflops_sustained"], "frac_of_burst_peak": tf / peaks["bf16_tflops"],
+           "frac_of_nominal": tf / NOMINAL["bf16_tflops"], "peak_source": peak_src,
+           "peak_note": "frac is against the cuBLAS bf16 rate this pool sustains under its power cap (the kernel runs "
+                        "inside a seconds-long step); burst and data-sheet fractions beside it",
+           "algorithmic_flops_per_launch": flops, "traffic": traffic, "traffic_provenance": provenance}
+    if cfg.dtype != "bf16":
+        out.update({"bound": "alu", "kernel": "calib_simt_kernel", "peak": None, "frac": None, "frac_of_burst_peak": None,
+                    "frac_of_nominal": None, "peak_note": "fp32 FMA correctness path of the tiny configuration; no roofline claim"})
+    return out
 
 
 def run_ours(args):
@@ -218,64 +316,63 @@ def run_ours(args):
         cfg = synth.scaled(cfg, T=args.tokens)
     alpha = 0.5
     peaks, peak_src = load_peaks()
+    extra = [n for n in PER_CONFIG if n != args.config] if (args.per_config and not args.tokens) else []
+    arena = None
+    if args.e2e_steps > 0:
+        arena = PinnedArena(max(e2e_bytes(c) for c in [cfg] + [synth.CONFIGS[n] for n in extra]))
 
     X = synth.make_x(cfg, device)
     pool = [synth.make_weights(cfg, device, layer=l) for l in layer_ids_for_rank(rank, world, args.pool, 0)]
     path = LayerPath(cfg, device, binding)
-
-    def barrier():
-        if world > 1:
-            import torch.distributed as dist
-            dist.barrier()
-        torch.cuda.synchronize()
-
-    for i in range(args.warmup):
-        path.step(X, *pool[i % len(pool)], alpha)
-    binding.calib_status(path.ws)
-
-    sampler = ClockSampler(local_rank)
-    if rank == 0:
-        sampler.start()
-    barrier()
-    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    t0.record()
-    for i in range(args.steps):
-        path.step(X, *pool[(args.warmup + i) % len(pool)], alpha, record=True)
-    t1.record()
-    barrier()
-    clocks = sampler.stop() if rank == 0 else None
-    binding.calib_status(path.ws)
-    seconds = max_over_ranks(t0.elapsed_time(t1) / 1e3, world, device)
+    seconds, clocks = timed_steps(path, X, pool, alpha, args.steps, args.warmup, world, device, rank, local_rank)
     value = aggregate_value(cfg.T, args.steps, world, seconds)
 
     # per-kernel durations measured live inside the timed region
-    calib_ms, score_ms, comp_ms = path.mean_ms("calib"), path.mean_ms("score"), path.mean_ms("compress")
-    flops = 4.0 * cfg.T * cfg.d * cfg.I
-    achieved_tf = flops / (calib_ms * 1e-3) / 1e12
-    sb, cb = stage_b_bytes(cfg)
-    score_gbs, comp_gbs = sb / (score_ms * 1e-3) / 1e9, cb / (comp_ms * 1e-3) / 1e9
+    calib_ms, prune_ms = path.mean_ms("calib"), path.mean_ms("prune")
+    sb, cb, fb = stage_b_bytes(cfg)
 
-    # stage (b) alone: the same launches back to back, away from the power-capped GEMM, so that the
-    # bandwidth-bound kernels are measured at the clocks they get by themselves
+    # stage (b) alone: the same launches back to back, away from the power-capped GEMM
     iso = isolated_stage_b(path, pool, alpha, iters=args.iso_iters) if args.iso_iters > 0 else None
-
     unstructured = unstructured_leg(path, pool, alpha, args.unstructured_iters, peaks) if args.unstructured_iters > 0 else None
-
     forward = None
     if args.forward_iters > 0 and cfg.dtype == "bf16":
         forward = forward_leg(path, X, pool[0], args.forward_tokens, args.forward_iters, peaks)
 
     # end to end: pinned host inputs -> device -> path -> results back to the host, every step
-    e2e = None
-    if args.e2e_steps > 0:
-        e2e = run_e2e(cfg, path, X, pool[0], alpha, args.e2e_steps, world, device)
+    e2e = run_e2e(cfg, path, X, pool[0], alpha, args.e2e_steps, world, device, arena) if args.e2e_steps > 0 else None
+
+    # the whole stack of layers through the layer stream: distinct weights per layer, produced on a second stream
+    stream = None
+    n_stream = args.stream_layers if args.stream_layers >= 0 else (cfg.layers if not args.tokens else 0)
+    if n_stream > 0:
+        stream = stream_leg(cfg, path, X, alpha, n_stream, rank, world, device)
 
     out = None
-    traffic = NCU_DRAM_BYTES.get(cfg.name, {}) if not args.tokens else {}
     if rank == 0:
         cpu = None
         if world == 1 and not args.no_cpu_baseline:
             cpu = cpu_baseline(cfg, X, pool[0], budget_s=args.cpu_seconds)
+        checks = {n: synth.checksum(t) for n, t in zip(("X", "Wg", "Wu", "Wd"), (X,) + tuple(pool[0]))}
+    del X, pool, path
+    torch.cuda.empty_cache()
+
+    per_config = []
+    for name in extra:
+        entry = config_entry(name, args, alpha, peaks, peak_src, world, device, rank, local_rank, binding, arena)
+        if rank == 0:
+            per_config.append(entry)
+
+    if rank == 0:
+        t_calib, prov_calib = (None, None) if args.tokens else ncu_traffic(cfg.name, "calib")
+        t_prune, prov_prune = ncu_traffic(cfg.name, "prune")
+        headline = {"config": cfg.name, "n_m": f"{cfg.n_keep}:{cfg.m}", "ms_per_step": seconds * 1e3 / args.steps,
+                    "tokens_per_s": value, "calib_ms": calib_ms, "prune_ms": prune_ms,
+                    "calib_tflops": 4.0 * cfg.T * cfg.d * cfg.I / (calib_ms * 1e-3) / 1e12,
+                    "calib_frac_sustained": 4.0 * cfg.T * cfg.d * cfg.I / (calib_ms * 1e-3) / 1e12 / peaks["bf16_tflops_sustained"],
+                    "calib_frac_burst": 4.0 * cfg.T * cfg.d * cfg.I / (calib_ms * 1e-3) / 1e12 / peaks["bf16_tflops"],
+                    "prune_in_step_frac": fb / (prune_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                    "prune_alone_frac": (fb / (iso["prune"] * 1e-3) / 1e9 / peaks["hbm_gbs"]) if iso else None,
+                    "e2e_tokens_per_s": e2e["value"] if e2e else None, "clocks": clocks}
         out = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": seconds * 1e3 / args.steps, "higher_is_better": True,
@@ -283,28 +380,24 @@ def run_ours(args):
             "config": {"workload": f"{cfg.name}-shaped {cfg.act} layer, d={cfg.d}, I={cfg.I}, T={cfg.T} calibration tokens, "
                                    f"{cfg.n_keep}:{cfg.m} on gate/up (Eq. 4, alpha={alpha}, input-balanced) and down (Eq. 5); "
                                    "mask + pruned weights + compressed values/metadata",
-                       "layers_per_rank": args.steps, "weight_sets_cycled": len(pool),
-                       "input_checksums": {n: synth.checksum(t) for n, t in zip(("X", "Wg", "Wu", "Wd"), (X,) + tuple(pool[0]))},
+                       "layers_per_rank": args.steps, "weight_sets_cycled": args.pool, "input_checksums": checks,
                        "l2": "inputs exceed L2 (X and each weight set are far larger than 126 MB); no flush",
                        "parallelism": "independent layers per GPU, no collective" if world > 1 else "single GPU"},
-            "stage_ms": {"calib": calib_ms, "score_x3": score_ms, "compress_x3": comp_ms},
-            "score_gbs": score_gbs, "compress_gbs": comp_gbs,
-            "roofline": {"bound": "tensor", "kernel": "calib_tc2_kernel", "achieved": achieved_tf,
-                         "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
-                         "frac": achieved_tf / peaks["bf16_tflops_sustained"],
-                         "frac_of_burst_peak": achieved_tf / peaks["bf16_tflops"], "peak_source": peak_src,
-                         "algorithmic_flops_per_launch": flops, "traffic": traffic.get("calib")},
-            "roofline_score": roofline_b("score_{rows,cols}_bf16_kernel x3 (gate, up, down)", sb, score_ms, iso and iso["score"],
-                                         peaks, peak_src, traffic.get("score")),
-            "roofline_compress": roofline_b("compress_rows_bf16_kernel x2 (gate, up) + compress_cols_bf16_kernel (down)", cb, comp_ms, iso and iso["compress"],
-                                            peaks, peak_src, traffic.get("compress")),
-            "unstructured": unstructured, "forward": forward,
+            "stage_ms": {"calib": calib_ms, "prune_x3": prune_ms},
+            "score_gbs": fb / (prune_ms * 1e-3) / 1e9,
+            "roofline": calib_roofline(cfg, calib_ms, peaks, peak_src, t_calib, prov_calib),
+            "roofline_prune": roofline_b("prune_rows_bf16_kernel x2 (gate, up) + prune_cols_bf16_kernel (down): score, N:M "
+                                         "selection, mask, pruned copy, values and metadata from one read of W",
+                                         fb, prune_ms, iso and iso["prune"], peaks, peak_src, t_prune, prov_prune),
+            "two_pass_alone": None if not iso else {
+                "note": "dass_score_nm then dass_compress_nm on the same matrices, timed alone: what the one-pass call replaces",
+                "score_ms": iso["score"], "compress_ms": iso["compress"],
+                "score_gbs": sb / (iso["score"] * 1e-3) / 1e9, "compress_gbs": cb / (iso["compress"] * 1e-3) / 1e9},
+            "unstructured": unstructured, "forward": forward, "stream": stream,
+            "per_config": [headline] + per_config,
             "e2e": e2e, "gpu_launches": KERNEL_LAUNCHES_PER_STEP * args.steps, "clocks": clocks,
             "cpu_baseline": cpu,
         }
-        if cfg.dtype != "bf16":
-            out["roofline"]["bound"] = "alu"
-            out["roofline"]["kernel"] = "calib_simt_kernel"
         print(json.dumps(out), flush=True)
     if world > 1:
         import torch.distributed as dist
@@ -313,17 +406,58 @@ def run_ours(args):
     return out
 
 
-def isolated_stage_b(path, pool, alpha, iters):
-    """Mean ms of the three scoring launches and of the three compression launches, timed alone."""
-    def score(ws):
-        path.pruner.score_nm(*ws, alpha)
+def config_entry(name, args, alpha, peaks, peak_src, world, device, rank, local_rank, binding, arena):
+    """The same step on another of the paper's shapes: its own inputs, its own timed loop (long enough for the clock
+    sampler to see it), its own stage-(b)-alone and end-to-end timings."""
+    cfg = synth.CONFIGS[name]
+    X = synth.make_x(cfg, device)
+    pool = [synth.make_weights(cfg, device, layer=l) for l in layer_ids_for_rank(rank, world, 2, 0)]
+    path = LayerPath(cfg, device, binding)
+    for i in range(2):
+        path.step(X, *pool[i % 2], alpha)
+    torch.cuda.synchronize()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    path.step(X, *pool[0], alpha)
+    b.record()
+    torch.cuda.synchronize()
+    est_ms = max(a.elapsed_time(b), 0.02)
+    steps = int(min(20000, max(4, math.ceil(args.per_config_seconds * 1e3 / est_ms))))
+    seconds, clocks = timed_steps(path, X, pool, alpha, steps, 3, world, device, rank, local_rank)
+    calib_ms, prune_ms = path.mean_ms("calib"), path.mean_ms("prune")
+    _, _, fb = stage_b_bytes(cfg)
+    iso = isolated_stage_b(path, pool, alpha, iters=20, two_pass=False)
+    e2e = None
+    if args.e2e_steps > 0:
+        e2e = run_e2e(cfg, path, X, pool[0], alpha, max(3, min(args.e2e_steps, 6)), world, device, arena)
+    flops = 4.0 * cfg.T * cfg.d * cfg.I
+    tf = flops / (calib_ms * 1e-3) / 1e12
+    bf16 = cfg.dtype == "bf16"
+    entry = {"config": cfg.name, "n_m": f"{cfg.n_keep}:{cfg.m}", "dtype": cfg.dtype, "steps": steps,
+             "ms_per_step": seconds * 1e3 / steps, "tokens_per_s": aggregate_value(cfg.T, steps, world, seconds),
+             "calib_ms": calib_ms, "prune_ms": prune_ms, "calib_tflops": tf,
+             "calib_frac_sustained": tf / peaks["bf16_tflops_sustained"] if bf16 else None,
+             "calib_frac_burst": tf / peaks["bf16_tflops"] if bf16 else None,
+             "prune_in_step_frac": fb / (prune_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+             "prune_alone_frac": fb / (iso["prune"] * 1e-3) / 1e9 / peaks["hbm_gbs"],
+             "e2e_tokens_per_s": e2e["value"] if e2e else None,
+             "e2e_bytes_per_step": (e2e["h2d_bytes_per_step"], e2e["d2h_bytes_per_step"]) if e2e else None,
+             "clocks": clocks}
+    if not bf16:
+        entry["note"] = "fp32 correctness configuration: a step is a handful of launch-bound kernels, no roofline claim"
+    del X, pool, path
+    torch.cuda.empty_cache()
+    return entry
 
-    def compress(ws):
-        path.pruner.compress_nm(*ws)
 
+def isolated_stage_b(path, pool, alpha, iters, two_pass=True):
+    """Mean ms of the three one-pass launches (and, for context, of the two-pass route), timed alone."""
+    legs = [("prune", lambda ws: path.pruner.prune_nm(*ws, alpha))]
+    if two_pass:
+        legs += [("score", lambda ws: path.pruner.score_nm(*ws, alpha)), ("compress", lambda ws: path.pruner.compress_nm(*ws))]
     out = {}
     time.sleep(0.5)                      # let the clocks recover from the power-capped GEMM
-    for key, fn in (("score", score), ("compress", compress)):
+    for key, fn in legs:
         for i in range(3):
             fn(pool[i % len(pool)])
         torch.cuda.synchronize()
@@ -342,22 +476,25 @@ def unstructured_leg(path, pool, alpha, iters, peaks, sparsity=0.5):
     (input-balanced) and per output row of down (output-balanced) the floor(s * L) lowest scores are pruned."""
     cfg = path.cfg
 
-    def run(ws):
-        path.pruner.select_unstructured(*ws, sparsity, alpha)
+    def timed(a):
+        for i in range(3):
+            path.pruner.select_unstructured(*pool[i % len(pool)], sparsity, a)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(iters):
+            path.pruner.select_unstructured(*pool[i % len(pool)], sparsity, a)
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / iters
 
-    for i in range(3):
-        run(pool[i % len(pool)])
-    torch.cuda.synchronize()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for i in range(iters):
-        run(pool[i % len(pool)])
-    e1.record()
-    torch.cuda.synchronize()
-    ms = e0.elapsed_time(e1) / iters
-    nbytes, _ = stage_b_bytes(cfg, compress=False)
+    ms = timed(alpha)
+    ms_a0 = timed(0.0)                   # alpha = 0: equal rounded products everywhere, the selection's worst case
+    nbytes, _, _ = stage_b_bytes(cfg, compress=False)
     gbs = nbytes / (ms * 1e-3) / 1e9
     return {"sparsity": sparsity, "ms_x3": ms, "achieved": gbs, "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"],
+            "frac_of_nominal": gbs / NOMINAL["hbm_gbs"],
+            "alpha0_ms_x3": ms_a0, "alpha0_frac": nbytes / (ms_a0 * 1e-3) / 1e9 / peaks["hbm_gbs"],
             "kernels": "select_cols_kernel + select_emit_cols_kernel (gate, up), select_rows_kernel (down)",
             "algorithmic_bytes_per_step": nbytes, "timed": "alone, back to back, after the step loop"}
 
@@ -386,20 +523,54 @@ def forward_leg(path, X, weights, tokens, iters, peaks):
     tf = flops / (ms * 1e-3) / 1e12
     return {"tokens": n, "ms": ms, "tokens_per_s": n / (ms * 1e-3), "achieved": tf, "unit": "TFLOP/s",
             "frac": tf / peaks["bf16_tflops_sustained"], "frac_of_burst_peak": tf / peaks["bf16_tflops"],
+            "frac_of_nominal": tf / NOMINAL["bf16_tflops"],
             "kernels": "mlp_forward_tc_kernel<GLU> + mlp_forward_tc_kernel<PLAIN>",
             "algorithmic_flops": flops, "timed": "alone, back to back, after the step loop"}
 
 
-def run_e2e(cfg, path, X, weights, alpha, steps, world, device):
+def stream_leg(cfg, path, X, alpha, n_layers, rank, world, device):
+    """All MLP layers of the model, one after another, through paper_2405_01943_b200.stream.LayerStream: every layer
+    has its own weights, produced on a second CUDA stream into the other of two device weight sets while the current
+    layer runs (X is reused: feeding a layer the previous layer's output needs the attention blocks in between)."""
+    from paper_2405_01943_b200.stream import LayerStream
+    first = rank * n_layers                                # every rank streams its own layers
+
+    def produce(layer, dst):
+        for d_, s_ in zip(dst, synth.make_weights(cfg, device, layer=first + layer)):
+            d_.copy_(s_)
+
+    stream = LayerStream(path.pruner, produce, n_layers, alpha=alpha)
+    torch.cuda.synchronize()
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    for _ in stream.run(X):
+        pass
+    b.record()
+    torch.cuda.synchronize()
+    path.check()
+    seconds = max_over_ranks(a.elapsed_time(b) / 1e3, world, device)
+    return {"layers": n_layers, "seconds": seconds, "ms_per_layer": seconds * 1e3 / n_layers,
+            "tokens_per_s": aggregate_value(cfg.T, n_layers, world, seconds),
+            "weights": "a distinct synthetic layer per index (seeded), generated on a second stream into two device "
+                       "weight sets while the previous layer runs; generation is inside the timed region",
+            "paper_context": "the paper's pruning pass alone took 20.70 s for LLaMA2-70B's 80 MLP layers on 8 A100 "
+                             "(table 'Pruning speed'; its calibration forward is not included)"}
+
+
+def run_e2e(cfg, path, X, weights, alpha, steps, world, device, arena):
     """Same step driven from pinned host memory: every step's inputs (X and the three weight matrices) are
     copied host -> device and its results (norms, masks, values, metadata) device -> host, all inside the
     timed region.  Copies run on a second stream into double-buffered device inputs, so the upload of step
     i+1 overlaps the kernels of step i, as a user streaming layers through the library would do."""
     Wg, Wu, Wd = weights
-    host_in = [torch.empty(t.shape, dtype=t.dtype, pin_memory=True).copy_(t) for t in (X, Wg, Wu, Wd)]
+    arena.reset()
+    host_in = [arena.take(t).copy_(t) for t in (X, Wg, Wu, Wd)]
     dev_in = [[torch.empty_like(t) for t in (X, Wg, Wu, Wd)] for _ in range(2)]
     outs = [path.norm] + [path.out[n][k] for n in ("gate", "up", "down") for k in ("mask", "values", "meta")]
-    host_out = [torch.empty(t.shape, dtype=t.dtype, pin_memory=True) for t in outs]
+    host_out = [arena.take(t) for t in outs]
     h2d = sum(t.numel() * t.element_size() for t in host_in)
     d2h = sum(t.numel() * t.element_size() for t in host_out)
     comp = torch.cuda.current_stream()
@@ -469,6 +640,7 @@ def run_e2e(cfg, path, X, weights, alpha, steps, world, device):
     run(steps)
     b.record()
     torch.cuda.synchronize()
+    path.check()
     seconds = max_over_ranks(a.elapsed_time(b) / 1e3, world, device)
     return {"value": aggregate_value(cfg.T, steps, world, seconds), "unit": UNIT, "steps": steps,
             "ms_per_step": seconds * 1e3 / steps, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
@@ -536,6 +708,36 @@ def run_reference(args):
     return out
 
 
+def free_port():
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        return sk.getsockname()[1]
+
+
+def launch_ranks(n, argv):
+    """`--gpus N` without a launcher around it: start the N ranks here (one process per GPU, torch.distributed.run on
+    this node, rendezvous on 127.0.0.1) and hand back their exit code."""
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}",
+           "--master-addr", "127.0.0.1", "--master-port", str(free_port()), os.path.abspath(__file__)] + argv
+    return subprocess.call(cmd)
+
+
+def launch_check(args):
+    """What `--gpus N` resolved to, without any GPU work (gloo on a box without GPUs): every rank reports its
+    (rank, world size); rank 0 prints them.  Used by the host tests of the launcher."""
+    import torch.distributed as dist
+    rank, _, world = dist_env()
+    if world > 1:
+        dist.init_process_group("gloo" if not torch.cuda.is_available() else "nccl")
+        seen = [None] * world
+        dist.all_gather_object(seen, (rank, world))
+        dist.destroy_process_group()
+    else:
+        seen = [(rank, world)]
+    if rank == 0:
+        print(json.dumps({"launch_check": True, "gpus": args.gpus, "ranks": seen}), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -551,11 +753,25 @@ def main():
                     help="iterations of the unstructured-selection timing loop on the same matrices (0 = skip)")
     ap.add_argument("--forward-iters", type=int, default=5, help="iterations of the forward-pass timing loop (0 = skip)")
     ap.add_argument("--forward-tokens", type=int, default=32768, help="tokens of the forward-pass timing loop")
+    ap.add_argument("--stream-layers", type=int, default=-1,
+                    help="layers of the layer-stream leg (-1 = all MLP layers of the model, 0 = skip)")
+    ap.add_argument("--per-config", type=int, default=1, help="1 = also run the paper's other shapes (0 = skip)")
+    ap.add_argument("--per-config-seconds", type=float, default=2.4, help="timed seconds per extra shape")
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--ref-tokens", type=int, default=64, help="tokens per step of the reference (oracle) arm")
+    ap.add_argument("--launch-check", action="store_true", help="only report the ranks --gpus resolved to")
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.gpus < 1:
+        raise SystemExit("bench.py: --gpus must be at least 1")
+    if "WORLD_SIZE" in os.environ:
+        if int(os.environ["WORLD_SIZE"]) != args.gpus:
+            raise SystemExit(f"bench.py: --gpus {args.gpus} but the launcher started WORLD_SIZE={os.environ['WORLD_SIZE']} ranks")
+    elif args.gpus > 1:
+        raise SystemExit(launch_ranks(args.gpus, sys.argv[1:]))
+    if args.launch_check:
+        launch_check(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)

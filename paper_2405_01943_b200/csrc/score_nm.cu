@@ -253,7 +253,9 @@ cudaError_t score_nm_launch(const void *W, int64_t rows, int64_t cols, int64_t l
                             const float *norm, bool norm_cols, float alpha, int n_keep, int m, bool group_cols,
                             uint32_t *mask_bits, void *W_pruned, cudaStream_t st)
 {
-    if (bf16)   // bf16 weights take the integer / bit-sliced kernels of score_nm_bf16.cu
+    if (bf16 && 2 * n_keep == m)   // 2:4 and 4:8: the one-pass kernels of prune_nm_bf16.cu, without the compressed outputs
+        return prune_nm_bf16_launch(W, rows, cols, ld, norm, norm_cols, alpha, m, group_cols, mask_bits, W_pruned, nullptr, nullptr, st);
+    if (bf16)   // other bf16 patterns: the integer / bit-sliced kernels of score_nm_bf16.cu
         return score_nm_bf16_launch(W, rows, cols, ld, norm, norm_cols, alpha, n_keep, m, group_cols, mask_bits, W_pruned, st);
     return generic_launch(W, rows, cols, ld, false, norm, norm_cols, alpha, n_keep, m, group_cols, mask_bits, W_pruned,
                           nullptr, nullptr, st);

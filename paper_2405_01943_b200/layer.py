@@ -113,10 +113,15 @@ class LayerPruner:
         """Z = (act(X Wg'^T) * (X Wu'^T)) Wd'^T (Eq. 2 then Eq. 3) with the pruned copies the last prune() /
         score_nm() / select_unstructured() wrote, e.g. to feed the next layer's calibration.  `workspace_bytes`
         bounds the scratch that holds the intermediate activations (default: all tokens in one pass)."""
+        return self.forward_with(X, self.out["gate"]["pruned"], self.out["up"]["pruned"], self.out["down"]["pruned"],
+                                 Z=Z, workspace_bytes=workspace_bytes)
+
+    def forward_with(self, X: torch.Tensor, Wg: torch.Tensor, Wu: torch.Tensor, Wd: torch.Tensor,
+                     Z: Optional[torch.Tensor] = None, workspace_bytes: Optional[int] = None) -> torch.Tensor:
+        """The layer's output for the weights given (e.g. the dense weights of a layer that is left unpruned)."""
         T = X.shape[0]
         lo, full = b.mlp_forward_workspace_bytes(T, self.d, self.I, self.dtype)
         nbytes = full if workspace_bytes is None else max(lo, min(full, int(workspace_bytes)))
         if self._forward_ws is None or self._forward_ws.numel() != nbytes:
             self._forward_ws = b.mlp_forward_workspace(nbytes, self.device)
-        return b.mlp_forward(X, self.out["gate"]["pruned"], self.out["up"]["pruned"], self.out["down"]["pruned"],
-                             self.act, Z=Z, workspace=self._forward_ws)
+        return b.mlp_forward(X, Wg, Wu, Wd, self.act, Z=Z, workspace=self._forward_ws)

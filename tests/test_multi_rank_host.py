@@ -53,3 +53,33 @@ def test_single_rank_is_identity():
     assert bench.max_over_ranks(2.5, 1, torch.device("cpu")) == 2.5
     assert bench.layer_ids_for_rank(0, 1, 8, 3) == list(range(11))
     assert bench.aggregate_value(10, 2, 1, 4.0) == 5.0
+
+
+def _bench(*flags, env=None):
+    import json
+    import subprocess
+    e = dict(os.environ)
+    for k in ("RANK", "LOCAL_RANK", "WORLD_SIZE", "MASTER_ADDR", "MASTER_PORT"):
+        e.pop(k, None)
+    e.update(env or {})
+    res = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), *flags], capture_output=True, text=True,
+                         cwd=ROOT, env=e, timeout=600)
+    lines = [json.loads(l) for l in res.stdout.splitlines() if l.startswith("{")]
+    return res.returncode, lines
+
+
+def test_gpus_flag_alone_starts_that_many_ranks():
+    """`bench.py --gpus 2` with no launcher around it starts two ranks itself (gloo here, no GPU work), and both
+    see WORLD_SIZE == 2."""
+    rc, lines = _bench("--gpus", "2", "--launch-check")
+    assert rc == 0 and len(lines) == 1
+    assert lines[0]["gpus"] == 2 and sorted(map(tuple, lines[0]["ranks"])) == [(0, 2), (1, 2)]
+    rc, lines = _bench("--launch-check")
+    assert rc == 0 and lines[0]["ranks"] == [[0, 1]]
+
+
+def test_gpus_flag_must_agree_with_the_launcher():
+    rc, lines = _bench("--gpus", "2", "--launch-check", env={"WORLD_SIZE": "3", "RANK": "0", "LOCAL_RANK": "0"})
+    assert rc != 0 and lines == []
+    rc, lines = _bench("--gpus", "0", "--launch-check")
+    assert rc != 0
