@@ -10,6 +10,15 @@
 //     barrier; tcgen05.commit multicasts the "slot free" and "accumulators ready" arrivals to both CTAs; the
 //     peer's epilogue warps release the accumulators with remote mbarrier arrives.
 //   * no TMA multicast is used anywhere.
+//   * the accumulators G and U fill all 512 TMEM columns, so the next tile's MMAs cannot start before the epilogue has
+//     READ them -- but they need not wait for its arithmetic.  Eight epilogue warps (two per TMEM lane quarter, each
+//     taking half of the tile's 256 token columns) pull the accumulators into registers in chunks of 16 columns,
+//     six chunks deep (the producer / MMA warpgroup gives its registers up with setmaxnreg so that the epilogue
+//     warpgroups can hold them); after two chunks of arithmetic every column has been read and the accumulators are
+//     handed back, the remaining six chunks are worked off out of registers under the next tile's MMAs.  The wait
+//     the tensor cores see per tile falls from the whole epilogue (2 MUFU per element: about 4.1 k cycles) to about
+//     a quarter of it.  The two warps of a lane quarter add their sums into the band's partial with one atomicAdd
+//     each onto a zeroed slot: two addends, so the order does not matter and the result stays bit-reproducible.
 // Everything else (item order, tile-boundary alignment barrier, L2 eviction hints, lane = neuron epilogue,
 // per-band partial sums, bounded waits) is as in calib_tc.cu.
 #include "tc_common.cuh"
@@ -23,7 +32,13 @@ constexpr int T2_BK = 64;
 constexpr int T2_UMMA_K = 16;
 constexpr int T2_STAGES = 4;
 constexpr unsigned long long T2_ALIGN_NS = 20000ull;
-constexpr int T2_THREADS = 192;
+constexpr int T2_EPI_WARPS = 8;      // two per TMEM lane quarter
+constexpr int T2_CHUNK = 16;         // accumulator columns per register chunk
+constexpr int T2_HELD = 6;           // chunks a thread holds at a time (g and u: 192 registers)
+constexpr int T2_THREADS = 128 + 32 * T2_EPI_WARPS;   // warpgroup 0: TMA producer, MMA issuer, two idle warps; warpgroups 1, 2: epilogue
+// Register split (setmaxnreg): 384 threads are launched with 168 registers each = 64512; 128 x 56 + 256 x 224 = 64512.
+constexpr int T2_REGS_LAUNCH = 168, T2_REGS_CONTROL = 56, T2_REGS_EPILOGUE = 224;
+static_assert(128 * T2_REGS_CONTROL + 32 * T2_EPI_WARPS * T2_REGS_EPILOGUE <= T2_THREADS * T2_REGS_LAUNCH, "setmaxnreg split exceeds the launch");
 constexpr uint32_t T2_TILE_BYTES = 128 * T2_BK * 2;                 // 16 KB: a 128-row, 64-column bf16 tile
 constexpr uint32_t T2_STAGE_BYTES = 3 * T2_TILE_BYTES;              // Wg + Wu + X half = 48 KB per CTA
 constexpr uint32_t T2_TMEM_COLS = 512;
@@ -67,7 +82,7 @@ calib_tc2_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
     const uint32_t bar_full = smem_u32(bars);                     // [T2_STAGES], used in the leader CTA only
     const uint32_t bar_empty = bar_full + 8 * T2_STAGES;          // [T2_STAGES], one set per CTA
     const uint32_t bar_acc_full = bar_empty + 8 * T2_STAGES;      // per CTA
-    const uint32_t bar_acc_empty = bar_acc_full + 8;              // leader CTA only: 8 epilogue warps arrive
+    const uint32_t bar_acc_empty = bar_acc_full + 8;              // leader CTA only: both CTAs' epilogue warps arrive
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * T2_STAGES + 2);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
 
@@ -83,7 +98,7 @@ calib_tc2_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
             mbar_init(bar_empty + 8 * s, 1);
         }
         mbar_init(bar_acc_full, 1);
-        mbar_init(bar_acc_empty, 8);
+        mbar_init(bar_acc_empty, 2 * T2_EPI_WARPS);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -98,6 +113,8 @@ calib_tc2_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
+    if (warp < 4) {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(T2_REGS_CONTROL));
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer (one per CTA)
         if (lane == 0) {
@@ -175,10 +192,15 @@ calib_tc2_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
             if (!ok) { *abort_flag = 1; atomicExch(p.status, (int)DASS_ERR_TIMEOUT); }
         }
         __syncwarp();
+    }
     } else {
-        // ------------------------------------------------------------ epilogue (4 warps, this CTA's 128 neurons)
-        const int quad = warp & 3;
-        const uint32_t lane_addr = tmem_base + ((uint32_t)(quad * 32) << 16);
+        // ------------------------------------------------------------ epilogue (8 warps, this CTA's 128 neurons)
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(T2_REGS_EPILOGUE));
+        constexpr int NCHUNK = (T2_BN / 2) / T2_CHUNK;        // chunks per warp: its half of the tile's token columns
+        static_assert(NCHUNK > T2_HELD && NCHUNK - T2_HELD < T2_HELD, "refills reuse the chunks computed first");
+        const int quad = warp & 3;                            // the TMEM lane quarter this warp may read
+        const int half = (warp - 4) >> 2;                     // which 128 of the 256 token columns
+        const uint32_t lane_addr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(half * (T2_BN / 2));
         const uint32_t leader_acc_empty = map_to_cta(bar_acc_empty, 0);
         uint32_t tile = 0;
         bool ok = true;
@@ -191,28 +213,39 @@ calib_tc2_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                 if (!mbar_wait(bar_acc_full, tile & 1u, abort_flag)) { ok = false; break; }
                 tc_fence_after();
                 float s = 0.0f;
-#pragma unroll 1
-                for (int col = 0; col < T2_BN; col += 32) {
-                    uint32_t g[32], u[32];
-                    tmem_ld_32(lane_addr + col, g);
-                    tmem_ld_32(lane_addr + T2_BN + col, u);
-                    tmem_wait_ld();
+                uint32_t g[T2_HELD][T2_CHUNK], u[T2_HELD][T2_CHUNK];
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) {
-                        const float h = glu_h<ACT>(__uint_as_float(g[j]), __uint_as_float(u[j]));
+                for (int ch = 0; ch < T2_HELD; ++ch) {
+                    tmem_ld_16(lane_addr + ch * T2_CHUNK, g[ch]);
+                    tmem_ld_16(lane_addr + T2_BN + ch * T2_CHUNK, u[ch]);
+                }
+                tmem_wait_ld();
+#pragma unroll
+                for (int ch = 0; ch < NCHUNK; ++ch) {
+                    const int b = ch % T2_HELD;
+#pragma unroll
+                    for (int j = 0; j < T2_CHUNK; ++j) {
+                        const float h = glu_h<ACT>(__uint_as_float(g[b][j]), __uint_as_float(u[b][j]));
                         s = fmaf(h, h, s);
                     }
-                }
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) {                         // release the accumulators to the leader's MMA warp
-                    if (rank == 0) mbar_arrive(bar_acc_empty);
-                    else mbar_arrive_cluster(leader_acc_empty);
+                    if (ch + T2_HELD < NCHUNK) {              // the registers just used take a chunk not read yet
+                        tmem_ld_16(lane_addr + (ch + T2_HELD) * T2_CHUNK, g[b]);
+                        tmem_ld_16(lane_addr + T2_BN + (ch + T2_HELD) * T2_CHUNK, u[b]);
+                    }
+                    if (ch + T2_HELD == NCHUNK - 1) {         // that was the last read: hand the accumulators back
+                        tmem_wait_ld();
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) {
+                            if (rank == 0) mbar_arrive(bar_acc_empty);
+                            else mbar_arrive_cluster(leader_acc_empty);
+                        }
+                    }
                 }
                 acc += (double)s;
             }
             const int64_t neuron = c.np * 2 * T2_BM + rank * T2_BM + quad * 32 + lane;
-            if (ok && neuron < p.I) p.partial[c.band * p.I + neuron] = acc;
+            if (ok && neuron < p.I) atomicAdd(&p.partial[c.band * p.I + neuron], acc);   // two addends onto a zeroed slot
         }
         if (!ok && lane == 0) { *abort_flag = 1; atomicExch(p.status, (int)DASS_ERR_TIMEOUT); }
     }
@@ -269,6 +302,8 @@ dass_status calib_tc2_launch(const void *X, int64_t T, int64_t ldx, const void *
     p.k_blocks = (d + T2_BK - 1) / T2_BK;
     const int64_t max_pairs = device_sm_count() / 2;
     const int grid = 2 * (int)(p.items < max_pairs ? p.items : max_pairs);
+    // the two epilogue warps of a lane quarter add into the partials: they start from zero
+    if (cudaMemsetAsync(partial, 0, (size_t)p.bands * (size_t)I * sizeof(double), st) != cudaSuccess) return DASS_ERR_CUDA;
     cudaError_t e;
     switch (act) {
     case DASS_ACT_SILU: e = launch_tc2<DASS_ACT_SILU>(mx, mg, mu, p, grid, st); break;
