@@ -27,8 +27,17 @@
  *     buffer must span rows * ld elements (vector loads may touch the padding
  *     between `cols` and `ld`; it is never written).
  *   - Errors are reported by the return code only: nothing aborts, throws or
- *     prints, and on a non-OK return no output has been touched.
+ *     prints.  Arguments are validated before anything is enqueued: on
+ *     DASS_ERR_NULL / SHAPE / ALIGN / DTYPE / UNSUPPORTED / WORKSPACE no output
+ *     has been touched.  DASS_ERR_CUDA means a CUDA runtime or driver call
+ *     failed part-way (a launch, a tensor-map encode, a copy): work enqueued
+ *     before it may still run, and the call's outputs are then unspecified.
  *   - Non-finite inputs are not diagnosed; results for them are unspecified.
+ *   - Host threads: the entry points keep no state besides per-device caches that
+ *     are atomic, so they may be called from several host threads (each with its
+ *     own current device and stream).  Calls that share a workspace, an output
+ *     buffer or the static scratch of dass_calib_accumulate_static must be
+ *     ordered by the caller, on the host and on the device.
  */
 #ifndef DASS_H
 #define DASS_H
@@ -107,7 +116,8 @@ dass_status dass_selftest_wait_timeout(void *status_word, int64_t limit_us, void
  *    one double per neuron and 4096 tokens) is refused with DASS_ERR_WORKSPACE and nothing is touched (16 MiB
  *    covers a 28672-neuron bf16 layer at 262144 tokens per call; feed larger token counts in several calls).
  *  - The first call on each device (made with that device current) looks up the scratch's device
- *    address once; make that first call before any stream capture begins.
+ *    address once; make that first call before any stream capture begins.  The look-up may be made by
+ *    several host threads at once (they cache the same address atomically).
  *  - All calls on a device share the one array, which keeps the previous call's contents; the call
  *    clears the status word itself and overwrites every partial sum it later reads.  Two calls that may
  *    overlap on the GPU (different streams, no ordering between them) race on it: order them.

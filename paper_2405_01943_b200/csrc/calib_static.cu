@@ -10,6 +10,7 @@
 //
 // The array's name is only a host-side handle.  Its device address is looked up once per device with
 // cudaGetSymbolAddress (with that device current) and cached; kernels are always given that address.
+#include <atomic>
 #include "dass_device.cuh"
 
 namespace dass {
@@ -30,20 +31,20 @@ dass_status calib_tc_launch(const void *X, int64_t T, int64_t ldx, const void *W
 static __device__ __align__(256) unsigned char g_static_scratch[DASS_STATIC_SCRATCH_BYTES];
 
 constexpr int MAX_DEVICES = 64;
-static void *g_scratch_addr[MAX_DEVICES];   // device address of g_static_scratch, per device ordinal
+static std::atomic<void *> g_scratch_addr[MAX_DEVICES];   // device address of g_static_scratch, per device ordinal
 
 // One-time set-up for the current device: resolve the symbol to its device address.
 static dass_status static_scratch_for_current_device(void **out)
 {
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MAX_DEVICES) return DASS_ERR_CUDA;
-    if (!g_scratch_addr[dev]) {
-        void *ptr = nullptr;
+    void *ptr = g_scratch_addr[dev].load(std::memory_order_acquire);
+    if (!ptr) {                         // two host threads may both resolve it: they store the same address
         const cudaError_t e = cudaGetSymbolAddress(&ptr, g_static_scratch);
         if (e != cudaSuccess || !ptr) return DASS_ERR_CUDA;
-        g_scratch_addr[dev] = ptr;
+        g_scratch_addr[dev].store(ptr, std::memory_order_release);
     }
-    *out = g_scratch_addr[dev];
+    *out = ptr;
     return DASS_OK;
 }
 

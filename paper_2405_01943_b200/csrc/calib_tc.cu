@@ -248,7 +248,8 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t
 
 static EncodeTiledFn encode_tiled_fn()
 {
-    static EncodeTiledFn fn = nullptr;
+    static std::atomic<EncodeTiledFn> cached{nullptr};      // the same value whichever host thread resolves it first
+    EncodeTiledFn fn = cached.load(std::memory_order_acquire);
     if (!fn) {
         void *ptr = nullptr;
         cudaDriverEntryPointQueryResult qres;
@@ -256,6 +257,7 @@ static EncodeTiledFn encode_tiled_fn()
             qres != cudaDriverEntryPointSuccess)
             return nullptr;
         fn = reinterpret_cast<EncodeTiledFn>(ptr);
+        cached.store(fn, std::memory_order_release);
     }
     return fn;
 }
@@ -290,8 +292,10 @@ bool tile_map_bf16(CUtensorMap *map, const void *ptr, int64_t rows, int64_t cols
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+int device_sm_count();   // dass_abi.cu
+
 // Token tiles per band.  16 keeps a W tile in L2 for 16 token tiles; with few tokens that leaves the persistent
-// grid (148 CTAs, which this library is written for) with a part-filled last round, so a shorter band is taken
+// grid (one CTA per SM: 148 on the B200 this library is written for) with a part-filled last round, so a shorter band is taken
 // when it saves at least 1 % of the modelled time -- rounds x (band's k-blocks + a per-item cost of about 29
 // k-blocks: new W tiles and the re-alignment of the CTAs, fitted to measurements) -- and the partial sums (one
 // double per band and neuron) stay within 14 MiB and within `partial_budget_bytes`, what the caller's scratch has
@@ -303,7 +307,8 @@ int calib_tc_band_tiles(int64_t T, int64_t I, int64_t d, int64_t partial_budget_
     const int64_t token_tiles = (T + TC_BN - 1) / TC_BN;
     const int64_t k_blocks = (d + TC_BK - 1) / TC_BK;
     auto bands = [&](int bt) { return (token_tiles + bt - 1) / bt; };
-    auto cost = [&](int bt) { return ((tiles * bands(bt) + 147) / 148) * (bt * k_blocks + 29); };
+    const int64_t sms = device_sm_count();   // 148 when no device is current (the size query works without one)
+    auto cost = [&](int bt) { return ((tiles * bands(bt) + sms - 1) / sms) * (bt * k_blocks + 29); };
     int best = TC_MAX_BAND_TILES;
     int64_t best_cost = cost(best);
     for (int bt = TC_MAX_BAND_TILES / 2; bt >= 1; bt >>= 1) {
@@ -342,7 +347,7 @@ template <int ACT>
 static cudaError_t launch_tc(const CUtensorMap &mx, const CUtensorMap &mg, const CUtensorMap &mu, const TcParams &p,
                              int grid, cudaStream_t st)
 {
-    static unsigned long long configured = 0ull;      // per device
+    static DeviceMask configured{0ull};               // per device
     const cudaError_t ce = ensure_dynamic_smem(calib_tc_kernel<ACT>, (int)TC_SMEM_BYTES, configured);
     if (ce != cudaSuccess) return ce;
     calib_tc_kernel<ACT><<<grid, TC_THREADS, TC_SMEM_BYTES, st>>>(mx, mg, mu, p);

@@ -273,7 +273,7 @@ template <int ACT>
 static cudaError_t launch_tc2(const CUtensorMap &mx, const CUtensorMap &mg, const CUtensorMap &mu, const T2Params &p,
                               int grid, cudaStream_t st)
 {
-    static unsigned long long configured = 0ull;      // per device
+    static DeviceMask configured{0ull};               // per device
     const cudaError_t ce = ensure_dynamic_smem(calib_tc2_kernel<ACT>, (int)T2_SMEM_BYTES, configured);
     if (ce != cudaSuccess) return ce;
     calib_tc2_kernel<ACT><<<grid, T2_THREADS, T2_SMEM_BYTES, st>>>(mx, mg, mu, p);

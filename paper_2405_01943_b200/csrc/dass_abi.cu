@@ -1,4 +1,5 @@
 // C ABI of the DaSS CUDA library: argument validation and dispatch only.  See include/dass.h.
+#include <atomic>
 #include <cmath>
 #include <cstdint>
 
@@ -32,18 +33,19 @@ dass_status calib_tc_launch(const void *X, int64_t T, int64_t ldx, const void *W
 
 cudaError_t bounded_wait_selftest_launch(int *status, unsigned long long limit_ns, cudaStream_t st);
 
+// SM count of the current device (148 when there is none, e.g. for the host-only size queries).  One atomic slot
+// per device ordinal, so host threads on different devices never see each other's value.
 int device_sm_count()
 {
-    static int cached_dev = -1, cached_sms = 0;
+    static std::atomic<int> cached[64];
     int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return 148;
-    if (dev != cached_dev) {
-        int sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0) return 148;
+    int sms = dev < 64 ? cached[dev].load(std::memory_order_relaxed) : 0;
+    if (sms <= 0) {
         if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) sms = 148;
-        cached_sms = sms;
-        cached_dev = dev;
+        if (dev < 64) cached[dev].store(sms, std::memory_order_relaxed);
     }
-    return cached_sms;
+    return sms;
 }
 
 constexpr size_t WS_HEADER = 256;   // status word + padding; partial sums start here

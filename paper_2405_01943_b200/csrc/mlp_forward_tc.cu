@@ -322,7 +322,7 @@ template <int MODE, int ACT>
 static cudaError_t fw_launch(const CUtensorMap &ma, const CUtensorMap &mb0, const CUtensorMap &mb1, const FwParams &p,
                              int grid, cudaStream_t st)
 {
-    static unsigned long long configured = 0ull;      // per device
+    static DeviceMask configured{0ull};               // per device
     const cudaError_t ce = ensure_dynamic_smem(mlp_forward_tc_kernel<MODE, ACT>, (int)FW_SMEM_BYTES, configured);
     if (ce != cudaSuccess) return ce;
     mlp_forward_tc_kernel<MODE, ACT><<<grid, FW_THREADS, FW_SMEM_BYTES, st>>>(ma, mb0, mb1, p);

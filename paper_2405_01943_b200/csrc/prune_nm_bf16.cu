@@ -769,7 +769,7 @@ int device_sm_count();   // dass_abi.cu
 bool tile_map_bf16(CUtensorMap *map, const void *ptr, int64_t rows, int64_t cols, int64_t ld, int box_cols, int box_rows);   // calib_tc.cu
 
 template <typename Kernel>
-static cudaError_t launch_prune(Kernel kernel, unsigned long long &configured, const CUtensorMap &map, const PruneParams &p,
+static cudaError_t launch_prune(Kernel kernel, DeviceMask &configured, const CUtensorMap &map, const PruneParams &p,
                                 int64_t grid, cudaStream_t st)
 {
     const cudaError_t e = ensure_dynamic_smem(kernel, (int)PN_SMEM_BYTES, configured);
@@ -781,7 +781,7 @@ static cudaError_t launch_prune(Kernel kernel, unsigned long long &configured, c
 template <int M, bool NORM_COLS, bool ALL>
 static cudaError_t launch_axis(bool group_cols, const CUtensorMap &map, const PruneParams &p, int64_t grid, cudaStream_t st)
 {
-    static unsigned long long cfg_rows = 0ull, cfg_cols = 0ull;      // per device, per instantiation
+    static DeviceMask cfg_rows{0ull}, cfg_cols{0ull};                // per device, per instantiation
     return group_cols ? launch_prune(prune_cols_bf16_kernel<M, NORM_COLS, ALL>, cfg_cols, map, p, grid, st)
                       : launch_prune(prune_rows_bf16_kernel<M, NORM_COLS, ALL>, cfg_rows, map, p, grid, st);
 }

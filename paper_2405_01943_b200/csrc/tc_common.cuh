@@ -3,6 +3,8 @@
 // Internal header.
 #pragma once
 
+#include <atomic>
+
 #include <cuda.h>
 
 #include "dass_device.cuh"
@@ -132,16 +134,18 @@ __host__ __device__ constexpr uint32_t idesc_bf16_f32(int m, int n)
 }
 
 // Raises a kernel's dynamic shared-memory limit once per device (the attribute belongs to the device's copy of
-// the kernel).  `done` holds one bit per device ordinal; ordinals past 63 are configured on every call.
+// the kernel).  `done` holds one bit per device ordinal; ordinals past 63 are configured on every call.  Safe to
+// call from several host threads: the mask is atomic, and setting the attribute twice is harmless.
+using DeviceMask = std::atomic<unsigned long long>;
 template <typename Kernel>
-inline cudaError_t ensure_dynamic_smem(Kernel kernel, int bytes, unsigned long long &done)
+inline cudaError_t ensure_dynamic_smem(Kernel kernel, int bytes, DeviceMask &done)
 {
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
-    if (dev < 64 && ((done >> dev) & 1ull)) return cudaSuccess;
+    if (dev < 64 && ((done.load(std::memory_order_acquire) >> dev) & 1ull)) return cudaSuccess;
     e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
-    if (e == cudaSuccess && dev < 64) done |= 1ull << dev;
+    if (e == cudaSuccess && dev < 64) done.fetch_or(1ull << dev, std::memory_order_release);
     return e;
 }
 

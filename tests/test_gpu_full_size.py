@@ -20,7 +20,7 @@ pytestmark = pytest.mark.gpu
 DEV = "cuda"
 NAMES = ["llama2_7b", "llama2_13b", "mistral_7b", "gemma_7b", "llama2_70b"]
 ORACLE_ACT = {"silu": oracle.ACT_SILU, "gelu_tanh": oracle.ACT_GELU_TANH}
-T_PREFIX = 300
+T_PREFIX = {"llama2_70b": 1024}         # tokens of the all-neuron prefix; 2048 for the other shapes
 N_SAMPLED = 64
 
 
@@ -59,38 +59,52 @@ def test_stage_a_sampled_neurons_over_all_tokens(layer):
     assert rel.max() <= 2e-3, f"{cfg.name}: sampled-neuron norm error {rel.max():.3e}"
 
 
+def _group_gaps(Wn, scale, na, ga, n_keep, m, diff):
+    """Oracle score gap (s_(n_keep) - s_(n_keep+1)) / s_(n_keep) of every group that holds a differing mask bit."""
+    r, c = diff[:, 0], diff[:, 1]
+    if ga == AXIS_COLS:
+        keys = np.unique(np.stack([r, c // m], 1), axis=0)
+        rr = np.repeat(keys[:, :1], m, 1)
+        cc = keys[:, 1:2] * m + np.arange(m)[None, :]
+    else:
+        keys = np.unique(np.stack([r // m, c], 1), axis=0)
+        rr = keys[:, :1] * m + np.arange(m)[None, :]
+        cc = np.repeat(keys[:, 1:2], m, 1)
+    score = np.abs(Wn[rr, cc].astype(np.float64)) * (scale[cc] if na == AXIS_COLS else scale[rr])
+    srt = -np.sort(-score, axis=1)
+    top, nxt = srt[:, n_keep - 1], srt[:, n_keep]
+    return keys, (top - nxt) / np.where(top > 0, top, 1.0)
+
+
 def test_stage_a_all_neurons_on_a_token_prefix_then_end_to_end_masks(layer):
     cfg, X, Wg, Wu, Wd = layer
-    Xp = X[:T_PREFIX]
+    Xp = X[:T_PREFIX.get(cfg.name, 2048)]
     sumsq = _gpu_sumsq(cfg, Xp, Wg, Wu)
     ref = oracle.calib_sumsq(to_np32(Xp), to_np32(Wg), to_np32(Wu), ORACLE_ACT[cfg.act])
     rel = np.abs(np.sqrt(sumsq.cpu().numpy()) - np.sqrt(ref)) / np.sqrt(ref)
     assert rel.max() <= 2e-3, f"{cfg.name}: prefix norm error {rel.max():.3e}"
 
-    # end to end on a slice of the down projection and of the gate projection
+    # end to end over the WHOLE down and gate projections: masks from the GPU's norms against the oracle's masks from
+    # the oracle's norms may differ only in groups whose oracle score gap is below 1e-3 (and such groups are rare)
     norm_gpu = binding.norm_finalize(sumsq)
     norm_ref = oracle.norm_from_sumsq(ref)
-    rows = 256
-    for W, na, alpha, ga in ((Wd[:rows], AXIS_COLS, 1.0, AXIS_COLS), (Wg[:, :rows].contiguous(), AXIS_ROWS, 0.5, AXIS_ROWS)):
-        mask_gpu, _ = binding.score_nm(W, norm_gpu, na, alpha, cfg.n_keep, cfg.m, ga, want_pruned=False)
-        torch.cuda.synchronize()
+    for W, na, alpha, ga in ((Wd, AXIS_COLS, 1.0, AXIS_COLS), (Wg, AXIS_ROWS, 0.5, AXIS_ROWS)):
+        mask_gpu, _, _, _ = binding.prune_nm(W, norm_gpu, na, alpha, cfg.n_keep, cfg.m, ga, want_pruned=False, want_compressed=False)
+        binding.prune_status()
         got = unpack_mask(u32(mask_gpu), W.shape[1])
         Wn = to_np32(W)
         want, _ = oracle.score_nm(Wn, norm_ref, na, alpha, cfg.n_keep, cfg.m, ga, want_pruned=False)
         diff = np.argwhere(got != want)
-        scale = np.array([oracle.scale(float(v), alpha) for v in norm_ref], dtype=np.float64)
-        score = np.abs(Wn.astype(np.float64)) * (scale[None, :] if na == AXIS_COLS else scale[:, None])
-        seen = set()
-        for r, c in diff:
-            key = (r, c // cfg.m) if ga == AXIS_COLS else (r // cfg.m, c)
-            if key in seen:
-                continue
-            seen.add(key)
-            grp = score[r, key[1] * cfg.m:(key[1] + 1) * cfg.m] if ga == AXIS_COLS else score[key[0] * cfg.m:(key[0] + 1) * cfg.m, c]
-            s = np.sort(grp)[::-1]
-            gap = (s[cfg.n_keep - 1] - s[cfg.n_keep]) / s[cfg.n_keep - 1]
-            assert gap < 1e-3, f"{cfg.name}: group {key} differs although the oracle gap is {gap:.3e}"
-        assert len(seen) <= 1e-3 * got.size / cfg.m                     # and such near-ties are rare
+        n_groups = got.size // cfg.m
+        if len(diff):
+            scale = np.array([oracle.scale(float(v), alpha) for v in norm_ref], dtype=np.float64)
+            keys, gaps = _group_gaps(Wn, scale, na, ga, cfg.n_keep, cfg.m, diff)
+            print(f"{cfg.name} {'down' if ga == AXIS_COLS else 'gate'}: {len(keys)} of {n_groups} groups differ, "
+                  f"largest oracle gap {gaps.max():.3e}")
+            worst = int(np.argmax(gaps))
+            assert gaps.max() < 1e-3, f"{cfg.name}: group {tuple(keys[worst])} differs although the oracle gap is {gaps.max():.3e}"
+            assert len(keys) <= 1e-3 * n_groups                            # and such near-ties are rare
+        del got, want, Wn
 
 
 def test_stage_b_full_matrices_bit_exact(layer):

@@ -209,6 +209,58 @@ def _py_scale(norm32, alpha):
     raise AssertionError
 
 
+def _is_rounded_sqrt(x: float, r: float) -> bool:
+    """r is the double nearest to sqrt(x): (r - ulp/2)^2 <= x <= (r + ulp/2)^2, in exact rationals."""
+    import math
+    half = Fraction(math.ulp(r)) / 2
+    lo, hi = Fraction(r) - half, Fraction(r) + half
+    return lo >= 0 and lo * lo <= Fraction(x) <= hi * hi
+
+
+def _is_rounded_f32(d: float, f: float) -> bool:
+    """f (a float32 value) is a float32 nearest to the double d."""
+    f32 = np.float32(f)
+    up, dn = np.nextafter(f32, np.float32(np.inf)), np.nextafter(f32, np.float32(-np.inf))
+    err = abs(Fraction(float(f32)) - Fraction(d))
+    return err <= abs(Fraction(float(up)) - Fraction(d)) and err <= abs(Fraction(float(dn)) - Fraction(d))
+
+
+@pytest.mark.parametrize("alpha", [0.25, 0.75, 0.5])
+def test_scale_roots_on_random_norms_bit_for_bit_and_by_exact_brackets(alpha):
+    """The norm^alpha recipe at 1/4 and 3/4 (and 1/2) where the roots are NOT exact: the oracle's value equals the
+    numpy restatement bit for bit, and every step of the stated route -- square root(s) correctly rounded in double,
+    their product rounded in double, one rounding to float -- is confirmed by exact-rational brackets, so another
+    rounding route (a float sqrt, pow, a fused product) would be caught."""
+    import math
+    rng = np.random.default_rng(int(alpha * 100))
+    norms = np.concatenate([rng.uniform(1e-3, 1e3, 300), rng.lognormal(0.0, 6.0, 300), [1e-30, 3.0e38, 2.0, 3.0, 0.1]]).astype(np.float32)
+    differ_from_float_route = 0
+    for n in norms:
+        got = oracle.scale(float(n), alpha)
+        assert Fraction(got) == _py_scale(n, alpha), (float(n), alpha)
+        x = float(n)
+        r1 = math.sqrt(x)
+        assert _is_rounded_sqrt(x, r1)
+        if alpha == 0.5:
+            d = r1
+        else:
+            r2 = math.sqrt(r1)
+            assert _is_rounded_sqrt(r1, r2)
+            if alpha == 0.25:
+                d = r2
+            else:
+                d = r1 * r2                                   # one rounding in double: check it as a nearest double
+                exact = Fraction(r1) * Fraction(r2)
+                assert abs(Fraction(d) - exact) <= Fraction(math.ulp(d)) / 2
+        assert _is_rounded_f32(d, got) and np.float32(got) == np.float32(d)
+        # the same exponent evaluated all in float32 differs for a fair share of inputs: the pin can tell them apart
+        f = np.float32(n)
+        alt = {0.5: np.sqrt(f), 0.25: np.sqrt(np.sqrt(f)), 0.75: np.float32(np.sqrt(f) * np.sqrt(np.sqrt(f)))}[alpha]
+        differ_from_float_route += int(np.float32(alt) != np.float32(got))
+    if alpha != 0.5:
+        assert differ_from_float_route > 0
+
+
 def _brute_force_group(scores, n_keep):
     """The unique subset whose every member precedes every non-member in
     (score desc, index asc); also returns the max-sum / lexicographically smallest subset."""

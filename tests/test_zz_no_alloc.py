@@ -8,6 +8,7 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 from paper_2405_01943_b200 import binding
 
 pytestmark = pytest.mark.gpu
@@ -45,10 +46,15 @@ def test_static_scratch_matches_workspace_entry_point_twice_in_a_row(dtype):
     # two different problems back to back: the second call finds the first one's partial sums in the scratch
     a = _layer(1500, 192, 520, dtype, seed=11)
     b = _layer(700, 128, 264, dtype, seed=12)
-    for (X, Wg, Wu), act in ((a, binding.ACT_SILU), (b, binding.ACT_GELU_TANH)):
+    for (X, Wg, Wu), act, oact in ((a, binding.ACT_SILU, oracle.ACT_SILU), (b, binding.ACT_GELU_TANH, oracle.ACT_GELU_TANH)):
         want = _regular(X, Wg, Wu, act).cpu().numpy()
         got = _static(X, Wg, Wu, act).cpu().numpy()
         rel = np.abs(np.sqrt(got) - np.sqrt(want)) / np.sqrt(want)
+        assert rel.max() <= TOL[dtype]
+        # and against the fp64 oracle, not only against the library's other entry point
+        f32 = lambda t: t.float().cpu().numpy()
+        ref = oracle.calib_sumsq(f32(X), f32(Wg), f32(Wu), oact)
+        rel = np.abs(np.sqrt(got) - np.sqrt(ref)) / np.sqrt(ref)
         assert rel.max() <= TOL[dtype]
     # and the very same call twice: equal to itself and to the regular path
     X, Wg, Wu = a
