@@ -255,6 +255,21 @@ dass_status dass_mlp_forward(const void *X, int64_t T, int64_t ldx,
                              void *Z, int64_t ldz,
                              void *workspace, size_t workspace_bytes, void *cuda_stream);
 
+/* ------------------------------------------------------------------ checked-access build
+ * (No counterpart in the paper: the stand-in for a memory sanitizer.)  libdass_check.so is this library compiled with
+ * -DDASS_BOUNDS_CHECK (python -m paper_2405_01943_b200.build --bounds-check).  In it every entry point registers the
+ * address ranges of the buffers it was handed (with the sizes this header states) and every global load and store of
+ * the library's kernels is tested against them; an access outside all ranges is skipped -- a load yields zero -- and
+ * counted.  Bulk tensor copies are not included: their extents are enforced by the tensor map in hardware.
+ * dass_bounds_report waits for `cuda_stream`, returns the number of such accesses since the last report together
+ * with the first offender's address, width in bytes and source line (each nullable), and clears the record.
+ * dass_bounds_shrink_next is a test hook: the next entry-point call registers every range `bytes` shorter at its end,
+ * so that the checker can be seen to catch (and skip) accesses to memory that is in fact valid.
+ * In the regular library both return DASS_ERR_UNSUPPORTED (and *violations = 0). */
+dass_status dass_bounds_report(int *violations /* HOST */, unsigned long long *first_address /* HOST, nullable */,
+                               int *first_bytes /* HOST, nullable */, int *first_line /* HOST, nullable */, void *cuda_stream);
+dass_status dass_bounds_shrink_next(size_t bytes);
+
 /* ------------------------------------------------------------------ misc */
 const char *dass_status_string(dass_status s);   /* static string, never NULL */
 int dass_version(void);                          /* major * 10000 + minor * 100 + patch */

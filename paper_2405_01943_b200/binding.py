@@ -29,6 +29,7 @@ EXPORTS = (
     "dass_score_nm", "dass_compress_nm", "dass_prune_nm", "dass_prune_status", "dass_select_workspace_bytes", "dass_select_unstructured",
     "dass_selftest_wait_timeout", "dass_feature_workspace_bytes", "dass_feature_sumsq",
     "dass_mlp_forward_workspace_bytes", "dass_mlp_forward",
+    "dass_bounds_report", "dass_bounds_shrink_next",
     "dass_status_string", "dass_version",
 )
 
@@ -50,7 +51,30 @@ def load() -> ctypes.CDLL:
     if not os.path.exists(LIB_PATH):
         raise RuntimeError(f"{LIB_PATH} is missing: build it with `python -m paper_2405_01943_b200.build` "
                            "(there is no fallback implementation)")
-    lib = ctypes.CDLL(LIB_PATH)
+    _lib = _declare(ctypes.CDLL(LIB_PATH))
+    return _lib
+
+
+class library:
+    """Context manager that routes every call of this module through another build of the library (the
+    checked-access build, ``libdass_check.so``) and switches back on exit."""
+
+    def __init__(self, path: str):
+        self.path = path
+
+    def __enter__(self):
+        global _lib
+        self._saved = _lib
+        _lib = _declare(ctypes.CDLL(self.path))
+        return _lib
+
+    def __exit__(self, *exc):
+        global _lib
+        _lib = self._saved
+        return False
+
+
+def _declare(lib: ctypes.CDLL) -> ctypes.CDLL:
     i64, vp, sz = ctypes.c_int64, ctypes.c_void_p, ctypes.c_size_t
     lib.dass_calib_workspace_bytes.restype = ctypes.c_int
     lib.dass_calib_workspace_bytes.argtypes = [i64, i64, i64, ctypes.c_int, ctypes.POINTER(sz)]
@@ -95,7 +119,11 @@ def load() -> ctypes.CDLL:
     lib.dass_status_string.argtypes = [ctypes.c_int]
     lib.dass_version.restype = ctypes.c_int
     lib.dass_version.argtypes = []
-    _lib = lib
+    lib.dass_bounds_report.restype = ctypes.c_int
+    lib.dass_bounds_report.argtypes = [ctypes.POINTER(ctypes.c_int), ctypes.POINTER(ctypes.c_ulonglong),
+                                       ctypes.POINTER(ctypes.c_int), ctypes.POINTER(ctypes.c_int), vp]
+    lib.dass_bounds_shrink_next.restype = ctypes.c_int
+    lib.dass_bounds_shrink_next.argtypes = [sz]
     return lib
 
 
@@ -323,6 +351,19 @@ def prune_nm(W: torch.Tensor, norm: torch.Tensor, norm_axis: int, alpha: float, 
 def prune_status(stream: Optional[torch.cuda.Stream] = None) -> None:
     """Waits for the stream and raises if a bounded wait inside a prune_nm kernel ran out since the last query."""
     _check(load().dass_prune_status(_stream(stream)), "dass_prune_status")
+
+
+def bounds_report(stream: Optional[torch.cuda.Stream] = None) -> dict:
+    """Checked-access build only: accesses outside the registered buffers since the last report (and clears it)."""
+    n, addr, nbytes, line = ctypes.c_int(0), ctypes.c_ulonglong(0), ctypes.c_int(0), ctypes.c_int(0)
+    _check(load().dass_bounds_report(ctypes.byref(n), ctypes.byref(addr), ctypes.byref(nbytes), ctypes.byref(line),
+                                     _stream(stream)), "dass_bounds_report")
+    return {"violations": n.value, "first_address": addr.value, "first_bytes": nbytes.value, "first_line": line.value}
+
+
+def bounds_shrink_next(nbytes: int) -> None:
+    """Checked-access build only (test hook): the next call registers every buffer `nbytes` shorter."""
+    _check(load().dass_bounds_shrink_next(int(nbytes)), "dass_bounds_shrink_next")
 
 
 def select_workspace(rows: int, cols: int, norm_axis: int, device="cuda") -> torch.Tensor:

@@ -65,9 +65,9 @@ calib_simt_kernel(const float *__restrict__ X, int64_t T, int64_t ldx,
             for (int e = 0; e < 4; ++e) {
                 const int64_t k = k0 + lk + e;
                 const int64_t t = t0 + lrow, n = n0 + lrow;
-                xs[lk + e][lrow] = (t < T && k < d) ? X[t * ldx + k] : 0.0f;
-                gs[lk + e][lrow] = (n < I && k < d) ? Wg[n * ldw + k] : 0.0f;
-                us[lk + e][lrow] = (n < I && k < d) ? Wu[n * ldw + k] : 0.0f;
+                xs[lk + e][lrow] = (t < T && k < d) ? DASS_LD(&X[t * ldx + k]) : 0.0f;
+                gs[lk + e][lrow] = (n < I && k < d) ? DASS_LD(&Wg[n * ldw + k]) : 0.0f;
+                us[lk + e][lrow] = (n < I && k < d) ? DASS_LD(&Wu[n * ldw + k]) : 0.0f;
             }
             __syncthreads();
 #pragma unroll
@@ -107,7 +107,7 @@ calib_simt_kernel(const float *__restrict__ X, int64_t T, int64_t ldx,
 #pragma unroll
         for (int off = 8; off >= 1; off >>= 1) v += __shfl_xor_sync(FULL_MASK, v, off);
         const int64_t n = n0 + ty * 4 + a;
-        if (tx == 0 && n < I) partial[(int64_t)blockIdx.y * I + n] = v;
+        if (tx == 0 && n < I) DASS_ST(&partial[(int64_t)blockIdx.y * I + n], v);
     }
 }
 
@@ -118,18 +118,18 @@ __global__ void calib_reduce_kernel(const double *__restrict__ partial, int64_t 
     const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= I) return;
     double s = 0.0;
-    for (int64_t p = 0; p < parts; ++p) s += partial[p * I + i];
-    sumsq[i] += s;
+    for (int64_t p = 0; p < parts; ++p) s += DASS_LD(&partial[p * I + i]);
+    DASS_ST(&sumsq[i], DASS_LD(&sumsq[i]) + s);
 }
 
 __global__ void norm_finalize_kernel(const double *__restrict__ sumsq, int64_t I, float *__restrict__ norm)
 {
     const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (i < I) norm[i] = __double2float_rn(sqrt(sumsq[i]));
+    if (i < I) DASS_ST(&norm[i], __double2float_rn(sqrt(DASS_LD(&sumsq[i]))));
 }
 
 // word 0: device status; word 1: the tensor-core kernel's alignment counter
-__global__ void status_clear_kernel(int *status) { status[0] = 0; status[1] = 0; }
+__global__ void status_clear_kernel(int *status) { DASS_ST(&status[0], 0); DASS_ST(&status[1], 0); }
 
 int64_t calib_simt_parts(int64_t T)
 {

@@ -80,6 +80,13 @@ extern "C" dass_status dass_calib_accumulate_static(const void *X, int64_t T, in
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     int *status = static_cast<int *>(scratch);
     double *partial = reinterpret_cast<double *>(static_cast<unsigned char *>(scratch) + 256);
+    DASS_BOUNDS_SCOPE(bs);
+    DASS_BOUNDS_ADD(bs, X, (size_t)T * ldx * (bf16 ? 2 : 4));
+    DASS_BOUNDS_ADD(bs, Wg, (size_t)I * ldw * (bf16 ? 2 : 4));
+    DASS_BOUNDS_ADD(bs, Wu, (size_t)I * ldw * (bf16 ? 2 : 4));
+    DASS_BOUNDS_ADD(bs, sumsq, (size_t)I * sizeof(double));
+    DASS_BOUNDS_ADD(bs, scratch, (size_t)DASS_STATIC_SCRATCH_BYTES);
+    DASS_BOUNDS_COMMIT(bs, st);
     // the status word must start at zero; the partial sums are overwritten in full by the kernels
     if (status_clear_launch(status, st) != cudaSuccess) return DASS_ERR_CUDA;
     int64_t parts;

@@ -221,7 +221,7 @@ calib_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
                 acc += (double)s;       // tokens past T are zero rows of X: act(0) * 0 adds nothing
             }
             const int64_t neuron = c.nt * TC_BM + quad * 32 + lane;
-            if (ok && neuron < p.I) p.partial[c.band * p.I + neuron] = acc;
+            if (ok && neuron < p.I) DASS_ST(&p.partial[c.band * p.I + neuron], acc);
         }
         if (!ok && lane == 0) { *abort_flag = 1; atomicExch(p.status, (int)DASS_ERR_TIMEOUT); }
     }
@@ -365,7 +365,7 @@ __global__ void bounded_wait_selftest_kernel(int *status, unsigned long long lim
         mbar_init(smem_u32(&bar), 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         const bool done = mbar_wait(smem_u32(&bar), 0u, &abort_flag, limit_ns);
-        *status = done ? 0 : (int)DASS_ERR_TIMEOUT;
+        DASS_ST(status, done ? 0 : (int)DASS_ERR_TIMEOUT);
     }
 }
 

@@ -245,7 +245,8 @@ calib_tc2_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                 acc += (double)s;
             }
             const int64_t neuron = c.np * 2 * T2_BM + rank * T2_BM + quad * 32 + lane;
-            if (ok && neuron < p.I) atomicAdd(&p.partial[c.band * p.I + neuron], acc);   // two addends onto a zeroed slot
+            if (ok && neuron < p.I && DASS_ACCESS_OK(&p.partial[c.band * p.I + neuron], 8))
+                atomicAdd(&p.partial[c.band * p.I + neuron], acc);   // two addends onto a zeroed slot
         }
         if (!ok && lane == 0) { *abort_flag = 1; atomicExch(p.status, (int)DASS_ERR_TIMEOUT); }
     }

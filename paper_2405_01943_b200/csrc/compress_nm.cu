@@ -57,7 +57,7 @@ __global__ void __launch_bounds__(C_THREADS) compress_group_cols_kernel(const Co
             for (int u = 0; u < UNROLL; ++u) {
                 if (rbase + u < p.rows && nvalid > 0) {
                     chunk_load<BF16>(ch[u], p.W, (rbase + u) * p.ld + c0, nvalid);
-                    mbyte[u] = (__ldg(p.mask + (rbase + u) * p.wpr + (c0 >> 5)) >> (8 * (lane & 3))) & 0xffu;
+                    mbyte[u] = (DASS_LD_G(p.mask + (rbase + u) * p.wpr + (c0 >> 5)) >> (8 * (lane & 3))) & 0xffu;
                 } else {
                     chunk_zero<BF16>(ch[u]);
                     mbyte[u] = 0u;
@@ -70,7 +70,7 @@ __global__ void __launch_bounds__(C_THREADS) compress_group_cols_kernel(const Co
                 const uint32_t field_byte = compact_cols<BF16, M, TWO_FOUR>(ch[u], mbyte[u], p.n_keep, nout, out);
                 const uint32_t word = quad_pack_bytes(field_byte, lane);
                 if (r < p.rows && nvalid > 0) {
-                    if ((lane & 3) == 0) p.meta[r * p.mwpl + (c0 >> 5)] = word;
+                    if ((lane & 3) == 0) DASS_ST(&p.meta[r * p.mwpl + (c0 >> 5)], word);
                     chunk_store_n<BF16>(out, p.values, r * p.vcols + c0 / M * p.n_keep, nout, p.vec_ok != 0);
                 }
             }
@@ -105,16 +105,16 @@ __global__ void __launch_bounds__(C_THREADS) compress_group_rows_kernel(const Co
 #pragma unroll
             for (int q = 0; q < M; ++q) {
                 chunk_load<BF16>(ch[q], p.W, (r0 + q) * p.ld + c0, nvalid);
-                mbyte[q] = (__ldg(p.mask + (r0 + q) * p.wpr + (c0 >> 5)) >> (8 * (lane & 3))) & 0xffu;
+                mbyte[q] = (DASS_LD_G(p.mask + (r0 + q) * p.wpr + (c0 >> 5)) >> (8 * (lane & 3))) & 0xffu;
             }
             Chunk<BF16> out[MAXK];
             uint32_t fields_lo, fields_hi;   // packed fields of columns 0..3 / 4..7 (or all 8 in lo)
             compact_rows<BF16, M, TWO_FOUR, MAXK>(ch, mbyte, p.n_keep, out, fields_lo, fields_hi);
             if constexpr (TWO_FOUR || M == 4) {
-                p.meta[line * p.mwpl + (c0 >> 3)] = fields_lo;
+                DASS_ST(&p.meta[line * p.mwpl + (c0 >> 3)], fields_lo);
             } else {
-                p.meta[line * p.mwpl + (c0 >> 2)] = fields_lo;
-                if (nvalid > 4) p.meta[line * p.mwpl + (c0 >> 2) + 1] = fields_hi;
+                DASS_ST(&p.meta[line * p.mwpl + (c0 >> 2)], fields_lo);
+                if (nvalid > 4) DASS_ST(&p.meta[line * p.mwpl + (c0 >> 2) + 1], fields_hi);
             }
 #pragma unroll
             for (int k = 0; k < MAXK; ++k)
@@ -172,14 +172,14 @@ __global__ void __launch_bounds__(C_THREADS) compress_rows_bf16_kernel(const Com
 #pragma unroll
                 for (int q = 0; q < 8; ++q) {
                     chunk_load<true>(ch[q], p.W, (rbase + q) * p.ld + c0, nvalid);
-                    mb[q] = (__ldg(p.mask + (rbase + q) * p.wpr + (c0 >> 5)) >> (8 * (lane & 3))) & 0xffu;
+                    mb[q] = (DASS_LD_G(p.mask + (rbase + q) * p.wpr + (c0 >> 5)) >> (8 * (lane & 3))) & 0xffu;
                 }
             } else {                                 // rows is a multiple of 4 only: the last group of 4 stands alone
 #pragma unroll
                 for (int q = 0; q < 8; ++q) {
                     if (q < 4) {
                         chunk_load<true>(ch[q], p.W, (rbase + q) * p.ld + c0, nvalid);
-                        mb[q] = (__ldg(p.mask + (rbase + q) * p.wpr + (c0 >> 5)) >> (8 * (lane & 3))) & 0xffu;
+                        mb[q] = (DASS_LD_G(p.mask + (rbase + q) * p.wpr + (c0 >> 5)) >> (8 * (lane & 3))) & 0xffu;
                     } else {
                         chunk_zero<true>(ch[q]);
                         mb[q] = 0u;
@@ -236,8 +236,8 @@ __global__ void __launch_bounds__(C_THREADS) compress_rows_bf16_kernel(const Com
                             if (j < 4) fields_lo |= colmask << (8 * j);
                             else fields_hi |= colmask << (8 * (j - 4));
                         }
-                        p.meta[line * p.mwpl + (c0 >> 2)] = fields_lo;
-                        if (nvalid > 4) p.meta[line * p.mwpl + (c0 >> 2) + 1] = fields_hi;
+                        DASS_ST(&p.meta[line * p.mwpl + (c0 >> 2)], fields_lo);
+                        if (nvalid > 4) DASS_ST(&p.meta[line * p.mwpl + (c0 >> 2) + 1], fields_hi);
                     } else {
                         // nibble j = keep mask of column j, or for 2:4 pos_lo | pos_hi << 2
                         const uint32_t x = TWO_FOUR ? (pos[0][0] | (pos[0][1] << 8) | (pos[1][0] << 16) | (pos[1][1] << 24))
@@ -245,7 +245,7 @@ __global__ void __launch_bounds__(C_THREADS) compress_rows_bf16_kernel(const Com
                         uint32_t fields = 0u;
 #pragma unroll
                         for (int j = 0; j < 8; ++j) fields |= gather_bit(x, j) << (4 * j);
-                        p.meta[line * p.mwpl + (c0 >> 3)] = fields;
+                        DASS_ST(&p.meta[line * p.mwpl + (c0 >> 3)], fields);
                     }
 #pragma unroll
                     for (int k = 0; k < K; ++k) {

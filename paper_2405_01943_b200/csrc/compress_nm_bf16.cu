@@ -94,8 +94,8 @@ __global__ void __launch_bounds__(CF_THREADS, 3) compress_cols_bf16_kernel(const
         for (int i = 0; i < CD_ROWS; ++i) {
             const bool ok = nvalid > 0 && r0 + i < p.rows;
             // the row pitch is a multiple of 8 elements: a whole vector stays inside the row's pitch
-            v[i] = ok ? __ldcs(reinterpret_cast<const uint4 *>(p.W + (r0 + i) * p.ld + c0)) : make_uint4(0u, 0u, 0u, 0u);
-            mw[i] = ok ? __ldg(p.mask + (r0 + i) * p.wpr + (c0 >> 5)) : 0u;
+            v[i] = ok ? DASS_LD_CS(reinterpret_cast<const uint4 *>(p.W + (r0 + i) * p.ld + c0)) : make_uint4(0u, 0u, 0u, 0u);
+            mw[i] = ok ? DASS_LD_G(p.mask + (r0 + i) * p.wpr + (c0 >> 5)) : 0u;
         }
         uint16_t *dst = p.values + r0 * p.vcols + (c0 >> p.log2m) * p.n_keep;
         uint32_t *mdst = p.meta + r0 * p.mwpl + (c0 >> 5);
@@ -108,11 +108,11 @@ __global__ void __launch_bounds__(CF_THREADS, 3) compress_cols_bf16_kernel(const
             for (int i = 0; i < CD_ROWS; ++i, dst += p.vcols, mdst += p.mwpl) {
                 const uint32_t mb = (mw[i] >> (8 * (lane & 3))) & 0xffu;
                 const uint32_t word = quad_pack_bytes((uint32_t)meta_lut[mb], lane);
-                if ((lane & 3) == 0) *mdst = word;
+                if ((lane & 3) == 0) DASS_ST(mdst, word);
                 const uint32_t s0 = sel_lut[0][mb], s1 = sel_lut[1][mb];
                 const uint32_t o0 = prmt_c(prmt_c(v[i].x, v[i].y, s0 & 0xffffu), prmt_c(v[i].z, v[i].w, s0 & 0xffffu), s0 >> 16);
                 const uint32_t o1 = prmt_c(prmt_c(v[i].x, v[i].y, s1 & 0xffffu), prmt_c(v[i].z, v[i].w, s1 & 0xffffu), s1 >> 16);
-                __stcs(reinterpret_cast<uint2 *>(dst), make_uint2(o0, o1));
+                DASS_ST_CS(reinterpret_cast<uint2 *>(dst), make_uint2(o0, o1));
             }
             continue;
         }
@@ -121,7 +121,7 @@ __global__ void __launch_bounds__(CF_THREADS, 3) compress_cols_bf16_kernel(const
             const uint32_t mb = (mw[i] >> (8 * (lane & 3))) & 0xffu;
             const uint32_t word = quad_pack_bytes((uint32_t)meta_lut[mb], lane);
             if (nvalid == 0 || r0 + i >= p.rows) continue;
-            if ((lane & 3) == 0) *mdst = word;
+            if ((lane & 3) == 0) DASS_ST(mdst, word);
             uint32_t out[4];
 #pragma unroll
             for (int w = 0; w < 4; ++w) {
@@ -135,11 +135,11 @@ __global__ void __launch_bounds__(CF_THREADS, 3) compress_cols_bf16_kernel(const
                 }
             }
             if (nout == 4 && p.vec_ok) {
-                __stcs(reinterpret_cast<uint2 *>(dst), make_uint2(out[0], out[1]));
+                DASS_ST_CS(reinterpret_cast<uint2 *>(dst), make_uint2(out[0], out[1]));
             } else {
                 for (int k = 0; k < nout; ++k) {
                     const uint32_t ow = k < 2 ? out[0] : k < 4 ? out[1] : k < 6 ? out[2] : out[3];
-                    dst[k] = (uint16_t)((k & 1) ? (ow >> 16) : (ow & 0xffffu));
+                    DASS_ST(&dst[k], (uint16_t)((k & 1) ? (ow >> 16) : (ow & 0xffffu)));
                 }
             }
         }

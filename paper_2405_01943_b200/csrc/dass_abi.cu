@@ -66,6 +66,33 @@ static dass_status check_nm(int64_t rows, int64_t cols, int64_t ld, int dt, int 
     return DASS_OK;
 }
 
+// Checking build: the address ranges of a stage-(b) call's buffers (sizes as include/dass.h states them).
+#ifdef DASS_BOUNDS_CHECK
+static void register_nm_ranges(BoundsScope &bs, const void *W, int64_t rows, int64_t cols, int64_t ld, int dt,
+                               const float *norm, int norm_axis, int n_keep, int m, int group_axis,
+                               const uint32_t *mask_bits, const void *W_pruned, const void *values, const uint32_t *meta)
+{
+    const size_t esz = dt == DASS_BF16 ? 2 : 4;
+    bs.add(W, (size_t)rows * ld * esz);
+    bs.add(W_pruned, (size_t)rows * ld * esz);
+    bs.add(norm, (size_t)(norm_axis == DASS_AXIS_ROWS ? rows : cols) * sizeof(float));
+    bs.add(mask_bits, (size_t)rows * ((cols + 31) / 32) * sizeof(uint32_t));
+    const int field_bits = (n_keep == 2 && m == 4) ? 4 : m;
+    const int64_t fpw = 32 / field_bits;
+    if (group_axis == DASS_AXIS_COLS) {
+        bs.add(values, (size_t)rows * (cols / m * n_keep) * esz);
+        bs.add(meta, (size_t)rows * ((cols / m + fpw - 1) / fpw) * sizeof(uint32_t));
+    } else {
+        bs.add(values, (size_t)(rows / m * n_keep) * cols * esz);
+        bs.add(meta, (size_t)(rows / m) * ((cols + fpw - 1) / fpw) * sizeof(uint32_t));
+    }
+}
+#define DASS_BOUNDS_REF(name) (name)
+#else
+#define register_nm_ranges(...) do { } while (0)
+#define DASS_BOUNDS_REF(name) 0
+#endif
+
 }  // namespace dass
 
 using namespace dass;
@@ -122,6 +149,13 @@ dass_status dass_calib_accumulate(const void *X, int64_t T, int64_t ldx,
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     int *status = static_cast<int *>(workspace);
     double *partial = reinterpret_cast<double *>(static_cast<char *>(workspace) + WS_HEADER);
+    DASS_BOUNDS_SCOPE(bs);
+    DASS_BOUNDS_ADD(bs, X, (size_t)T * ldx * (bf16 ? 2 : 4));
+    DASS_BOUNDS_ADD(bs, Wg, (size_t)I * ldw * (bf16 ? 2 : 4));
+    DASS_BOUNDS_ADD(bs, Wu, (size_t)I * ldw * (bf16 ? 2 : 4));
+    DASS_BOUNDS_ADD(bs, sumsq, (size_t)I * sizeof(double));
+    DASS_BOUNDS_ADD(bs, workspace, workspace_bytes);
+    DASS_BOUNDS_COMMIT(bs, st);
     if (status_clear_launch(status, st) != cudaSuccess) return DASS_ERR_CUDA;
     int64_t parts;
     if (bf16) {
@@ -154,6 +188,9 @@ dass_status dass_selftest_wait_timeout(void *status_word, int64_t limit_us, void
     if (!status_word) return DASS_ERR_NULL;
     if (limit_us < 1 || limit_us > 1000000) return DASS_ERR_SHAPE;
     if (reinterpret_cast<uintptr_t>(status_word) & 3u) return DASS_ERR_ALIGN;
+    DASS_BOUNDS_SCOPE(bs);
+    DASS_BOUNDS_ADD(bs, status_word, sizeof(int));
+    DASS_BOUNDS_COMMIT(bs, static_cast<cudaStream_t>(cuda_stream));
     if (bounded_wait_selftest_launch(static_cast<int *>(status_word), (unsigned long long)limit_us * 1000ull,
                                      static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
         return DASS_ERR_CUDA;
@@ -164,6 +201,10 @@ dass_status dass_norm_finalize(const double *sumsq, int64_t I, float *norm, void
 {
     if (!sumsq || !norm) return DASS_ERR_NULL;
     if (I < 1) return DASS_ERR_SHAPE;
+    DASS_BOUNDS_SCOPE(bs);
+    DASS_BOUNDS_ADD(bs, sumsq, (size_t)I * sizeof(double));
+    DASS_BOUNDS_ADD(bs, norm, (size_t)I * sizeof(float));
+    DASS_BOUNDS_COMMIT(bs, static_cast<cudaStream_t>(cuda_stream));
     if (norm_finalize_launch(sumsq, I, norm, static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) return DASS_ERR_CUDA;
     return DASS_OK;
 }
@@ -180,6 +221,9 @@ dass_status dass_score_nm(const void *W, int64_t rows, int64_t cols, int64_t ld,
     if (!std::isfinite(alpha) || alpha < 0.0f) return DASS_ERR_UNSUPPORTED;
     if (!aligned16(W) || (W_pruned && !aligned16(W_pruned))) return DASS_ERR_ALIGN;
     if ((reinterpret_cast<uintptr_t>(norm) & 3u) || (reinterpret_cast<uintptr_t>(mask_bits) & 3u)) return DASS_ERR_ALIGN;
+    DASS_BOUNDS_SCOPE(bs);
+    register_nm_ranges(DASS_BOUNDS_REF(bs), W, rows, cols, ld, dt, norm, norm_axis, n_keep, m, group_axis, mask_bits, W_pruned, nullptr, nullptr);
+    DASS_BOUNDS_COMMIT(bs, static_cast<cudaStream_t>(cuda_stream));
     if (score_nm_launch(W, rows, cols, ld, dt == DASS_BF16, norm, norm_axis == DASS_AXIS_COLS, alpha, n_keep, m,
                         group_axis == DASS_AXIS_COLS, mask_bits, W_pruned,
                         static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
@@ -203,6 +247,9 @@ dass_status dass_prune_nm(const void *W, int64_t rows, int64_t cols, int64_t ld,
         (reinterpret_cast<uintptr_t>(meta) & 3u))
         return DASS_ERR_ALIGN;
     if (reinterpret_cast<uintptr_t>(values) & (dt == DASS_BF16 ? 1u : 3u)) return DASS_ERR_ALIGN;
+    DASS_BOUNDS_SCOPE(bs);
+    register_nm_ranges(DASS_BOUNDS_REF(bs), W, rows, cols, ld, dt, norm, norm_axis, n_keep, m, group_axis, mask_bits, W_pruned, values, meta);
+    DASS_BOUNDS_COMMIT(bs, static_cast<cudaStream_t>(cuda_stream));
     if (prune_nm_launch(W, rows, cols, ld, dt == DASS_BF16, norm, norm_axis == DASS_AXIS_COLS, alpha, n_keep, m,
                         group_axis == DASS_AXIS_COLS, mask_bits, W_pruned, values, meta,
                         static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
@@ -228,6 +275,9 @@ dass_status dass_compress_nm(const void *W, const uint32_t *mask_bits,
     if (!aligned16(W)) return DASS_ERR_ALIGN;
     if ((reinterpret_cast<uintptr_t>(mask_bits) & 3u) || (reinterpret_cast<uintptr_t>(meta) & 3u)) return DASS_ERR_ALIGN;
     if (reinterpret_cast<uintptr_t>(values) & (dt == DASS_BF16 ? 1u : 3u)) return DASS_ERR_ALIGN;
+    DASS_BOUNDS_SCOPE(bs);
+    register_nm_ranges(DASS_BOUNDS_REF(bs), W, rows, cols, ld, dt, nullptr, DASS_AXIS_ROWS, n_keep, m, group_axis, mask_bits, nullptr, values, meta);
+    DASS_BOUNDS_COMMIT(bs, static_cast<cudaStream_t>(cuda_stream));
     if (compress_nm_launch(W, mask_bits, rows, cols, ld, dt == DASS_BF16, n_keep, m, group_axis == DASS_AXIS_COLS,
                            values, meta, static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
         return DASS_ERR_CUDA;

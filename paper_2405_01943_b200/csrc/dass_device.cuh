@@ -6,6 +6,7 @@
 #include <stdint.h>
 
 #include "dass.h"
+#include "bounds_check.cuh"
 
 namespace dass {
 
@@ -73,14 +74,14 @@ template <bool BF16>
 __device__ __forceinline__ void chunk_load(Chunk<BF16> &c, const void *base, int64_t off, int nvalid)
 {
     if constexpr (BF16) {
-        const uint4 v = __ldcs(reinterpret_cast<const uint4 *>(static_cast<const uint16_t *>(base) + off));
+        const uint4 v = DASS_LD_CS(reinterpret_cast<const uint4 *>(static_cast<const uint16_t *>(base) + off));
         c.w[0] = v.x; c.w[1] = v.y; c.w[2] = v.z; c.w[3] = v.w;
     } else {
         const uint4 *p = reinterpret_cast<const uint4 *>(static_cast<const uint32_t *>(base) + off);
-        const uint4 a = __ldcs(p);
+        const uint4 a = DASS_LD_CS(p);
         c.w[0] = a.x; c.w[1] = a.y; c.w[2] = a.z; c.w[3] = a.w;
         if (nvalid > 4) {
-            const uint4 b = __ldcs(p + 1);
+            const uint4 b = DASS_LD_CS(p + 1);
             c.w[4] = b.x; c.w[5] = b.y; c.w[6] = b.z; c.w[7] = b.w;
         } else {
             c.w[4] = c.w[5] = c.w[6] = c.w[7] = 0u;
@@ -133,17 +134,17 @@ __device__ __forceinline__ void chunk_store(const Chunk<BF16> &c, void *base, in
     if constexpr (BF16) {
         uint16_t *p = static_cast<uint16_t *>(base) + off;
         if (nvalid == 8) {
-            __stcs(reinterpret_cast<uint4 *>(p), make_uint4(c.w[0], c.w[1], c.w[2], c.w[3]));
+            DASS_ST_CS(reinterpret_cast<uint4 *>(p), make_uint4(c.w[0], c.w[1], c.w[2], c.w[3]));
         } else {
-            for (int j = 0; j < nvalid; ++j) p[j] = (uint16_t)chunk_bits<true>(c, j);
+            for (int j = 0; j < nvalid; ++j) DASS_ST(&p[j], (uint16_t)chunk_bits<true>(c, j));
         }
     } else {
         uint32_t *p = static_cast<uint32_t *>(base) + off;
-        if (nvalid >= 4) __stcs(reinterpret_cast<uint4 *>(p), make_uint4(c.w[0], c.w[1], c.w[2], c.w[3]));
+        if (nvalid >= 4) DASS_ST_CS(reinterpret_cast<uint4 *>(p), make_uint4(c.w[0], c.w[1], c.w[2], c.w[3]));
         if (nvalid == 8) {
-            __stcs(reinterpret_cast<uint4 *>(p) + 1, make_uint4(c.w[4], c.w[5], c.w[6], c.w[7]));
+            DASS_ST_CS(reinterpret_cast<uint4 *>(p) + 1, make_uint4(c.w[4], c.w[5], c.w[6], c.w[7]));
         } else {
-            for (int j = (nvalid >= 4 ? 4 : 0); j < nvalid; ++j) p[j] = c.w[j];
+            for (int j = (nvalid >= 4 ? 4 : 0); j < nvalid; ++j) DASS_ST(&p[j], c.w[j]);
         }
     }
 }

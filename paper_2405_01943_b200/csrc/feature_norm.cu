@@ -14,12 +14,13 @@ constexpr int FN_MAX_SLICES = 256;
 
 template <bool BF16>
 __global__ void __launch_bounds__(FN_THREADS) feature_sumsq_kernel(const void *__restrict__ X, int64_t T, int64_t d, int64_t ldx,
-                                                                    int64_t rows_per_slice, int64_t col_blocks,
+                                                                    int64_t rows_per_slice, int64_t col_blocks, int64_t slices,
                                                                     double *__restrict__ partial /* [slices][d] */)
 {
     const int lane = threadIdx.x & 31;
     const int64_t warp = (int64_t)blockIdx.x * (FN_THREADS / 32) + (threadIdx.x >> 5);
     const int64_t cb = warp % col_blocks, slice = warp / col_blocks;
+    if (slice >= slices) return;          // the last block's spare warps have no slice (and no row of `partial`)
     const int64_t c0 = cb * 256 + lane * 8;
     const int64_t left = d - c0;
     const int nvalid = left >= 8 ? 8 : (left > 0 ? (int)left : 0);
@@ -46,7 +47,7 @@ __global__ void __launch_bounds__(FN_THREADS) feature_sumsq_kernel(const void *_
 #pragma unroll
             for (int j = 0; j < 8; ++j) acc[j] += (double)s[j];   // 64 fp32 terms at a time, double across blocks
         }
-        for (int j = 0; j < nvalid; ++j) partial[slice * d + c0 + j] = acc[j];
+        for (int j = 0; j < nvalid; ++j) DASS_ST(&partial[slice * d + c0 + j], acc[j]);
     }
 }
 
@@ -65,8 +66,8 @@ cudaError_t feature_sumsq_launch(const void *X, int64_t T, int64_t d, int64_t ld
     const int64_t col_blocks = (d + 255) / 256;
     const int64_t warps = col_blocks * slices;
     const unsigned grid = (unsigned)((warps + FN_THREADS / 32 - 1) / (FN_THREADS / 32));
-    if (bf16) feature_sumsq_kernel<true><<<grid, FN_THREADS, 0, st>>>(X, T, d, ldx, rows_per_slice, col_blocks, partial);
-    else feature_sumsq_kernel<false><<<grid, FN_THREADS, 0, st>>>(X, T, d, ldx, rows_per_slice, col_blocks, partial);
+    if (bf16) feature_sumsq_kernel<true><<<grid, FN_THREADS, 0, st>>>(X, T, d, ldx, rows_per_slice, col_blocks, slices, partial);
+    else feature_sumsq_kernel<false><<<grid, FN_THREADS, 0, st>>>(X, T, d, ldx, rows_per_slice, col_blocks, slices, partial);
     return cudaGetLastError();
 }
 
@@ -100,6 +101,11 @@ extern "C" dass_status dass_feature_sumsq(const void *X, int64_t T, int64_t d, i
     if (reinterpret_cast<uintptr_t>(workspace) & 15u) return DASS_ERR_ALIGN;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     double *partial = static_cast<double *>(workspace);
+    DASS_BOUNDS_SCOPE(bs);
+    DASS_BOUNDS_ADD(bs, X, (size_t)T * ldx * (bf16 ? 2 : 4));
+    DASS_BOUNDS_ADD(bs, sumsq, (size_t)d * sizeof(double));
+    DASS_BOUNDS_ADD(bs, workspace, workspace_bytes);
+    DASS_BOUNDS_COMMIT(bs, st);
     if (feature_sumsq_launch(X, T, d, ldx, bf16, partial, st) != cudaSuccess) return DASS_ERR_CUDA;
     if (calib_reduce_launch(partial, feature_slices(T), d, sumsq, st) != cudaSuccess) return DASS_ERR_CUDA;
     return DASS_OK;

@@ -77,6 +77,14 @@ dass_status dass_mlp_forward(const void *X, int64_t T, int64_t ldx,
     else rows -= rows % FWD_MIN_ROWS;
     if (rows < 1) return DASS_ERR_WORKSPACE;
 
+    DASS_BOUNDS_SCOPE(bs);
+    DASS_BOUNDS_ADD(bs, X, (size_t)T * ldx * elt);
+    DASS_BOUNDS_ADD(bs, Wg, (size_t)I * ldw * elt);
+    DASS_BOUNDS_ADD(bs, Wu, (size_t)I * ldw * elt);
+    DASS_BOUNDS_ADD(bs, Wd, (size_t)d * ldd * elt);
+    DASS_BOUNDS_ADD(bs, Z, ((size_t)(T - 1) * ldz + d) * elt);
+    DASS_BOUNDS_ADD(bs, workspace, workspace_bytes);
+    DASS_BOUNDS_COMMIT(bs, st);
     if (status_clear_launch(words, st) != cudaSuccess) return DASS_ERR_CUDA;
     for (int64_t t0 = 0; t0 < T; t0 += rows) {
         const int64_t tc = T - t0 < rows ? T - t0 : rows;

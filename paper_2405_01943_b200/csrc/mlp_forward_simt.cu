@@ -30,9 +30,9 @@ mlp_forward_simt_kernel(const float *__restrict__ B, int64_t T, int64_t ldb,
             const int row = ty + 8 * r;
             const int64_t k = k0 + tx;
             const bool kin = k < K;
-            sb[row][tx] = (kin && t0 + row < T) ? B[(t0 + row) * ldb + k] : 0.f;
-            sa0[row][tx] = (kin && n0 + row < n_out) ? A0[(n0 + row) * lda + k] : 0.f;
-            if constexpr (GLU) sa1[row][tx] = (kin && n0 + row < n_out) ? A1[(n0 + row) * lda + k] : 0.f;
+            sb[row][tx] = (kin && t0 + row < T) ? DASS_LD(&B[(t0 + row) * ldb + k]) : 0.f;
+            sa0[row][tx] = (kin && n0 + row < n_out) ? DASS_LD(&A0[(n0 + row) * lda + k]) : 0.f;
+            if constexpr (GLU) sa1[row][tx] = (kin && n0 + row < n_out) ? DASS_LD(&A1[(n0 + row) * lda + k]) : 0.f;
         }
         __syncthreads();
 #pragma unroll 8
@@ -61,9 +61,9 @@ mlp_forward_simt_kernel(const float *__restrict__ B, int64_t T, int64_t ldb,
             if constexpr (ACT == DASS_ACT_SILU) a = g / (1.0f + expf(-g));
             else if constexpr (ACT == DASS_ACT_GELU_TANH) a = 0.5f * g * (1.0f + tanhf(0.7978845608028654f * (g + 0.044715f * g * g * g)));
             else a = fmaxf(g, 0.0f);
-            out[t * ldo + n] = a * acc1[r];
+            DASS_ST(&out[t * ldo + n], a * acc1[r]);
         } else {
-            out[t * ldo + n] = acc0[r];
+            DASS_ST(&out[t * ldo + n], acc0[r]);
         }
     }
 }

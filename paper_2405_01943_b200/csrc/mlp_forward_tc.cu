@@ -87,11 +87,11 @@ __device__ __forceinline__ void fw_store_32(const FwParams &p, uint16_t *row, in
     if (p.vector_ok && n0 + 32 <= p.n_out) {
         uint4 *dst = reinterpret_cast<uint4 *>(row + n0);               // n0 is a multiple of 32
 #pragma unroll
-        for (int v = 0; v < 4; ++v) dst[v] = make_uint4(w[4 * v], w[4 * v + 1], w[4 * v + 2], w[4 * v + 3]);
+        for (int v = 0; v < 4; ++v) DASS_ST(&dst[v], make_uint4(w[4 * v], w[4 * v + 1], w[4 * v + 2], w[4 * v + 3]));
     } else {
 #pragma unroll
         for (int j = 0; j < 32; ++j)
-            if (n0 + j < p.n_out) row[n0 + j] = (uint16_t)((j & 1) ? (w[j >> 1] >> 16) : (w[j >> 1] & 0xffffu));
+            if (n0 + j < p.n_out) DASS_ST(&row[n0 + j], (uint16_t)((j & 1) ? (w[j >> 1] >> 16) : (w[j >> 1] & 0xffffu)));
     }
 }
 

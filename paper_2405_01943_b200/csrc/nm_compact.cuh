@@ -46,21 +46,21 @@ __device__ __forceinline__ void chunk_store_n(const Chunk<BF16> &c, void *base, 
     if constexpr (BF16) {
         uint16_t *p = static_cast<uint16_t *>(base) + off;
         if (vec && n == 8) {
-            __stcs(reinterpret_cast<uint4 *>(p), make_uint4(c.w[0], c.w[1], c.w[2], c.w[3]));
+            DASS_ST_CS(reinterpret_cast<uint4 *>(p), make_uint4(c.w[0], c.w[1], c.w[2], c.w[3]));
         } else if (vec && n == 4) {
-            __stcs(reinterpret_cast<uint2 *>(p), make_uint2(c.w[0], c.w[1]));
+            DASS_ST_CS(reinterpret_cast<uint2 *>(p), make_uint2(c.w[0], c.w[1]));
         } else {
-            for (int j = 0; j < n; ++j) p[j] = (uint16_t)chunk_bits_dyn<true>(c, j);
+            for (int j = 0; j < n; ++j) DASS_ST(&p[j], (uint16_t)chunk_bits_dyn<true>(c, j));
         }
     } else {
         uint32_t *p = static_cast<uint32_t *>(base) + off;
         if (vec && n == 8) {
-            __stcs(reinterpret_cast<uint4 *>(p), make_uint4(c.w[0], c.w[1], c.w[2], c.w[3]));
-            __stcs(reinterpret_cast<uint4 *>(p) + 1, make_uint4(c.w[4], c.w[5], c.w[6], c.w[7]));
+            DASS_ST_CS(reinterpret_cast<uint4 *>(p), make_uint4(c.w[0], c.w[1], c.w[2], c.w[3]));
+            DASS_ST_CS(reinterpret_cast<uint4 *>(p) + 1, make_uint4(c.w[4], c.w[5], c.w[6], c.w[7]));
         } else if (vec && n == 4) {
-            __stcs(reinterpret_cast<uint4 *>(p), make_uint4(c.w[0], c.w[1], c.w[2], c.w[3]));
+            DASS_ST_CS(reinterpret_cast<uint4 *>(p), make_uint4(c.w[0], c.w[1], c.w[2], c.w[3]));
         } else {
-            for (int j = 0; j < n; ++j) p[j] = chunk_bits_dyn<false>(c, j);
+            for (int j = 0; j < n; ++j) DASS_ST(&p[j], chunk_bits_dyn<false>(c, j));
         }
     }
 }

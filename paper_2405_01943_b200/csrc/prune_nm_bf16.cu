@@ -172,11 +172,11 @@ __device__ __forceinline__ uint32_t quad_transpose(uint32_t x, uint32_t sel1, ui
 __device__ __forceinline__ void store_row8(uint16_t *dst, const uint4 &v, int n, bool vec = true)
 {
     if (vec && n == 8) {
-        __stcs(reinterpret_cast<uint4 *>(dst), v);
+        DASS_ST_CS(reinterpret_cast<uint4 *>(dst), v);
     } else {
         for (int j = 0; j < n; ++j) {
             const uint32_t w = wsel(v, j >> 1);
-            dst[j] = (uint16_t)((j & 1) ? (w >> 16) : (w & 0xffffu));
+            DASS_ST(&dst[j], (uint16_t)((j & 1) ? (w >> 16) : (w & 0xffffu)));
         }
     }
 }
@@ -367,7 +367,7 @@ __device__ __forceinline__ void run_scales(const PruneParams &p, const Run<NORM_
     if constexpr (NORM_COLS) {
         for (int e = threadIdx.x; e < PN_COLS; e += PN_THREADS) {
             const int64_t c = (int64_t)run.line * PN_COLS + e;
-            cta_scales[e] = c < p.cols ? pn_scale_of(p.norm[c], p.scale_mode, p.alpha) : 0.0f;
+            cta_scales[e] = c < p.cols ? pn_scale_of(DASS_LD(&p.norm[c]), p.scale_mode, p.alpha) : 0.0f;
         }
         __syncthreads();
         const float4 a = reinterpret_cast<const float4 *>(cta_scales)[lane * 2];
@@ -375,7 +375,7 @@ __device__ __forceinline__ void run_scales(const PruneParams &p, const Run<NORM_
         s[0] = a.x; s[1] = a.y; s[2] = a.z; s[3] = a.w; s[4] = b.x; s[5] = b.y; s[6] = b.z; s[7] = b.w;
     } else {
         const int64_t r = (int64_t)run.line * PN_ROWS + (lane & 7);
-        const float mine = (run.f1 > run.f0 && r < p.rows) ? pn_scale_of(p.norm[r], p.scale_mode, p.alpha) : 0.0f;
+        const float mine = (run.f1 > run.f0 && r < p.rows) ? pn_scale_of(DASS_LD(&p.norm[r]), p.scale_mode, p.alpha) : 0.0f;
 #pragma unroll
         for (int q = 0; q < 8; ++q) s[q] = __shfl_sync(FULL_MASK, mine, q);
     }
@@ -457,7 +457,7 @@ __device__ __forceinline__ void rows_unit(const PruneParams &p, const uint4 *til
 #pragma unroll
             for (int h = 0; h < M / 4; ++h) {
                 const uint32_t word = quad_transpose(keep[h], sel1, sel2);
-                if (quad_live) kp[(g * M + 4 * h) * p.wpr] = word;
+                if (quad_live) DASS_ST(&kp[(g * M + 4 * h) * p.wpr], word);
             }
         }
         if (!FULL && nvalid == 0) continue;        // no shuffles below: lanes are independent from here on
@@ -470,7 +470,7 @@ __device__ __forceinline__ void rows_unit(const PruneParams &p, const uint4 *til
 #pragma unroll
             for (int k = 0; k < 4; ++k) wref(row, k) = wsel(v[q], k) & ~Z[q][k];
             if (want_pruned) {
-                if (FULL) __stcs(reinterpret_cast<uint4 *>(wp + (g * M + q) * p.ld), row);
+                if (FULL) DASS_ST_CS(reinterpret_cast<uint4 *>(wp + (g * M + q) * p.ld), row);
                 else store_row8(wp + (g * M + q) * p.ld, row, nvalid);
             }
         }
@@ -488,8 +488,8 @@ __device__ __forceinline__ void rows_unit(const PruneParams &p, const uint4 *til
                 wref(o1, k) = wsel(P[3], k) | (Z[3][k] & (wsel(P[2], k) | (Z[2][k] & wsel(P[1], k))));
             }
             if (FULL) {
-                __stcs(reinterpret_cast<uint4 *>(vg), o0);
-                __stcs(reinterpret_cast<uint4 *>(vg + p.vcols), o1);
+                DASS_ST_CS(reinterpret_cast<uint4 *>(vg), o0);
+                DASS_ST_CS(reinterpret_cast<uint4 *>(vg + p.vcols), o1);
             } else {
                 store_row8(vg, o0, nvalid, p.vec_ok != 0);
                 store_row8(vg + p.vcols, o1, nvalid, p.vec_ok != 0);
@@ -500,7 +500,7 @@ __device__ __forceinline__ void rows_unit(const PruneParams &p, const uint4 *til
             const uint32_t b0 = (~k0 & k1) & 0xffu, b1 = ~(k0 | k1) & 0xffu, b2 = (k3 | ~k2) & 0xffu, b3 = (k3 | k2) & 0xffu;
             uint32_t fields = spread_lut[b0] | (spread_lut[b1] << 1) | (spread_lut[b2] << 2) | (spread_lut[b3] << 3);
             if (!FULL) fields &= spread_lut[valid] * 15u;
-            p.meta[line * p.mwpl + (c0 >> 3)] = fields;
+            DASS_ST(&p.meta[line * p.mwpl + (c0 >> 3)], fields);
         } else {
             // Row q of the group goes to output row k = number of kept rows above it (bit-sliced over the 8
             // columns); for every possible (q, k) the byte "kept and count == k" becomes lane masks.
@@ -527,7 +527,7 @@ __device__ __forceinline__ void rows_unit(const PruneParams &p, const uint4 *til
             }
 #pragma unroll
             for (int k = 0; k < K; ++k) {
-                if (FULL) __stcs(reinterpret_cast<uint4 *>(vg + k * p.vcols), o[k]);
+                if (FULL) DASS_ST_CS(reinterpret_cast<uint4 *>(vg + k * p.vcols), o[k]);
                 else store_row8(vg + k * p.vcols, o[k], nvalid, p.vec_ok != 0);
             }
             // field of column j = its 8-bit keep mask (bit q = row q): the bit transpose of the keep bytes
@@ -538,8 +538,8 @@ __device__ __forceinline__ void rows_unit(const PruneParams &p, const uint4 *til
                 if (j < 4) f_lo |= colmask << (8 * j);
                 else f_hi |= colmask << (8 * (j - 4));
             }
-            p.meta[line * p.mwpl + (c0 >> 2)] = f_lo;
-            if (FULL || nvalid > 4) p.meta[line * p.mwpl + (c0 >> 2) + 1] = f_hi;
+            DASS_ST(&p.meta[line * p.mwpl + (c0 >> 2)], f_lo);
+            if (FULL || nvalid > 4) DASS_ST(&p.meta[line * p.mwpl + (c0 >> 2) + 1], f_hi);
         }
     }
 }
@@ -687,7 +687,7 @@ __device__ __forceinline__ void cols_unit(const PruneParams &p, const uint4 *til
         const bool row_live = FULL || (lane & 3) < nrows;
         if (want_mask) {
             const uint32_t word = quad_transpose(keep, sel1, sel2);
-            if (quad_live && row_live) kp[4 * h * p.wpr] = word;
+            if (quad_live && row_live) DASS_ST(&kp[4 * h * p.wpr], word);
         }
         uint32_t metab = 0u;               // byte i = metadata byte of row i
 #pragma unroll
@@ -697,7 +697,7 @@ __device__ __forceinline__ void cols_unit(const PruneParams &p, const uint4 *til
                     uint4 P;
 #pragma unroll
                     for (int k = 0; k < 4; ++k) wref(P, k) = wsel(v[i], k) & ~Z[i][k];
-                    if (FULL) __stcs(reinterpret_cast<uint4 *>(wp + (4 * h + i) * p.ld), P);
+                    if (FULL) DASS_ST_CS(reinterpret_cast<uint4 *>(wp + (4 * h + i) * p.ld), P);
                     else store_row8(wp + (4 * h + i) * p.ld, P, nvalid);
                 }
                 if (want_values) {
@@ -714,11 +714,11 @@ __device__ __forceinline__ void cols_unit(const PruneParams &p, const uint4 *til
                     }
                     uint16_t *dst = vp + (4 * h + i) * p.vcols;
                     if (FULL || (nout == 4 && p.vec_ok)) {
-                        __stcs(reinterpret_cast<uint2 *>(dst), make_uint2(o0, o1));
+                        DASS_ST_CS(reinterpret_cast<uint2 *>(dst), make_uint2(o0, o1));
                     } else {
                         for (int k = 0; k < nout; ++k) {
                             const uint32_t ow = k < 2 ? o0 : o1;
-                            dst[k] = (uint16_t)((k & 1) ? (ow >> 16) : (ow & 0xffffu));
+                            DASS_ST(&dst[k], (uint16_t)((k & 1) ? (ow >> 16) : (ow & 0xffffu)));
                         }
                     }
                 }
@@ -727,7 +727,7 @@ __device__ __forceinline__ void cols_unit(const PruneParams &p, const uint4 *til
         if (want_values) {
             // 2:4: nibbles pos_lo | pos_hi << 2; 4:8: the 8-bit keep mask of the group, i.e. the keep byte
             const uint32_t word = quad_transpose(M == 4 ? metab : keep, sel1, sel2);
-            if (quad_live && row_live) mp[4 * h * p.mwpl] = word;
+            if (quad_live && row_live) DASS_ST(&mp[4 * h * p.mwpl], word);
         }
     }
 }

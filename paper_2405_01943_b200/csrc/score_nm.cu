@@ -64,10 +64,10 @@ __global__ void __launch_bounds__(SCORE_THREADS) score_group_cols_kernel(const S
         if constexpr (NORM_COLS) {
 #pragma unroll
             for (int j = 0; j < 8; ++j)
-                sc[j] = j < nvalid ? (double)scale_from_norm(p.norm[c0 + j], p.scale_mode, p.alpha) : 0.0;
+                sc[j] = j < nvalid ? (double)scale_from_norm(DASS_LD(&p.norm[c0 + j]), p.scale_mode, p.alpha) : 0.0;
         } else {
             const int64_t r = rb * TILE_ROWS + lane;
-            if (r < p.rows) row_scale = scale_from_norm(p.norm[r], p.scale_mode, p.alpha);
+            if (r < p.rows) row_scale = scale_from_norm(DASS_LD(&p.norm[r]), p.scale_mode, p.alpha);
         }
 
         for (int i = 0; i < TILE_ROWS; i += UNROLL) {
@@ -107,12 +107,12 @@ __global__ void __launch_bounds__(SCORE_THREADS) score_group_cols_kernel(const S
                     else fb = compact_cols<BF16, M, false>(ch[u], keep, p.n_keep, nout, out);
                     const uint32_t mword = quad_pack_bytes(fb, lane);
                     if (r < p.rows && nvalid > 0) {
-                        if ((lane & 3) == 0) p.meta[r * p.mwpl + (c0 >> 5)] = mword;
+                        if ((lane & 3) == 0) DASS_ST(&p.meta[r * p.mwpl + (c0 >> 5)], mword);
                         chunk_store_n<BF16>(out, p.values, r * p.vcols + c0 / M * p.n_keep, nout, p.vec_ok != 0);
                     }
                 }
                 if (r < p.rows) {
-                    if (p.mask && (lane & 3) == 0 && nvalid > 0) p.mask[r * p.wpr + (c0 >> 5)] = word;
+                    if (p.mask && (lane & 3) == 0 && nvalid > 0) DASS_ST(&p.mask[r * p.wpr + (c0 >> 5)], word);
                     if (p.Wp && nvalid > 0) {
                         chunk_apply_mask<BF16>(ch[u], keep);
                         chunk_store<BF16>(ch[u], p.Wp, r * p.ld + c0, nvalid);
@@ -135,10 +135,10 @@ __device__ __forceinline__ void emit_rows(const ScoreParams &p, const Chunk<BF16
     uint32_t fields_lo, fields_hi;
     compact_rows<BF16, M, TWO_FOUR, MAXK>(ch, keep_row, p.n_keep, out, fields_lo, fields_hi);
     if constexpr (M == 4) {
-        p.meta[line * p.mwpl + (c0 >> 3)] = fields_lo;
+        DASS_ST(&p.meta[line * p.mwpl + (c0 >> 3)], fields_lo);
     } else {
-        p.meta[line * p.mwpl + (c0 >> 2)] = fields_lo;
-        if (nvalid > 4) p.meta[line * p.mwpl + (c0 >> 2) + 1] = fields_hi;
+        DASS_ST(&p.meta[line * p.mwpl + (c0 >> 2)], fields_lo);
+        if (nvalid > 4) DASS_ST(&p.meta[line * p.mwpl + (c0 >> 2) + 1], fields_hi);
     }
 #pragma unroll
     for (int k = 0; k < MAXK; ++k)
@@ -166,10 +166,10 @@ __global__ void __launch_bounds__(SCORE_THREADS) score_group_rows_kernel(const S
         if constexpr (NORM_COLS) {
 #pragma unroll
             for (int j = 0; j < 8; ++j)
-                sc[j] = j < nvalid ? (double)scale_from_norm(p.norm[c0 + j], p.scale_mode, p.alpha) : 0.0;
+                sc[j] = j < nvalid ? (double)scale_from_norm(DASS_LD(&p.norm[c0 + j]), p.scale_mode, p.alpha) : 0.0;
         } else {
             const int64_t r = rb * TILE_ROWS + lane;
-            if (r < p.rows) row_scale = scale_from_norm(p.norm[r], p.scale_mode, p.alpha);
+            if (r < p.rows) row_scale = scale_from_norm(DASS_LD(&p.norm[r]), p.scale_mode, p.alpha);
         }
 
         for (int g = 0; g < TILE_ROWS / M; ++g) {
@@ -212,7 +212,7 @@ __global__ void __launch_bounds__(SCORE_THREADS) score_group_rows_kernel(const S
 #pragma unroll
             for (int q = 0; q < M; ++q) {
                 const uint32_t word = quad_pack_bytes(keep_row[q], lane);
-                if (p.mask && (lane & 3) == 0 && nvalid > 0) p.mask[(r0 + q) * p.wpr + (c0 >> 5)] = word;
+                if (p.mask && (lane & 3) == 0 && nvalid > 0) DASS_ST(&p.mask[(r0 + q) * p.wpr + (c0 >> 5)], word);
                 if (p.Wp && nvalid > 0) {
                     chunk_apply_mask<BF16>(ch[q], keep_row[q]);
                     chunk_store<BF16>(ch[q], p.Wp, (r0 + q) * p.ld + c0, nvalid);

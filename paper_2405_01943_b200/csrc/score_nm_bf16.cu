@@ -49,6 +49,7 @@ __device__ __noinline__ float scale_of(float n, int mode, float alpha) { return 
 // 16-byte asynchronous copy global -> shared (src_bytes = 0 writes zeros and reads nothing)
 __device__ __forceinline__ void cp_async16(void *smem_dst, const void *gsrc, int src_bytes)
 {
+    if (src_bytes != 0 && !DASS_ACCESS_OK(gsrc, 16)) src_bytes = 0;     // checking build: an outside source reads as zeros
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;"
                  ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gsrc), "r"(src_bytes) : "memory");
 }
@@ -182,11 +183,11 @@ __device__ __forceinline__ uint32_t word_of(const uint4 &v, int k) { return k ==
 __device__ __forceinline__ void store_chunk(uint16_t *dst, const uint4 &v, int nvalid)
 {
     if (nvalid == 8) {
-        __stcs(reinterpret_cast<uint4 *>(dst), v);
+        DASS_ST_CS(reinterpret_cast<uint4 *>(dst), v);
     } else {
         for (int j = 0; j < nvalid; ++j) {
             const uint32_t w = word_of(v, j >> 1);
-            dst[j] = (uint16_t)((j & 1) ? (w >> 16) : (w & 0xffffu));
+            DASS_ST(&dst[j], (uint16_t)((j & 1) ? (w >> 16) : (w & 0xffffu)));
         }
     }
 }
@@ -288,7 +289,7 @@ __global__ void __launch_bounds__(F_THREADS, M == 8 ? 2 : F_MIN_BLOCKS) score_ro
             if constexpr (NORM_COLS) {
 #pragma unroll
                 for (int j = 0; j < 8; ++j)
-                    sc[j] = j < nvalid ? scale_of(p.norm[c0 + j], p.scale_mode, p.alpha) : 0.0f;
+                    sc[j] = j < nvalid ? scale_of(DASS_LD(&p.norm[c0 + j]), p.scale_mode, p.alpha) : 0.0f;
             }
         }
         if constexpr (!NORM_COLS) {
@@ -296,7 +297,7 @@ __global__ void __launch_bounds__(F_THREADS, M == 8 ? 2 : F_MIN_BLOCKS) score_ro
             if (base != cached_base) {
                 cached_base = base;
                 const int64_t r = base + lane;
-                lane_scale = r < p.rows ? scale_of(p.norm[r], p.scale_mode, p.alpha) : 0.0f;
+                lane_scale = r < p.rows ? scale_of(DASS_LD(&p.norm[r]), p.scale_mode, p.alpha) : 0.0f;
             }
         }
 
@@ -348,7 +349,7 @@ __global__ void __launch_bounds__(F_THREADS, M == 8 ? 2 : F_MIN_BLOCKS) score_ro
         for (int q = 0; q < M; ++q) {
             const uint32_t keep = K[q] & valid;
             const uint32_t word = quad_pack_bytes(keep, lane);
-            if (p.mask && (lane & 3) == 0 && nvalid > 0) p.mask[(r0 + q) * p.wpr + (c0 >> 5)] = word;
+            if (p.mask && (lane & 3) == 0 && nvalid > 0) DASS_ST(&p.mask[(r0 + q) * p.wpr + (c0 >> 5)], word);
             if (p.Wp && nvalid > 0) {
                 apply_keep_byte(v[q], keep);
                 store_chunk(p.Wp + (r0 + q) * p.ld + c0, v[q], nvalid);
@@ -404,7 +405,7 @@ __global__ void __launch_bounds__(F_THREADS, 3) score_cols_bf16_kernel(const Sco
             if constexpr (NORM_COLS) {
 #pragma unroll
                 for (int j = 0; j < 8; ++j)
-                    sc[j] = j < nvalid ? scale_of(p.norm[c0 + j], p.scale_mode, p.alpha) : 0.0f;
+                    sc[j] = j < nvalid ? scale_of(DASS_LD(&p.norm[c0 + j]), p.scale_mode, p.alpha) : 0.0f;
             }
         }
         if constexpr (!NORM_COLS) {
@@ -412,7 +413,7 @@ __global__ void __launch_bounds__(F_THREADS, 3) score_cols_bf16_kernel(const Sco
             if (base != cached_base) {
                 cached_base = base;
                 const int64_t r = base + lane;
-                lane_scale = r < p.rows ? scale_of(p.norm[r], p.scale_mode, p.alpha) : 0.0f;
+                lane_scale = r < p.rows ? scale_of(DASS_LD(&p.norm[r]), p.scale_mode, p.alpha) : 0.0f;
             }
         }
 
@@ -470,7 +471,7 @@ __global__ void __launch_bounds__(F_THREADS, 3) score_cols_bf16_kernel(const Sco
             const uint32_t keep = row_keep[i] & valid;
             const uint32_t word = quad_pack_bytes(keep, lane);
             if (r0 + i < p.rows && nvalid > 0) {
-                if (p.mask && (lane & 3) == 0) p.mask[(r0 + i) * p.wpr + (c0 >> 5)] = word;
+                if (p.mask && (lane & 3) == 0) DASS_ST(&p.mask[(r0 + i) * p.wpr + (c0 >> 5)], word);
                 if (p.Wp) {
                     apply_keep_byte(v[i], keep);
                     store_chunk(p.Wp + (r0 + i) * p.ld + c0, v[i], nvalid);

@@ -56,8 +56,8 @@ __global__ void scale_vector_kernel(const float *__restrict__ norm, int64_t n, i
                                     float *__restrict__ out)
 {
     const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (i < n) out[i] = scale_from_norm(norm[i], mode, alpha);
-    else if (i < npad) out[i] = 0.0f;
+    if (i < n) DASS_ST(&out[i], scale_from_norm(DASS_LD(&norm[i]), mode, alpha));
+    else if (i < npad) DASS_ST(&out[i], 0.0f);
 }
 
 // ---------------------------------------------------------------- radix select on a three-part key
@@ -460,10 +460,10 @@ __global__ void __launch_bounds__(ROW_THREADS) select_rows_kernel(const SelectPa
         uint4 *dst = reinterpret_cast<uint4 *>(line_mem);
         const int64_t nvec = (p.L + EPV - 1) / EPV;
         for (int64_t v = tid; v < (int64_t)(p.lpad / EPV); v += ROW_THREADS)
-            dst[v] = v < nvec ? __ldcs(src + v) : make_uint4(0u, 0u, 0u, 0u);
+            dst[v] = v < nvec ? DASS_LD_CS(src + v) : make_uint4(0u, 0u, 0u, 0u);
     }
     if (tid == 0) { line_init(st, p.k); s_long = 0u; }
-    const float line_scale = p.scale_along_line ? 0.0f : p.scale[row];
+    const float line_scale = p.scale_along_line ? 0.0f : DASS_LD(&p.scale[row]);
 
     // the 8 signed weights and scales of chunk q
     auto fetch = [&](int64_t q, float (&w)[8], float (&sc)[8]) {
@@ -472,8 +472,8 @@ __global__ void __launch_bounds__(ROW_THREADS) select_rows_kernel(const SelectPa
 #pragma unroll
         for (int j = 0; j < 8; ++j) w[j] = chunk_float<BF16>(ch, j);
         if (p.scale_along_line) {
-            const float4 s0 = __ldg(reinterpret_cast<const float4 *>(p.scale + q * 8));
-            const float4 s1 = __ldg(reinterpret_cast<const float4 *>(p.scale + q * 8) + 1);   // the vector is padded to 8
+            const float4 s0 = DASS_LD_G(reinterpret_cast<const float4 *>(p.scale + q * 8));
+            const float4 s1 = DASS_LD_G(reinterpret_cast<const float4 *>(p.scale + q * 8) + 1);   // the vector is padded to 8
             sc[0] = s0.x; sc[1] = s0.y; sc[2] = s0.z; sc[3] = s0.w; sc[4] = s1.x; sc[5] = s1.y; sc[6] = s1.z; sc[7] = s1.w;
         } else {
 #pragma unroll
@@ -511,7 +511,7 @@ __global__ void __launch_bounds__(ROW_THREADS) select_rows_kernel(const SelectPa
             float wf;
             if constexpr (BF16) wf = __uint_as_float((uint32_t)line_mem[e] << 16);
             else wf = __uint_as_float(line_mem[e]);
-            samp[i] = product_key(wf, p.scale_along_line ? __ldg(p.scale + e) : line_scale);
+            samp[i] = product_key(wf, p.scale_along_line ? DASS_LD_G(p.scale + e) : line_scale);
         }
         __syncthreads();
         sort_samples<1, ROW_THREADS>(samp, tid);
@@ -607,7 +607,7 @@ __global__ void __launch_bounds__(ROW_THREADS) select_rows_kernel(const SelectPa
         const int64_t e0 = q * 8;
         const int64_t left = p.L - e0;
         const int nvalid = left >= 8 ? 8 : (int)left;
-        if (p.mask) reinterpret_cast<uint8_t *>(p.mask + row * p.wpr)[q] = (uint8_t)keep;   // byte q = columns 8q..8q+7
+        if (p.mask) DASS_ST(&reinterpret_cast<uint8_t *>(p.mask + row * p.wpr)[q], (uint8_t)keep);   // byte q = columns 8q..8q+7
         if (p.Wp) {
             Chunk<BF16> ch;
             chunk_from<BF16>(ch, reinterpret_cast<const uint4 *>(line_mem + e0));
@@ -645,7 +645,7 @@ __global__ void __launch_bounds__(COL_THREADS, 1) select_cols_kernel(const Selec
     if (tid == 0) s_long = 0u;
     float col_scale[COL_LINES];
 #pragma unroll
-    for (int j = 0; j < COL_LINES; ++j) col_scale[j] = (!p.scale_along_line && j < nl) ? p.scale[c0 + j] : 0.0f;
+    for (int j = 0; j < COL_LINES; ++j) col_scale[j] = (!p.scale_along_line && j < nl) ? DASS_LD(&p.scale[c0 + j]) : 0.0f;
 
     // One pass over the strip: UNROLL rows per thread are loaded before any is counted, so that several
     // L2 round trips are in flight per thread.
@@ -665,15 +665,15 @@ __global__ void __launch_bounds__(COL_THREADS, 1) select_cols_kernel(const Selec
                     // the row pitch is a multiple of 16 bytes and c0 of 8 elements: aligned vectors inside the row's
                     // pitch (an f32 row is padded to 4 elements only: its second vector is read when it holds a column)
                     const uint4 *src = reinterpret_cast<const uint4 *>(strip + r * p.ld);
-                    const uint4 v0 = __ldg(src);
+                    const uint4 v0 = DASS_LD_G(src);
                     ch[u].w[0] = v0.x; ch[u].w[1] = v0.y; ch[u].w[2] = v0.z; ch[u].w[3] = v0.w;
                     if constexpr (!BF16) {
                         if (nl > 4) {
-                            const uint4 v1 = __ldg(src + 1);
+                            const uint4 v1 = DASS_LD_G(src + 1);
                             ch[u].w[4] = v1.x; ch[u].w[5] = v1.y; ch[u].w[6] = v1.z; ch[u].w[7] = v1.w;
                         }
                     }
-                    if (p.scale_along_line) row_scale[u] = __ldg(p.scale + r);
+                    if (p.scale_along_line) row_scale[u] = DASS_LD_G(p.scale + r);
                 }
             }
 #pragma unroll
@@ -701,12 +701,12 @@ __global__ void __launch_bounds__(COL_THREADS, 1) select_cols_kernel(const Selec
         // loads one row of the strip (the vector loads of count_pass)
         auto load_row = [&](int64_t r, Chunk<BF16> &ch) {
             const uint4 *src = reinterpret_cast<const uint4 *>(strip + r * p.ld);
-            const uint4 v0 = __ldg(src);
+            const uint4 v0 = DASS_LD_G(src);
             ch.w[0] = v0.x; ch.w[1] = v0.y; ch.w[2] = v0.z; ch.w[3] = v0.w;
             if constexpr (!BF16) {
                 ch.w[4] = ch.w[5] = ch.w[6] = ch.w[7] = 0u;
                 if (nl > 4) {
-                    const uint4 v1 = __ldg(src + 1);
+                    const uint4 v1 = DASS_LD_G(src + 1);
                     ch.w[4] = v1.x; ch.w[5] = v1.y; ch.w[6] = v1.z; ch.w[7] = v1.w;
                 }
             }
@@ -715,7 +715,7 @@ __global__ void __launch_bounds__(COL_THREADS, 1) select_cols_kernel(const Selec
             const int64_t r = ((int64_t)i * p.L) / SAMPLE;
             Chunk<BF16> ch;
             load_row(r, ch);
-            const float rs = p.scale_along_line ? __ldg(p.scale + r) : 0.0f;
+            const float rs = p.scale_along_line ? DASS_LD_G(p.scale + r) : 0.0f;
 #pragma unroll
             for (int j = 0; j < COL_LINES; ++j)
                 samp[j * SAMPLE + i] = product_key(chunk_float<BF16>(ch, j), p.scale_along_line ? rs : col_scale[j]);
@@ -746,7 +746,7 @@ __global__ void __launch_bounds__(COL_THREADS, 1) select_cols_kernel(const Selec
                     row_scale[u] = 0.0f;
                     if (r < p.L) {
                         load_row(r, ch[u]);
-                        if (p.scale_along_line) row_scale[u] = __ldg(p.scale + r);
+                        if (p.scale_along_line) row_scale[u] = DASS_LD_G(p.scale + r);
                     }
                 }
 #pragma unroll
@@ -793,7 +793,7 @@ __global__ void __launch_bounds__(COL_THREADS, 1) select_cols_kernel(const Selec
                         row_scale[u] = 0.0f;
                         if (r < p.L) {
                             load_row(r, ch[u]);
-                            if (p.scale_along_line) row_scale[u] = __ldg(p.scale + r);
+                            if (p.scale_along_line) row_scale[u] = DASS_LD_G(p.scale + r);
                         }
                     }
 #pragma unroll
@@ -851,7 +851,7 @@ __global__ void __launch_bounds__(COL_THREADS, 1) select_cols_kernel(const Selec
         if (!sched_next<BF16>(sc, s_long != 0u, p.idx_bits)) break;
         if (was_rounded && s_long && tid < COL_LINES) st[tid].base = 0ull;   // read again only after the next barrier
     }
-    if (tid < nl) p.results[c0 + tid] = fl[tid].ok ? fl[tid].res : line_result(st[tid], idx_top);
+    if (tid < nl) DASS_ST(&p.results[c0 + tid], fl[tid].ok ? fl[tid].res : line_result(st[tid], idx_top));
 }
 
 // ---------------------------------------------------------------- column lines: streaming emit
@@ -873,7 +873,8 @@ struct EmitParams {
 __device__ __noinline__ bool exact_tie_keeps(const LineResult *res, float a, float s, int64_t r)
 {
     const unsigned long long k64 = (unsigned long long)__double_as_longlong((double)a * (double)s);
-    return k64 > res->tau64 || (k64 == res->tau64 && (long long)r <= res->cut);
+    const LineResult t = DASS_LD(res);
+    return k64 > t.tau64 || (k64 == t.tau64 && (long long)r <= t.cut);
 }
 
 template <bool BF16>
@@ -896,9 +897,9 @@ __global__ void __launch_bounds__(256, 4) select_emit_cols_kernel(const EmitPara
             tau[j] = 0xffffffffu;
             sc[j] = 0.0f;
             if (j < nvalid) {
-                tau[j] = p.results[c0 + j].tau32;
-                exact_cols |= (p.results[c0 + j].exact ? 1u : 0u) << j;
-                if (!p.scale_per_row) sc[j] = p.scale[c0 + j];
+                tau[j] = DASS_LD(&p.results[c0 + j].tau32);
+                exact_cols |= (DASS_LD(&p.results[c0 + j].exact) ? 1u : 0u) << j;
+                if (!p.scale_per_row) sc[j] = DASS_LD(&p.scale[c0 + j]);
             }
         }
         if ((cb + 1) * 256 > p.cols) {
@@ -909,7 +910,7 @@ __global__ void __launch_bounds__(256, 4) select_emit_cols_kernel(const EmitPara
                 Chunk<BF16> ch;
                 if (nvalid > 0) chunk_load<BF16>(ch, p.W, r * p.ld + c0, nvalid);
                 else chunk_zero<BF16>(ch);
-                const float rs = p.scale_per_row ? __ldg(p.scale + r) : 0.0f;
+                const float rs = p.scale_per_row ? DASS_LD_G(p.scale + r) : 0.0f;
                 uint32_t keep = 0u;
 #pragma unroll
                 for (int j = 0; j < 8; ++j) {
@@ -920,7 +921,7 @@ __global__ void __launch_bounds__(256, 4) select_emit_cols_kernel(const EmitPara
                     if (key == tau[j] && j < nvalid) {
                         k = true;                           // products equal to the threshold stay ...
                         if ((exact_cols >> j) & 1u) {       // ... unless the exact stage had to split them
-                            const LineResult res = p.results[c0 + j];
+                            const LineResult res = DASS_LD(&p.results[c0 + j]);
                             const unsigned long long k64 = (unsigned long long)__double_as_longlong((double)a * (double)s);
                             k = k64 > res.tau64 || (k64 == res.tau64 && (long long)r <= res.cut);
                         }
@@ -929,7 +930,7 @@ __global__ void __launch_bounds__(256, 4) select_emit_cols_kernel(const EmitPara
                 }
                 const uint32_t word = quad_pack_bytes(keep, lane);
                 if (nvalid > 0) {
-                    if (p.mask && (lane & 3) == 0) p.mask[r * p.wpr + (c0 >> 5)] = word;
+                    if (p.mask && (lane & 3) == 0) DASS_ST(&p.mask[r * p.wpr + (c0 >> 5)], word);
                     if (p.Wp) {
                         chunk_apply_mask<BF16>(ch, keep);
                         chunk_store<BF16>(ch, p.Wp, r * p.ld + c0, nvalid);
@@ -951,7 +952,7 @@ __global__ void __launch_bounds__(256, 4) select_emit_cols_kernel(const EmitPara
                 const int64_t r = rbase + u;
                 if (r < p.rows) chunk_load<BF16>(chs[u], p.W, r * p.ld + c0, 8);
                 else chunk_zero<BF16>(chs[u]);
-                rss[u] = (p.scale_per_row && r < p.rows) ? __ldg(p.scale + r) : 0.0f;
+                rss[u] = (p.scale_per_row && r < p.rows) ? DASS_LD_G(p.scale + r) : 0.0f;
             }
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
@@ -969,16 +970,16 @@ __global__ void __launch_bounds__(256, 4) select_emit_cols_kernel(const EmitPara
                 }
                 const uint32_t word = quad_pack_bytes(keep, lane);
                 if (r < p.rows) {
-                    if (p.mask && (lane & 3) == 0) p.mask[r * p.wpr + (c0 >> 5)] = word;
+                    if (p.mask && (lane & 3) == 0) DASS_ST(&p.mask[r * p.wpr + (c0 >> 5)], word);
                     if (p.Wp) {
                         chunk_apply_mask<BF16>(chs[u], keep);
                         if constexpr (BF16) {
-                            __stcs(reinterpret_cast<uint4 *>(static_cast<uint16_t *>(p.Wp) + r * p.ld + c0),
+                            DASS_ST_CS(reinterpret_cast<uint4 *>(static_cast<uint16_t *>(p.Wp) + r * p.ld + c0),
                                    make_uint4(chs[u].w[0], chs[u].w[1], chs[u].w[2], chs[u].w[3]));
                         } else {
                             uint4 *dst = reinterpret_cast<uint4 *>(static_cast<uint32_t *>(p.Wp) + r * p.ld + c0);
-                            __stcs(dst, make_uint4(chs[u].w[0], chs[u].w[1], chs[u].w[2], chs[u].w[3]));
-                            __stcs(dst + 1, make_uint4(chs[u].w[4], chs[u].w[5], chs[u].w[6], chs[u].w[7]));
+                            DASS_ST_CS(dst, make_uint4(chs[u].w[0], chs[u].w[1], chs[u].w[2], chs[u].w[3]));
+                            DASS_ST_CS(dst + 1, make_uint4(chs[u].w[4], chs[u].w[5], chs[u].w[6], chs[u].w[7]));
                         }
                     }
                 }
@@ -1109,6 +1110,13 @@ extern "C" dass_status dass_select_unstructured(const void *W, int64_t rows, int
     if (line_is_row && select_row_smem_bytes(L, bf16) > (size_t)220 * 1024) return DASS_ERR_UNSUPPORTED;   // a row line is cached in shared memory
     const int64_t n_prune = (int64_t)std::floor(sparsity * (double)L);
     const uint32_t k = (uint32_t)(L - n_prune);
+    DASS_BOUNDS_SCOPE(bs);
+    DASS_BOUNDS_ADD(bs, W, (size_t)rows * ld * (bf16 ? 2 : 4));
+    DASS_BOUNDS_ADD(bs, W_pruned, (size_t)rows * ld * (bf16 ? 2 : 4));
+    DASS_BOUNDS_ADD(bs, norm, (size_t)(norm_axis == DASS_AXIS_ROWS ? rows : cols) * sizeof(float));
+    DASS_BOUNDS_ADD(bs, mask_bits, (size_t)rows * ((cols + 31) / 32) * sizeof(uint32_t));
+    DASS_BOUNDS_ADD(bs, workspace, workspace_bytes);
+    DASS_BOUNDS_COMMIT(bs, static_cast<cudaStream_t>(cuda_stream));
     if (select_unstructured_launch(W, rows, cols, ld, bf16, norm, norm_axis == DASS_AXIS_COLS, alpha, k, line_is_row,
                                    mask_bits, W_pruned, workspace,
                                    static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
