@@ -76,7 +76,16 @@ def _git_blob_sha(path):
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per launch, from ncu captures summarised under profiles/.
 # Each entry names its summary and the git blob id of the kernel source it was captured from; when the source has
 # changed since, the number is withheld (reported as null) instead of going stale.
-NCU_DRAM_BYTES = {}
+NCU_DRAM_BYTES = {
+    "llama2_70b": {
+        "calib": {"bytes": 4 * (29.607549696e9 + 15.025152e6), "profile": "profiles/calib_tc2_kernel_llama2_70b_T65536_dram.md",
+                  "source": "paper_2405_01943_b200/csrc/calib_tc2.cu", "blob": "729748d82f305308578b4f36418f5fcceedbd567",
+                  "how": "one launch at T = 65536 (one group of 16 interleaved bands) x 4: the full launch repeats that group four times"},
+        "prune": {"bytes": (2 * (470.0 + 706.4) + 470.0 + 708.5) * 1e6, "profile": "profiles/prune_bf16_kernels_llama2_70b_matrices.md",
+                  "source": "paper_2405_01943_b200/csrc/prune_nm_bf16.cu", "blob": "fcc444888ad6e9461fd7ad586f333d7f33683726",
+                  "how": "the three launches of one step (gate, up, down) on the full-size matrices"},
+    },
+}
 
 
 def ncu_traffic(cfg_name, key):
