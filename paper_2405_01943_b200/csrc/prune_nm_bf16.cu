@@ -26,160 +26,27 @@
 //     products (rare on real data, always correct).
 // Every mbarrier wait is bounded; a wait that runs out records DASS_ERR_TIMEOUT in a status word of the library
 // (read by dass_prune_status) and the warp returns.
-#include "tc_common.cuh"
+#include "stream_units.cuh"
 
 namespace dass {
 
-struct PruneParams {
+struct PruneParams : UnitGrid {
     const uint16_t *W;
     uint16_t *Wp;        // nullable
     uint32_t *mask;      // nullable
     uint16_t *values;    // nullable (then meta is null too)
     uint32_t *meta;
     const float *norm;
-    int64_t rows, cols, ld;
+    int64_t ld;
     int64_t wpr;         // mask words per row
     int64_t vcols;       // elements per row of the values matrix
     int64_t mwpl;        // metadata words per line
-    int64_t strips, blocks;          // 256-column strips, 8-row blocks
-    int64_t fast;        // units along the direction a warp walks (the scales stay the same along it)
-    int runs;            // a line of `fast` units is cut into this many near-equal runs, one per warp
-    int ctas_per_line;   // per-column scales: CTAs that share one strip (runs / warps per CTA, rounded up)
     int scale_mode;
     float alpha;
     int vec_ok;          // value rows start 16-byte (row groups) / 8-byte (column groups) aligned
-    uint32_t box_bytes;  // bytes of one TMA box (box columns x box rows x 2)
-    uint32_t pitch16;    // row pitch of a box in shared memory, in 16-byte vectors
 };
 
 namespace {
-
-constexpr int PN_THREADS = 128;
-constexpr int PN_MIN_BLOCKS = 4;     // 16 warps per SM at up to 128 registers
-constexpr int PN_COLS = 256;
-constexpr int PN_ROWS = 8;
-
-// Out of line: the double-precision sqrt / pow sequences run once per strip or per 32 rows only.
-__device__ __noinline__ float pn_scale_of(float n, int mode, float alpha) { return scale_from_norm(n, mode, alpha); }
-
-__device__ __forceinline__ uint32_t pn_prmt(uint32_t a, uint32_t b, uint32_t sel)
-{
-    uint32_t d;
-    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
-    return d;
-}
-
-__device__ __forceinline__ float max3f(float a, float b, float c)
-{
-    float d;
-    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
-    return d;
-}
-
-__device__ __forceinline__ uint32_t wsel(const uint4 &v, int k) { return k == 0 ? v.x : k == 1 ? v.y : k == 2 ? v.z : v.w; }
-__device__ __forceinline__ uint32_t &wref(uint4 &v, int k) { return k == 0 ? v.x : k == 1 ? v.y : k == 2 ? v.z : v.w; }
-
-// fl32(|low bf16 of word| * s) and the same for the high one.  The low half is moved up with a multiply so that it
-// runs beside the float pipe rather than on the logic pipe.
-__device__ __forceinline__ float prod_lo(uint32_t word, float s) { return fabsf(__uint_as_float(word * 65536u)) * s; }
-__device__ __forceinline__ float prod_hi(uint32_t word, float s) { return fabsf(__uint_as_float(word & 0xffff0000u)) * s; }
-
-// Second largest of four.
-__device__ __forceinline__ float cut_2of4(float a, float b, float c, float d)
-{
-    const float h1 = fmaxf(a, b), l1 = fminf(a, b), h2 = fmaxf(c, d), l2 = fminf(c, d);
-    return max3f(fminf(h1, h2), l1, l2);
-}
-
-__device__ __forceinline__ void sort4_desc(float &a, float &b, float &c, float &d)
-{
-    const float h1 = fmaxf(a, b), l1 = fminf(a, b), h2 = fmaxf(c, d), l2 = fminf(c, d);
-    const float m = fminf(h1, h2), l = fmaxf(l1, l2);
-    a = fmaxf(h1, h2);
-    b = fmaxf(m, l);
-    c = fminf(m, l);
-    d = fminf(l1, l2);
-}
-
-// Fourth largest of eight: both halves sorted, then the merge rule "the k-th largest of two sorted lists is the
-// largest of min(a_i, b_(k-2-i)) and of a_(k-1), b_(k-1)".
-__device__ __forceinline__ float cut_4of8(const float (&x)[8])
-{
-    float a0 = x[0], a1 = x[1], a2 = x[2], a3 = x[3], b0 = x[4], b1 = x[5], b2 = x[6], b3 = x[7];
-    sort4_desc(a0, a1, a2, a3);
-    sort4_desc(b0, b1, b2, b3);
-    return max3f(max3f(a3, b3, fminf(a0, b2)), fminf(a1, b1), fminf(a2, b0));
-}
-
-template <int M>
-__device__ __forceinline__ float cut_of(const float (&x)[M])
-{
-    if constexpr (M == 4) return cut_2of4(x[0], x[1], x[2], x[3]);
-    else return cut_4of8(x);
-}
-
-// Lane mask of a word from the differences of its two elements: 0xffff where the difference is negative.
-__device__ __forceinline__ uint32_t pruned_lanes(float d_lo, float d_hi)
-{
-    return pn_prmt(__float_as_uint(d_lo), __float_as_uint(d_hi), 0xFFBBu);
-}
-
-// Bytes (bit j = column j) of the lane-mask words of two rows, in the low 16 bits of the result (row a in byte 0,
-// row b in byte 1).  Even columns sit in the low lanes and land on their bit directly; odd columns sit in the high
-// lanes, are picked 16 bits up and folded down at the end.
-__device__ __forceinline__ uint32_t bytes_of_lanes2(const uint32_t (&za)[4], const uint32_t (&zb)[4])
-{
-    uint32_t x = za[0] & 0x00020001u;
-    x |= za[1] & 0x00080004u;
-    x |= za[2] & 0x00200010u;
-    x |= za[3] & 0x00800040u;
-    x |= zb[0] & 0x02000100u;
-    x |= zb[1] & 0x08000400u;
-    x |= zb[2] & 0x20001000u;
-    x |= zb[3] & 0x80004000u;
-    return x | (x >> 16);
-}
-
-// "Pruned" bytes of four rows in one word (byte i = row i).
-__device__ __forceinline__ uint32_t bytes_of_lanes4(const uint32_t (&z0)[4], const uint32_t (&z1)[4], const uint32_t (&z2)[4],
-                                                    const uint32_t (&z3)[4])
-{
-    return pn_prmt(bytes_of_lanes2(z0, z1), bytes_of_lanes2(z2, z3), 0x5410u);
-}
-
-// 16-bit lane masks (0xffff per set bit) of an 8-bit byte: bit j -> sign of byte j, then sign-replicating permutes.
-__device__ __forceinline__ void lanes_of_byte(uint32_t byte, uint32_t (&m)[4])
-{
-    const uint32_t zlo = (byte & 0xfu) * 0x10204080u;
-    const uint32_t zhi = ((byte >> 4) & 0xfu) * 0x10204080u;
-    m[0] = pn_prmt(zlo, 0u, 0x9988u);
-    m[1] = pn_prmt(zlo, 0u, 0xbbaau);
-    m[2] = pn_prmt(zhi, 0u, 0x9988u);
-    m[3] = pn_prmt(zhi, 0u, 0xbbaau);
-}
-
-// 4 x 4 byte transpose across a quad of lanes: on entry byte i of x belongs to row i (this lane's 8 columns); on
-// return lane k of the quad holds the word of row k (byte l from lane l of the quad).  Whole warp must call.
-__device__ __forceinline__ uint32_t quad_transpose(uint32_t x, uint32_t sel1, uint32_t sel2)
-{
-    const uint32_t y = __shfl_xor_sync(FULL_MASK, x, 1);
-    const uint32_t z = pn_prmt(x, y, sel1);
-    const uint32_t y2 = __shfl_xor_sync(FULL_MASK, z, 2);
-    return pn_prmt(z, y2, sel2);
-}
-
-// Stores the first n of a lane's 8 elements; one 16-byte store when all 8 exist and the address is known to be aligned.
-__device__ __forceinline__ void store_row8(uint16_t *dst, const uint4 &v, int n, bool vec = true)
-{
-    if (vec && n == 8) {
-        DASS_ST_CS(reinterpret_cast<uint4 *>(dst), v);
-    } else {
-        for (int j = 0; j < n; ++j) {
-            const uint32_t w = wsel(v, j >> 1);
-            DASS_ST(&dst[j], (uint16_t)((j & 1) ? (w >> 16) : (w & 0xffffu)));
-        }
-    }
-}
 
 // ---------------------------------------------------------------- exact selection (rare path)
 template <int R> struct Tile { uint4 v[R]; };
@@ -242,121 +109,6 @@ __device__ __forceinline__ uint32_t spread_bits(uint32_t b)
 
 // nibble made of bit j of each of the four bytes of x (byte a -> bit a)
 __device__ __forceinline__ uint32_t gather_bit4(uint32_t x, int j) { return (((x >> j) & 0x01010101u) * 0x10204080u) >> 28; }
-
-// ---------------------------------------------------------------- work decomposition
-// A unit is 8 rows x 256 columns.  A warp walks a run of consecutive units in the direction along which its
-// scales stay the same: down a strip when the scales belong to columns, across the strips of one 8-row block when
-// they belong to rows.  A line of units along that direction is cut into p.runs near-equal runs.  CTAs are small
-// (4 warps, a few units per warp) and numerous, so the hardware's block scheduler evens out the SMs.
-//   per-column scales: the warps of a CTA take consecutive runs of ONE strip and share its 256 scales through
-//                      shared memory;
-//   per-row scales:    the warps of a CTA take the same strip range at consecutive row blocks.
-constexpr int PN_STAGES = 3;
-constexpr uint32_t PN_SLOT_BYTES = PN_ROWS * PN_COLS * 2;           // 4 KB: one full box
-constexpr uint32_t PN_WARPS = PN_THREADS / 32;
-constexpr uint32_t PN_SMEM_BYTES = PN_WARPS * PN_STAGES * PN_SLOT_BYTES + PN_WARPS * PN_STAGES * 8 + 128;
-constexpr unsigned long long PN_WAIT_NS = 2000000000ull;            // a wait gives up after 2 s
-
-__device__ int g_prune_status = 0;     // DASS_OK or DASS_ERR_TIMEOUT; read and cleared through dass_prune_status
-
-template <bool NORM_COLS>
-struct Run {
-    int line;        // the fixed index: strip (per-column scales) or row block (per-row scales)
-    int f0, f1;      // units [f0, f1) along the walking direction; empty for a warp without work
-    __device__ __forceinline__ void set(const PruneParams &p, int warp_in_cta)
-    {
-        int r;
-        bool live;
-        if constexpr (NORM_COLS) {
-            line = (int)(blockIdx.x / (unsigned)p.ctas_per_line);
-            r = (int)(blockIdx.x % (unsigned)p.ctas_per_line) * (int)PN_WARPS + warp_in_cta;
-            live = r < p.runs;
-        } else {
-            line = (int)(blockIdx.x / (unsigned)p.runs) * (int)PN_WARPS + warp_in_cta;
-            r = (int)(blockIdx.x % (unsigned)p.runs);
-            live = line < p.blocks;
-        }
-        f0 = live ? (int)((int64_t)r * p.fast / p.runs) : 0;
-        f1 = live ? (int)((int64_t)(r + 1) * p.fast / p.runs) : 0;
-    }
-    __device__ __forceinline__ int strip(int f) const { return NORM_COLS ? line : f; }
-    __device__ __forceinline__ int blk(int f) const { return NORM_COLS ? f : line; }
-};
-
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int x, int y)
-{
-    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-                 ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(x), "r"(y) : "memory");
-}
-
-// Bounded wait of the whole warp on one of its slots.  False after PN_WAIT_NS.
-__device__ __forceinline__ bool slot_wait(uint32_t bar, uint32_t parity)
-{
-    if (mbar_try_wait(bar, parity)) return true;
-    const unsigned long long t0 = global_ns();
-    for (uint32_t spin = 1; spin < (1u << 30); ++spin) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if ((spin & 63u) == 0 && global_ns() - t0 > PN_WAIT_NS) return false;
-    }
-    return false;
-}
-
-// The TMA-fed ring of a warp: PN_STAGES slots of one box each, one mbarrier per slot.
-template <bool NORM_COLS>
-struct UnitRing {
-    uint32_t slots, bars;            // shared-memory addresses of this warp's slots and barriers
-    const uint8_t *generic;          // generic pointer to slot 0
-    int f_pre;                       // next unit of the run to fetch
-    int slot = 0;
-    uint32_t phase = 0;
-
-    __device__ __forceinline__ void issue(const CUtensorMap *map, const PruneParams &p, const Run<NORM_COLS> &run, int into, int lane)
-    {
-        if (lane == 0 && f_pre < run.f1) {
-            const uint32_t bar = bars + 8u * into;
-            mbar_arrive_expect_tx(bar, p.box_bytes);
-            tma_load_2d(slots + into * PN_SLOT_BYTES, map, bar, run.strip(f_pre) * PN_COLS, run.blk(f_pre) * PN_ROWS);
-        }
-        ++f_pre;
-    }
-    __device__ __forceinline__ void start(uint8_t *smem_aligned, int warp_in_cta, const CUtensorMap *map, const PruneParams &p,
-                                          const Run<NORM_COLS> &run, int lane)
-    {
-        generic = smem_aligned + warp_in_cta * PN_STAGES * PN_SLOT_BYTES;
-        slots = smem_u32(generic);
-        bars = smem_u32(smem_aligned + PN_WARPS * PN_STAGES * PN_SLOT_BYTES) + warp_in_cta * PN_STAGES * 8;
-        if (lane == 0) {
-#pragma unroll
-            for (int s = 0; s < PN_STAGES; ++s) mbar_init(bars + 8u * s, 1);
-            asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        }
-        __syncwarp();
-        f_pre = run.f0;
-#pragma unroll
-        for (int s = 0; s < PN_STAGES - 1; ++s) issue(map, p, run, s, lane);
-    }
-    // Refills the slot consumed one iteration ago, then waits for the current unit.  Returns its tile (16-byte
-    // vectors, row pitch p.pitch16) or nullptr when the wait ran out.
-    __device__ __forceinline__ const uint4 *next(const CUtensorMap *map, const PruneParams &p, const Run<NORM_COLS> &run, int lane)
-    {
-        __syncwarp();                  // every lane is done reading the slot that is refilled now
-        issue(map, p, run, slot == 0 ? PN_STAGES - 1 : slot - 1, lane);
-        const bool ok = slot_wait(bars + 8u * slot, phase);
-        const uint4 *tile = reinterpret_cast<const uint4 *>(generic + slot * PN_SLOT_BYTES);
-        if (++slot == PN_STAGES) { slot = 0; phase ^= 1u; }
-        return ok ? tile : nullptr;
-    }
-    // After a failed wait: record it and give the copies still in flight one more bounded chance to land.
-    __device__ __forceinline__ void fail(int lane)
-    {
-        if (lane == 0) atomicExch(&g_prune_status, (int)DASS_ERR_TIMEOUT);
-#pragma unroll
-        for (int s = 0; s < PN_STAGES; ++s) {
-            slot_wait(bars + 8u * s, 0u);
-            slot_wait(bars + 8u * s, 1u);
-        }
-    }
-};
 
 // Scales of a run.  Per-column: the CTA evaluates its strip's 256 scales once (two per thread) into shared memory
 // and a lane picks up its 8.  Per-row: lanes 0..7 evaluate the block's 8 rows and the warp shares them.
@@ -568,7 +320,7 @@ __global__ void __launch_bounds__(PN_THREADS, PN_MIN_BLOCKS) prune_rows_bf16_ker
 
     for (int f = run.f0; f < run.f1; ++f) {
         const uint4 *tile = ring.next(&map_w, p, run, lane);
-        if (tile == nullptr) { ring.fail(lane); return; }
+        if (tile == nullptr) { ring.fail(lane, p.status); return; }
         const int strip = run.strip(f);
         const int64_t r0 = (int64_t)run.blk(f) * PN_ROWS;
         const int64_t c0 = (int64_t)strip * PN_COLS + lane * 8;
@@ -755,7 +507,7 @@ __global__ void __launch_bounds__(PN_THREADS, PN_MIN_BLOCKS) prune_cols_bf16_ker
 
     for (int f = run.f0; f < run.f1; ++f) {
         const uint4 *tile = ring.next(&map_w, p, run, lane);
-        if (tile == nullptr) { ring.fail(lane); return; }
+        if (tile == nullptr) { ring.fail(lane, p.status); return; }
         const int strip = run.strip(f);
         const int64_t r0 = (int64_t)run.blk(f) * PN_ROWS;
         const int64_t c0 = (int64_t)strip * PN_COLS + lane * 8;
@@ -767,6 +519,56 @@ __global__ void __launch_bounds__(PN_THREADS, PN_MIN_BLOCKS) prune_cols_bf16_ker
 
 int device_sm_count();   // dass_abi.cu
 bool tile_map_bf16(CUtensorMap *map, const void *ptr, int64_t rows, int64_t cols, int64_t ld, int box_cols, int box_rows);   // calib_tc.cu
+
+__device__ int g_stage_b_status = 0;     // DASS_OK or DASS_ERR_TIMEOUT; read and cleared through dass_prune_status
+
+// Device address of the status word of the TMA-fed stage-(b) kernels (looked up once per device).
+int *stage_b_status_word()
+{
+    static std::atomic<int *> cached[64];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    int *ptr = cached[dev].load(std::memory_order_acquire);
+    if (!ptr) {
+        void *sym = nullptr;
+        if (cudaGetSymbolAddress(&sym, g_stage_b_status) != cudaSuccess) return nullptr;
+        ptr = static_cast<int *>(sym);
+        cached[dev].store(ptr, std::memory_order_release);
+    }
+    return ptr;
+}
+
+// Fills the decomposition of a [rows x cols] bf16 matrix into units and runs, encodes its tensor map and returns the
+// grid size.  Runs: about 8 CTAs per resident slot so that the block scheduler can even out the SMs, but at least 4
+// units per warp so that a warp's start-up (scales, first tile) stays small beside its work.
+cudaError_t unit_grid_setup(UnitGrid &g, CUtensorMap *map, int64_t *grid, const void *W, int64_t rows, int64_t cols, int64_t ld,
+                            bool walk_down)
+{
+    if (rows > 0x7fffffffll - PN_ROWS || cols > 0x7fffffffll - PN_COLS) return cudaErrorInvalidValue;
+    g.rows = rows; g.cols = cols;
+    g.strips = (cols + PN_COLS - 1) / PN_COLS;
+    g.blocks = (rows + PN_ROWS - 1) / PN_ROWS;
+    // one TMA box per unit; a box never exceeds the matrix (narrow or short matrices get a smaller box)
+    const int box_cols = cols >= PN_COLS ? PN_COLS : (int)((cols + 7) / 8 * 8);
+    const int box_rows = rows >= PN_ROWS ? PN_ROWS : (int)rows;
+    g.box_bytes = (uint32_t)(box_cols * box_rows * 2);
+    g.pitch16 = (uint32_t)(box_cols / 8);
+    if (!tile_map_bf16(map, W, rows, cols, ld, box_cols, box_rows)) return cudaErrorInvalidValue;
+    g.fast = walk_down ? g.blocks : g.strips;
+    const int64_t lines = walk_down ? g.strips : g.blocks;
+    const int64_t units = g.fast * lines;
+    const int64_t target_ctas = (int64_t)device_sm_count() * PN_MIN_BLOCKS * 8;
+    int64_t per_warp = units / (target_ctas * PN_WARPS);
+    per_warp = per_warp < 4 ? 4 : (per_warp > 64 ? 64 : per_warp);
+    const int64_t runs = (g.fast + per_warp - 1) / per_warp;
+    if (runs > 0x7fffffffll) return cudaErrorInvalidValue;
+    g.runs = (int)runs;
+    g.ctas_per_line = (int)((runs + PN_WARPS - 1) / PN_WARPS);
+    *grid = walk_down ? lines * g.ctas_per_line : ((lines + PN_WARPS - 1) / PN_WARPS) * runs;
+    if (*grid > 0x7fffffffll) return cudaErrorInvalidValue;
+    g.status = stage_b_status_word();
+    return cudaSuccess;
+}
 
 template <typename Kernel>
 static cudaError_t launch_prune(Kernel kernel, DeviceMask &configured, const CUtensorMap &map, const PruneParams &p,
@@ -798,7 +600,7 @@ cudaError_t prune_nm_bf16_launch(const void *W, int64_t rows, int64_t cols, int6
     p.values = static_cast<uint16_t *>(values);
     p.meta = meta;
     p.norm = norm;
-    p.rows = rows; p.cols = cols; p.ld = ld;
+    p.ld = ld;
     p.wpr = (cols + 31) / 32;
     const bool two_four = m == 4;
     if (group_cols) {
@@ -811,33 +613,12 @@ cudaError_t prune_nm_bf16_launch(const void *W, int64_t rows, int64_t cols, int6
         p.mwpl = (cols + fpw - 1) / fpw;
         p.vec_ok = (cols % 8 == 0) && ((reinterpret_cast<uintptr_t>(values) & 15u) == 0);
     }
-    p.strips = (cols + PN_COLS - 1) / PN_COLS;
-    p.blocks = (rows + PN_ROWS - 1) / PN_ROWS;
     p.scale_mode = (int)scale_mode_for(alpha);
     p.alpha = alpha;
-    if (rows > 0x7fffffffll - PN_ROWS || cols > 0x7fffffffll - PN_COLS) return cudaErrorInvalidValue;
-    // one TMA box per unit; a box never exceeds the matrix (narrow or short matrices get a smaller box)
-    const int box_cols = cols >= PN_COLS ? PN_COLS : (int)((cols + 7) / 8 * 8);
-    const int box_rows = rows >= PN_ROWS ? PN_ROWS : (int)rows;
-    p.box_bytes = (uint32_t)(box_cols * box_rows * 2);
-    p.pitch16 = (uint32_t)(box_cols / 8);
     CUtensorMap map;
-    if (!tile_map_bf16(&map, W, rows, cols, ld, box_cols, box_rows)) return cudaErrorInvalidValue;
-
-    // Runs: about 8 CTAs per resident slot so that the block scheduler can even out the SMs, but at least 4 units
-    // per warp so that a warp's start-up (scales, first tile) stays small beside its work.
-    p.fast = norm_cols ? p.blocks : p.strips;
-    const int64_t lines = norm_cols ? p.strips : p.blocks;
-    const int64_t units = p.fast * lines;
-    const int64_t target_ctas = (int64_t)device_sm_count() * PN_MIN_BLOCKS * 8;
-    int64_t per_warp = units / (target_ctas * PN_WARPS);
-    per_warp = per_warp < 4 ? 4 : (per_warp > 64 ? 64 : per_warp);
-    int64_t runs = (p.fast + per_warp - 1) / per_warp;
-    if (runs > 0x7fffffffll) return cudaErrorInvalidValue;
-    p.runs = (int)runs;
-    p.ctas_per_line = (int)((runs + PN_WARPS - 1) / PN_WARPS);
-    const int64_t grid = norm_cols ? lines * p.ctas_per_line : ((lines + PN_WARPS - 1) / PN_WARPS) * runs;
-    if (grid > 0x7fffffffll) return cudaErrorInvalidValue;
+    int64_t grid = 0;
+    const cudaError_t ge = unit_grid_setup(p, &map, &grid, W, rows, cols, ld, norm_cols);
+    if (ge != cudaSuccess) return ge;
 
     const bool all = mask_bits && W_pruned && values;
     if (m == 4) {
@@ -851,13 +632,13 @@ cudaError_t prune_nm_bf16_launch(const void *W, int64_t rows, int64_t cols, int6
 // Reads and clears the status word of the one-pass kernels (waits for the stream).
 cudaError_t prune_status_read(int *host_value, cudaStream_t st)
 {
-    cudaError_t e = cudaMemcpyFromSymbolAsync(host_value, g_prune_status, sizeof(int), 0, cudaMemcpyDeviceToHost, st);
+    cudaError_t e = cudaMemcpyFromSymbolAsync(host_value, g_stage_b_status, sizeof(int), 0, cudaMemcpyDeviceToHost, st);
     if (e != cudaSuccess) return e;
     e = cudaStreamSynchronize(st);
     if (e != cudaSuccess) return e;
     if (*host_value != 0) {
         const int zero = 0;
-        e = cudaMemcpyToSymbolAsync(g_prune_status, &zero, sizeof(int), 0, cudaMemcpyHostToDevice, st);
+        e = cudaMemcpyToSymbolAsync(g_stage_b_status, &zero, sizeof(int), 0, cudaMemcpyHostToDevice, st);
         if (e == cudaSuccess) e = cudaStreamSynchronize(st);
     }
     return e;

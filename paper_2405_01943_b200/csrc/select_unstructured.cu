@@ -20,7 +20,7 @@
 #include <cmath>
 #include <type_traits>
 
-#include "dass_device.cuh"
+#include "stream_units.cuh"
 
 namespace dass {
 
@@ -46,7 +46,6 @@ struct SelectParams {
     int64_t lpad;        // L rounded up to 8
     uint32_t k;          // survivors per line
     int idx_bits;        // bits of L - 1 (at least 1): width of the index part of the key
-    int margin;          // sampled bracket: sample positions on either side of the wanted rank
     int scale_along_line;   // 1: scale[e] varies along the line; 0: scale[line]
 };
 
@@ -276,14 +275,14 @@ __device__ __forceinline__ bool keeps(const LineResult &res, float a, float s, l
     return k64 > res.tau64 || (k64 == res.tau64 && idx <= res.cut);
 }
 
-// ---------------------------------------------------------------- sampled bracket in front of the radix select
-constexpr int SAMPLE = 512;                     // sample size per line (a power of two)
+// ---------------------------------------------------------------- octave window in front of the radix select
+constexpr int WIN_SAMPLE = 256;                 // evenly spaced elements of a line whose exponents place its window
+constexpr int WIN_BELOW = 3;                    // the window: 3 octaves below the octave of the sample's quantile, that octave, 4 above
+constexpr int WIN_SHIFT = 15;                   // 2^26 keys in 2048 bins of 2^15: 256 bins per octave
+constexpr uint32_t WIN_SPAN = 1u << (WIN_SHIFT + HB);
+constexpr int CODE_SHIFT = 11;                  // 16-bit code of a key inside the window: 1 + (key - window start) >> 11, 16 codes per bin
 constexpr int CAND_CAP = 96;                    // elements of the cut's bin that the final ranking takes
-constexpr int64_t FAST_MIN_L = 4 * SAMPLE;      // shorter lines go straight to the radix select
-// Row lines keep to the radix select: with the line cached in shared memory its passes are cheap enough that the
-// bracket's sort and two extra sweeps cost more than the hot first histogram they avoid (measured on the 70B-shaped
-// down projection: 0.75 ms with the bracket, 0.60 ms without).  Column lines gain (0.60 -> 0.53 ms).
-constexpr bool FAST_ROW_LINES = false;
+constexpr int64_t FAST_MIN_L = 4096;            // shorter lines go straight to the radix select
 
 struct FastLine {                // bracket state of one comparison line (shared memory)
     uint32_t lo, hi;             // candidates: lo <= key < hi (key = bits of the rounded product, sign cleared)
@@ -305,39 +304,50 @@ struct CandSet {                 // the collected elements of one line
 
 __device__ __forceinline__ uint32_t product_key(float wf, float s) { return __float_as_uint(__fmul_rn(wf, s)) & 0x7fffffffu; }
 
-// Ascending bitonic sort of NL arrays of SAMPLE keys each (shared memory); every thread of the block takes part.
-template <int NL, int THREADS>
-__device__ __forceinline__ void sort_samples(uint32_t *samp, int tid)
+// One warp: places the window of one line from the exponent histogram (256 bins, key >> 23) of its sample.  The
+// octave that holds the sample's `target`-th largest key is found, and the window starts WIN_BELOW octaves below it.
+// The line's true cut lies within a fraction of an octave of the sample's; if it does not lie in the window after
+// all, bracket_pick_bin sees that from the counts and the line takes the radix select.
+__device__ __forceinline__ void window_from_exponents(const uint32_t *eh, FastLine &f, uint32_t target, int lane)
 {
-    for (int k = 2; k <= SAMPLE; k <<= 1) {
-        for (int j = k >> 1; j > 0; j >>= 1) {
-            for (int t = tid; t < NL * (SAMPLE / 2); t += THREADS) {
-                const int line = t / (SAMPLE / 2), i = t % (SAMPLE / 2);
-                const int a = ((i & ~(j - 1)) << 1) | (i & (j - 1)), b = a | j;
-                uint32_t *row = samp + line * SAMPLE;
-                const uint32_t x = row[a], y = row[b];
-                if ((x > y) == ((a & k) == 0)) { row[a] = y; row[b] = x; }
-            }
-            __syncthreads();
+    uint32_t c[8], mine = 0u;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) { c[i] = eh[lane * 8 + i]; mine += c[i]; }
+    uint32_t v = mine;                                // becomes the sum over lanes >= this one
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const uint32_t t = __shfl_down_sync(FULL_MASK, v, off);
+        if (lane + off < 32) v += t;
+    }
+    uint32_t above = v - mine;
+    const bool here = above < target && target <= above + mine;
+    int e = 0;
+    if (here) {
+#pragma unroll
+        for (int i = 7; i >= 0; --i) {
+            if (target <= above + c[i]) { e = lane * 8 + i; break; }
+            above += c[i];
         }
+    }
+    const uint32_t who = __ballot_sync(FULL_MASK, here);
+    e = who ? __shfl_sync(FULL_MASK, e, __ffs(who) - 1) : 0;
+    if (lane == 0) {
+        const int e0 = e > WIN_BELOW ? e - WIN_BELOW : 0;
+        f.lo = (uint32_t)e0 << 23;
+        f.hi = f.lo + WIN_SPAN;
+        f.sh = WIN_SHIFT;
+        f.above = 0u; f.ncoll = 0u; f.ok = 1u; f.krem2 = 0u; f.bucket = 0u; f.blo = 0u; f.bhi = 0u;
     }
 }
 
-// Bracket of one line from its sorted sample: the survivors' cut has ascending rank L - k; `margin` sample
-// positions on either side are four standard deviations of the rank of a sample quantile.
-__device__ __forceinline__ void bracket_from_sample(FastLine &f, const uint32_t *sorted, int64_t L, uint32_t k, int margin)
+// Rank, from the top, of the sample key that stands for the line's k-th largest.
+__device__ __forceinline__ uint32_t win_target(uint32_t k, int64_t L)
 {
-    const int pos = (int)(((L - (int64_t)k) * SAMPLE) / L);
-    const int lo_i = pos - margin, hi_i = pos + margin;
-    f.lo = lo_i < 0 ? 0u : sorted[lo_i];
-    f.hi = hi_i >= SAMPLE ? 0x80000000u : sorted[hi_i] + 1u;
-    const uint32_t span = f.hi - f.lo - 1u;                  // largest offset inside the bracket
-    const int bits = 32 - __clz(span);                       // __clz(0) = 32
-    f.sh = bits > HB ? bits - HB : 0;
-    f.above = 0u; f.ncoll = 0u; f.ok = 1u; f.krem2 = 0u; f.bucket = 0u; f.blo = 0u; f.bhi = 0u;
+    const int64_t t = ((int64_t)k * WIN_SAMPLE + L - 1) / L;
+    return (uint32_t)(t < 1 ? 1 : (t > WIN_SAMPLE ? WIN_SAMPLE : t));
 }
 
-// One warp: the bin of the bracket's histogram that holds the line's last survivor.
+// One warp: the bin of the window's histogram that holds the line's last survivor.
 __device__ __forceinline__ void bracket_pick_bin(const uint32_t *h, FastLine &f, uint32_t k, int lane)
 {
     const uint32_t *mine_bins = h + lane * 64;
@@ -454,16 +464,196 @@ __global__ void __launch_bounds__(ROW_THREADS) select_rows_kernel(const SelectPa
     const int64_t nchunks = p.lpad >> 3;
     const uint32_t idx_top = (uint32_t)((1ull << p.idx_bits) - 1ull);
 
+    const float line_scale = p.scale_along_line ? 0.0f : DASS_LD(&p.scale[row]);
+    const elem_t *wrow = static_cast<const elem_t *>(p.W) + row * p.ld;
+    const int64_t nfull = p.L >> 3;                  // chunks whose 8 elements all exist
+
+    // ---------------------------------------------------------------- octave window (see the top of the file)
+    // The line is read once from global memory; what stays in shared memory is a 16-bit code per element: 0 below
+    // the window, 0xffff above it, else 1 + (key - window start) >> 11, which orders any two elements that differ in
+    // it.  The window's histogram is filled in the same pass, the cut's bin is searched in the codes, and the
+    // outputs are written from the codes and a second read of the weights; the scale vector, which is twice the
+    // size of a bf16 line, is read once instead of once per pass.
+    __shared__ FastLine fl;
+    __shared__ CandSet cand;
+    if (p.L >= FAST_MIN_L) {                         // the same for every thread
+        uint16_t *codes = reinterpret_cast<uint16_t *>(u_smem);      // [lpad]
+        auto weight_at = [&](int64_t e) {
+            if constexpr (BF16) return __uint_as_float((uint32_t)DASS_LD_G(wrow + e) << 16);
+            else return __uint_as_float(DASS_LD_G(wrow + e));
+        };
+        auto scale_at = [&](int64_t e) { return p.scale_along_line ? DASS_LD_G(p.scale + e) : line_scale; };
+        // the 8 weights of chunk q as stored, and their scales
+        auto load_chunk = [&](int64_t q, Chunk<BF16> &ch, float (&sc)[8]) {
+            const uint4 *src = reinterpret_cast<const uint4 *>(wrow + q * 8);
+            const uint4 v0 = DASS_LD_G(src);
+            ch.w[0] = v0.x; ch.w[1] = v0.y; ch.w[2] = v0.z; ch.w[3] = v0.w;
+            if constexpr (!BF16) {
+                const uint4 v1 = DASS_LD_G(src + 1);         // a row's pitch covers whole 8-element chunks
+                ch.w[4] = v1.x; ch.w[5] = v1.y; ch.w[6] = v1.z; ch.w[7] = v1.w;
+            }
+            if (p.scale_along_line) {
+                const float4 s0 = DASS_LD_G(reinterpret_cast<const float4 *>(p.scale + q * 8));
+                const float4 s1 = DASS_LD_G(reinterpret_cast<const float4 *>(p.scale + q * 8) + 1);   // the vector is padded to 8
+                sc[0] = s0.x; sc[1] = s0.y; sc[2] = s0.z; sc[3] = s0.w; sc[4] = s1.x; sc[5] = s1.y; sc[6] = s1.z; sc[7] = s1.w;
+            } else {
+#pragma unroll
+                for (int j = 0; j < 8; ++j) sc[j] = line_scale;
+            }
+        };
+        uint32_t *ehist = hist;                      // [256] exponent counts of the sample, before the bins
+        for (int i = tid; i < 256; i += ROW_THREADS) ehist[i] = 0u;
+        if (tid == 0) fl.ok = 0u;
+        __syncthreads();
+        for (int i = tid; i < WIN_SAMPLE; i += ROW_THREADS) {
+            const int64_t e = ((int64_t)i * p.L) / WIN_SAMPLE;
+            atomicAdd(ehist + (product_key(weight_at(e), scale_at(e)) >> 23), 1u);
+        }
+        __syncthreads();
+        if (warp == 0) window_from_exponents(ehist, fl, win_target(p.k, p.L), lane);
+        __syncthreads();
+        for (int i = tid; i < HBINS; i += ROW_THREADS) hist[i] = 0u;
+        __syncthreads();
+        const uint32_t lo = fl.lo;
+        {   // first pass: codes to shared memory, elements inside the window to the histogram, those above it counted
+            uint32_t above = 0u;
+            auto code_of = [&](float wf, float s) {
+                const uint32_t key = product_key(wf, s);
+                const uint32_t off = key - lo;
+                if (off < WIN_SPAN) {
+                    atomicAdd(hist + (off >> WIN_SHIFT), 1u);
+                    return (off >> CODE_SHIFT) + 1u;
+                }
+                const uint32_t up = key > lo ? 1u : 0u;
+                above += up;
+                return up ? 0xffffu : 0u;
+            };
+            auto code_chunk = [&](int64_t q, const Chunk<BF16> &ch, const float (&sc)[8], int nvalid) {
+                uint32_t cw[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const uint32_t c0 = 2 * i < nvalid ? code_of(chunk_float<BF16>(ch, 2 * i), sc[2 * i]) : 0u;
+                    const uint32_t c1 = 2 * i + 1 < nvalid ? code_of(chunk_float<BF16>(ch, 2 * i + 1), sc[2 * i + 1]) : 0u;
+                    cw[i] = c0 | (c1 << 16);
+                }
+                *reinterpret_cast<uint4 *>(codes + q * 8) = make_uint4(cw[0], cw[1], cw[2], cw[3]);
+            };
+            int64_t q = tid;
+            for (; q + ROW_THREADS < nfull; q += 2 * ROW_THREADS) {      // two chunks of a thread in flight
+                Chunk<BF16> ch0, ch1;
+                float s0[8], s1[8];
+                load_chunk(q, ch0, s0);
+                load_chunk(q + ROW_THREADS, ch1, s1);
+                code_chunk(q, ch0, s0, 8);
+                code_chunk(q + ROW_THREADS, ch1, s1, 8);
+            }
+            for (; q < nchunks; q += ROW_THREADS) {
+                Chunk<BF16> ch;
+                float s[8];
+                load_chunk(q, ch, s);
+                const int64_t left = p.L - q * 8;
+                code_chunk(q, ch, s, left >= 8 ? 8 : (int)left);
+            }
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) above += __shfl_xor_sync(FULL_MASK, above, off);
+            if (lane == 0 && above) atomicAdd(&fl.above, above);
+        }
+        __syncthreads();
+        if (warp == 0) bracket_pick_bin(hist, fl, p.k, lane);
+        __syncthreads();
+        if (fl.ok) {                                 // the same for every thread
+            // the elements of the cut's bin: 16 consecutive codes
+            const uint32_t base2 = (((fl.blo - lo) >> CODE_SHIFT) + 1u) * 0x00010001u;
+            const uint32_t span2 = (1u << (WIN_SHIFT - CODE_SHIFT)) * 0x00010001u;
+            for (int64_t q = tid; q < nchunks; q += ROW_THREADS) {
+                const uint4 c = *reinterpret_cast<const uint4 *>(codes + q * 8);
+                const uint32_t cw[4] = {c.x, c.y, c.z, c.w};
+                uint32_t hit[4], any = 0u;
+#pragma unroll
+                for (int i = 0; i < 4; ++i) { hit[i] = __vcmpltu2(__vsub2(cw[i], base2), span2); any |= hit[i]; }
+                if (any) {
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        if ((hit[j >> 1] >> (16 * (j & 1))) & 1u) {
+                            const int64_t e = q * 8 + j;
+                            const float wf = weight_at(e), sv = scale_at(e);
+                            const uint32_t slot = atomicAdd(&fl.ncoll, 1u);
+                            if (slot < (uint32_t)CAND_CAP) {
+                                cand.key[slot] = product_key(wf, sv); cand.idx[slot] = (uint32_t)e; cand.k64[slot] = exact_key(fabsf(wf), sv);
+                            }
+                        }
+                    }
+                }
+            }
+            __syncthreads();
+            if (warp == 0) bracket_rank(cand, fl, lane);
+            __syncthreads();
+        }
+        if (fl.ok) {                                 // the same for every thread: the line is decided, write it out
+            const LineResult res = fl.res;
+            const uint32_t tau2 = (((res.tau32 - lo) >> CODE_SHIFT) + 1u) * 0x00010001u;
+            for (int64_t q = tid; q < nchunks; q += ROW_THREADS) {
+                const uint4 c = *reinterpret_cast<const uint4 *>(codes + q * 8);
+                const uint32_t cw[4] = {c.x, c.y, c.z, c.w};
+                const int64_t e0 = q * 8;
+                Chunk<BF16> ch;
+                if (p.Wp) {
+                    const uint4 *src = reinterpret_cast<const uint4 *>(wrow + e0);
+                    const uint4 v0 = DASS_LD_G(src);
+                    ch.w[0] = v0.x; ch.w[1] = v0.y; ch.w[2] = v0.z; ch.w[3] = v0.w;
+                    if constexpr (!BF16) {
+                        const uint4 v1 = DASS_LD_G(src + 1);
+                        ch.w[4] = v1.x; ch.w[5] = v1.y; ch.w[6] = v1.z; ch.w[7] = v1.w;
+                    }
+                }
+                uint32_t gt[4], tie = 0u;            // per 16-bit half: all ones where the element stays
+#pragma unroll
+                for (int i = 0; i < 4; ++i) { gt[i] = __vcmpgtu2(cw[i], tau2); tie |= __vcmpeq2(cw[i], tau2); }
+                if (tie) {                           // same code as the cut: the full rule decides
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        if (((cw[j >> 1] >> (16 * (j & 1))) & 0xffffu) == (tau2 & 0xffffu)) {
+                            const int64_t e = e0 + j;
+                            if (keeps(res, weight_at(e), scale_at(e), e)) gt[j >> 1] |= 0xffffu << (16 * (j & 1));
+                        }
+                    }
+                }
+                if (p.mask) {
+                    const uint32_t b0 = __byte_perm(gt[0], gt[1], 0x6420) & 0x08040201u;
+                    const uint32_t b1 = __byte_perm(gt[2], gt[3], 0x6420) & 0x80402010u;
+                    const uint32_t keep = ((b0 | b1) * 0x01010101u) >> 24;
+                    DASS_ST(&reinterpret_cast<uint8_t *>(p.mask + row * p.wpr)[q], (uint8_t)keep);   // byte q = columns 8q..8q+7
+                }
+                if (p.Wp) {
+                    if constexpr (BF16) {
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) ch.w[i] &= gt[i];
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            ch.w[2 * i] &= (uint32_t)((int32_t)(gt[i] << 16) >> 16);
+                            ch.w[2 * i + 1] &= (uint32_t)((int32_t)gt[i] >> 16);
+                        }
+                    }
+                    const int64_t left = p.L - e0;
+                    chunk_store<BF16>(ch, p.Wp, row * p.ld + e0, left >= 8 ? 8 : (int)left);
+                }
+            }
+            return;
+        }
+        __syncthreads();                             // the codes give way to the line itself
+    }
+
+    // ---------------------------------------------------------------- radix select on the line in shared memory
     {   // rows are 16-byte aligned and padded to whole vectors by the ld rule; what a vector drags in past L is
         // never used (every consumer checks the index against L)
-        const uint4 *src = reinterpret_cast<const uint4 *>(static_cast<const elem_t *>(p.W) + row * p.ld);
+        const uint4 *src = reinterpret_cast<const uint4 *>(wrow);
         uint4 *dst = reinterpret_cast<uint4 *>(line_mem);
         const int64_t nvec = (p.L + EPV - 1) / EPV;
         for (int64_t v = tid; v < (int64_t)(p.lpad / EPV); v += ROW_THREADS)
             dst[v] = v < nvec ? DASS_LD_CS(src + v) : make_uint4(0u, 0u, 0u, 0u);
     }
     if (tid == 0) { line_init(st, p.k); s_long = 0u; }
-    const float line_scale = p.scale_along_line ? 0.0f : DASS_LD(&p.scale[row]);
 
     // the 8 signed weights and scales of chunk q
     auto fetch = [&](int64_t q, float (&w)[8], float (&sc)[8]) {
@@ -480,7 +670,6 @@ __global__ void __launch_bounds__(ROW_THREADS) select_rows_kernel(const SelectPa
             for (int j = 0; j < 8; ++j) sc[j] = line_scale;
         }
     };
-    const int64_t nfull = p.L >> 3;                  // chunks whose 8 elements all exist
     uint32_t *my_hist = hist + (lane % ROW_COPIES) * HBINS;
     auto count_pass = [&](auto mode_tag, const Sched &sc, uint32_t t32) {
         constexpr int MODE = decltype(mode_tag)::value;
@@ -499,86 +688,9 @@ __global__ void __launch_bounds__(ROW_THREADS) select_rows_kernel(const SelectPa
         }
     };
 
-    // ---------------------------------------------------------------- sampled bracket (see the top of the file)
-    __shared__ FastLine fl;
-    __shared__ CandSet cand;
-    __shared__ uint32_t samp[SAMPLE];
-    bool fast_done = false;
-    if (FAST_ROW_LINES && p.L >= FAST_MIN_L) {       // the same for every thread
-        __syncthreads();                             // the line is in shared memory
-        for (int i = tid; i < SAMPLE; i += ROW_THREADS) {
-            const int64_t e = ((int64_t)i * p.L) / SAMPLE;
-            float wf;
-            if constexpr (BF16) wf = __uint_as_float((uint32_t)line_mem[e] << 16);
-            else wf = __uint_as_float(line_mem[e]);
-            samp[i] = product_key(wf, p.scale_along_line ? DASS_LD_G(p.scale + e) : line_scale);
-        }
-        __syncthreads();
-        sort_samples<1, ROW_THREADS>(samp, tid);
-        if (tid == 0) bracket_from_sample(fl, samp, p.L, p.k, p.margin);
-        for (int i = tid; i < HBINS; i += ROW_THREADS) hist[i] = 0u;
-        __syncthreads();
-        {   // one pass: elements above the bracket are counted, those inside go to the histogram
-            const uint32_t lo = fl.lo, hi = fl.hi;
-            const int sh = fl.sh;
-            uint32_t above = 0u;
-            auto visit = [&](float wf, float s) {
-                const uint32_t key = product_key(wf, s);
-                if (key >= hi) ++above;
-                else if (key >= lo) atomicAdd(hist + ((key - lo) >> sh), 1u);
-            };
-            for (int64_t q = tid; q < nfull; q += ROW_THREADS) {
-                float w[8], s[8];
-                fetch(q, w, s);
-#pragma unroll
-                for (int j = 0; j < 8; ++j) visit(w[j], s[j]);
-            }
-            if (tid == 0 && nfull < nchunks) {
-                float w[8], s[8];
-                fetch(nfull, w, s);
-#pragma unroll
-                for (int j = 0; j < 8; ++j)
-                    if (nfull * 8 + j < p.L) visit(w[j], s[j]);
-            }
-#pragma unroll
-            for (int off = 16; off > 0; off >>= 1) above += __shfl_xor_sync(FULL_MASK, above, off);
-            if (lane == 0 && above) atomicAdd(&fl.above, above);
-        }
-        __syncthreads();
-        if (warp == 0) bracket_pick_bin(hist, fl, p.k, lane);
-        __syncthreads();
-        if (fl.ok) {                                 // the same for every thread
-            const uint32_t blo = fl.blo, bhi = fl.bhi;
-            auto visit = [&](float wf, float s, uint32_t idx) {
-                const uint32_t key = product_key(wf, s);
-                if (key >= blo && key < bhi) {
-                    const uint32_t slot = atomicAdd(&fl.ncoll, 1u);
-                    if (slot < (uint32_t)CAND_CAP) { cand.key[slot] = key; cand.idx[slot] = idx; cand.k64[slot] = exact_key(fabsf(wf), s); }
-                }
-            };
-            for (int64_t q = tid; q < nfull; q += ROW_THREADS) {
-                float w[8], s[8];
-                fetch(q, w, s);
-#pragma unroll
-                for (int j = 0; j < 8; ++j) visit(w[j], s[j], (uint32_t)(q * 8 + j));
-            }
-            if (tid == 0 && nfull < nchunks) {
-                float w[8], s[8];
-                fetch(nfull, w, s);
-#pragma unroll
-                for (int j = 0; j < 8; ++j)
-                    if (nfull * 8 + j < p.L) visit(w[j], s[j], (uint32_t)(nfull * 8 + j));
-            }
-            __syncthreads();
-            if (warp == 0) bracket_rank(cand, fl, lane);
-            __syncthreads();
-        }
-        fast_done = fl.ok != 0u;
-    }
-
     Sched sc;
     sched_begin(sc, STAGE_ROUNDED, 31, 0);
-    while (!fast_done) {
+    for (;;) {
         for (int i = tid; i < ROW_COPIES * HBINS; i += ROW_THREADS) hist[i] = 0u;
         __syncthreads();
         const uint32_t t32 = st.tau32;
@@ -596,7 +708,7 @@ __global__ void __launch_bounds__(ROW_THREADS) select_rows_kernel(const SelectPa
     }
 
     // ---------------------------------------------------------------- emit in place
-    const LineResult res = fast_done ? fl.res : line_result(st, idx_top);
+    const LineResult res = line_result(st, idx_top);
     for (int64_t q = tid; q < nchunks; q += ROW_THREADS) {
         float a[8], s[8];
         fetch(q, a, s);
@@ -691,10 +803,9 @@ __global__ void __launch_bounds__(COL_THREADS, 1) select_cols_kernel(const Selec
         }
     };
 
-    // ---------------------------------------------------------------- sampled bracket (see the top of the file)
+    // ---------------------------------------------------------------- octave window (see the top of the file)
     __shared__ FastLine fl[COL_LINES];
     __shared__ CandSet cand[COL_LINES];
-    __shared__ uint32_t samp[COL_LINES * SAMPLE];
     bool any_pending = true;
     if (tid < COL_LINES) fl[tid].ok = 0u;
     if (p.L >= FAST_MIN_L) {                         // the same for every thread
@@ -711,31 +822,8 @@ __global__ void __launch_bounds__(COL_THREADS, 1) select_cols_kernel(const Selec
                 }
             }
         };
-        for (int i = tid; i < SAMPLE; i += COL_THREADS) {
-            const int64_t r = ((int64_t)i * p.L) / SAMPLE;
-            Chunk<BF16> ch;
-            load_row(r, ch);
-            const float rs = p.scale_along_line ? DASS_LD_G(p.scale + r) : 0.0f;
-#pragma unroll
-            for (int j = 0; j < COL_LINES; ++j)
-                samp[j * SAMPLE + i] = product_key(chunk_float<BF16>(ch, j), p.scale_along_line ? rs : col_scale[j]);
-        }
-        __syncthreads();
-        sort_samples<COL_LINES, COL_THREADS>(samp, tid);
-        if (tid < nl) bracket_from_sample(fl[tid], samp + tid * SAMPLE, p.L, p.k, p.margin);
-        for (int i = tid; i < COL_LINES * HBINS; i += COL_THREADS) hist[i] = 0u;
-        __syncthreads();
-        {   // one pass over the strip: elements above a column's bracket are counted, those inside go to its histogram
-            uint32_t lo[COL_LINES], hi[COL_LINES], above[COL_LINES];
-            int sh[COL_LINES];
-#pragma unroll
-            for (int j = 0; j < COL_LINES; ++j) {
-                const bool live = j < nl;
-                lo[j] = live ? fl[j].lo : 0xffffffffu;       // a column past the matrix edge takes nothing
-                hi[j] = live ? fl[j].hi : 0xffffffffu;
-                sh[j] = live ? fl[j].sh : 0;
-                above[j] = 0u;
-            }
+        // visits every row of the strip, UNROLL rows of a thread in flight: f(column, signed weight, scale, row)
+        auto sweep = [&](auto &&f) {
             for (int64_t r0 = tid; r0 < p.L; r0 += (int64_t)UNROLL * COL_THREADS) {
                 Chunk<BF16> ch[UNROLL];
                 float row_scale[UNROLL];
@@ -751,16 +839,45 @@ __global__ void __launch_bounds__(COL_THREADS, 1) select_cols_kernel(const Selec
                 }
 #pragma unroll
                 for (int u = 0; u < UNROLL; ++u) {
-                    if (r0 + (int64_t)u * COL_THREADS < p.L) {
+                    const int64_t r = r0 + (int64_t)u * COL_THREADS;
+                    if (r < p.L) {
 #pragma unroll
-                        for (int j = 0; j < COL_LINES; ++j) {
-                            const uint32_t key = product_key(chunk_float<BF16>(ch[u], j), p.scale_along_line ? row_scale[u] : col_scale[j]);
-                            if (key >= hi[j]) ++above[j];
-                            else if (key >= lo[j]) atomicAdd(hist + j * HBINS + ((key - lo[j]) >> sh[j]), 1u);
-                        }
+                        for (int j = 0; j < COL_LINES; ++j)
+                            f(j, chunk_float<BF16>(ch[u], j), p.scale_along_line ? row_scale[u] : col_scale[j], r);
                     }
                 }
             }
+        };
+        uint32_t *ehist = hist;                      // [COL_LINES][256] exponent counts of the sample, before the bins
+        for (int i = tid; i < COL_LINES * 256; i += COL_THREADS) ehist[i] = 0u;
+        __syncthreads();
+        if (tid < WIN_SAMPLE) {
+            const int64_t r = ((int64_t)tid * p.L) / WIN_SAMPLE;
+            Chunk<BF16> ch;
+            load_row(r, ch);
+            const float rs = p.scale_along_line ? DASS_LD_G(p.scale + r) : 0.0f;
+#pragma unroll
+            for (int j = 0; j < COL_LINES; ++j)
+                atomicAdd(ehist + j * 256 + (product_key(chunk_float<BF16>(ch, j), p.scale_along_line ? rs : col_scale[j]) >> 23), 1u);
+        }
+        __syncthreads();
+        if (warp < nl) window_from_exponents(ehist + warp * 256, fl[warp], win_target(p.k, p.L), lane);
+        __syncthreads();
+        for (int i = tid; i < COL_LINES * HBINS; i += COL_THREADS) hist[i] = 0u;
+        __syncthreads();
+        {   // first pass: elements above a column's window are counted, those inside go to its histogram
+            uint32_t lo[COL_LINES], above[COL_LINES];
+#pragma unroll
+            for (int j = 0; j < COL_LINES; ++j) {
+                lo[j] = j < nl ? fl[j].lo : 0u;      // a column past the matrix edge fills bins nobody reads
+                above[j] = 0u;
+            }
+            sweep([&](int j, float wf, float sc_, int64_t) {
+                const uint32_t key = product_key(wf, sc_);
+                const uint32_t off = key - lo[j];
+                if (off < WIN_SPAN) atomicAdd(hist + j * HBINS + (off >> WIN_SHIFT), 1u);
+                else above[j] += key > lo[j] ? 1u : 0u;
+            });
 #pragma unroll
             for (int j = 0; j < COL_LINES; ++j) {
                 uint32_t a = above[j];
@@ -773,48 +890,25 @@ __global__ void __launch_bounds__(COL_THREADS, 1) select_cols_kernel(const Selec
         if (warp < nl) bracket_pick_bin(hist + warp * HBINS, fl[warp], p.k, lane);
         __syncthreads();
         {   // second pass: the elements of each column's bin are collected
-            uint32_t blo[COL_LINES], bhi[COL_LINES];
+            uint32_t blo[COL_LINES], bw[COL_LINES];
             uint32_t some = 0u;
 #pragma unroll
             for (int j = 0; j < COL_LINES; ++j) {
                 const bool live = j < nl && fl[j].ok;
-                blo[j] = live ? fl[j].blo : 0xffffffffu;
-                bhi[j] = live ? fl[j].bhi : 0u;
+                blo[j] = live ? fl[j].blo : 0u;
+                bw[j] = live ? fl[j].bhi - fl[j].blo : 0u;
                 some |= live ? 1u : 0u;
             }
             if (some) {                              // the same for every thread
-                for (int64_t r0 = tid; r0 < p.L; r0 += (int64_t)UNROLL * COL_THREADS) {
-                    Chunk<BF16> ch[UNROLL];
-                    float row_scale[UNROLL];
-#pragma unroll
-                    for (int u = 0; u < UNROLL; ++u) {
-                        const int64_t r = r0 + (int64_t)u * COL_THREADS;
-                        chunk_zero<BF16>(ch[u]);
-                        row_scale[u] = 0.0f;
-                        if (r < p.L) {
-                            load_row(r, ch[u]);
-                            if (p.scale_along_line) row_scale[u] = DASS_LD_G(p.scale + r);
+                sweep([&](int j, float wf, float sc_, int64_t r) {
+                    const uint32_t key = product_key(wf, sc_);
+                    if (key - blo[j] < bw[j]) {
+                        const uint32_t slot = atomicAdd(&fl[j].ncoll, 1u);
+                        if (slot < (uint32_t)CAND_CAP) {
+                            cand[j].key[slot] = key; cand[j].idx[slot] = (uint32_t)r; cand[j].k64[slot] = exact_key(fabsf(wf), sc_);
                         }
                     }
-#pragma unroll
-                    for (int u = 0; u < UNROLL; ++u) {
-                        const int64_t r = r0 + (int64_t)u * COL_THREADS;
-                        if (r < p.L) {
-#pragma unroll
-                            for (int j = 0; j < COL_LINES; ++j) {
-                                const float wf = chunk_float<BF16>(ch[u], j);
-                                const float s = p.scale_along_line ? row_scale[u] : col_scale[j];
-                                const uint32_t key = product_key(wf, s);
-                                if (key >= blo[j] && key < bhi[j]) {
-                                    const uint32_t slot = atomicAdd(&fl[j].ncoll, 1u);
-                                    if (slot < (uint32_t)CAND_CAP) {
-                                        cand[j].key[slot] = key; cand[j].idx[slot] = (uint32_t)r; cand[j].k64[slot] = exact_key(fabsf(wf), s);
-                                    }
-                                }
-                            }
-                        }
-                    }
-                }
+                });
                 __syncthreads();
                 if (warp < nl && fl[warp].ok) bracket_rank(cand[warp], fl[warp], lane);
                 __syncthreads();
@@ -988,7 +1082,159 @@ __global__ void __launch_bounds__(256, 4) select_emit_cols_kernel(const EmitPara
     }
 }
 
+// ---------------------------------------------------------------- column lines, bf16: streaming emit fed by TMA
+// The same job with the machinery of the one-pass N:M kernels (stream_units.cuh): 8 x 256 units arrive through a
+// per-warp ring of TMA boxes, a warp walks down a strip so that a lane's 8 columns -- and with them its thresholds --
+// stay the same for the whole run, and "product < threshold" is read off the sign of a float difference that one
+// byte permute turns into the pruned-lane mask of a word.  Columns whose threshold the exact stage had to split
+// (rounded products tie across the cut) take a scalar fix-up for the elements equal to the threshold.
+struct EmitStreamParams : UnitGrid {
+    const uint16_t *W;
+    uint16_t *Wp;        // nullable
+    uint32_t *mask;      // nullable
+    const float *scale;
+    const LineResult *results;
+    int64_t ld, wpr;
+    int scale_per_row;
+};
+
+// Keep byte of one row of a lane's tile when some of its columns need the exact rule (rare).
+__device__ __noinline__ uint32_t emit_exact_row(uint4 row, uint32_t keep, uint32_t exact_cols, const LineResult *res8,
+                                                const float *sc8, float row_scale, int scale_per_row, long long r)
+{
+    for (int j = 0; j < 8; ++j) {
+        if (!((exact_cols >> j) & 1u)) continue;
+        const uint32_t w = wsel(row, j >> 1);
+        const float a = fabsf(__uint_as_float((j & 1) ? (w & 0xffff0000u) : (w << 16)));
+        const float s = scale_per_row ? row_scale : sc8[j];
+        const LineResult t = DASS_LD(res8 + j);
+        if (__float_as_uint(__fmul_rn(a, s)) != t.tau32) continue;          // only products equal to the threshold
+        const unsigned long long k64 = (unsigned long long)__double_as_longlong((double)a * (double)s);
+        const bool k = k64 > t.tau64 || (k64 == t.tau64 && r <= t.cut);
+        keep = (keep & ~(1u << j)) | ((k ? 1u : 0u) << j);
+    }
+    return keep;
+}
+
+__global__ void __launch_bounds__(PN_THREADS, PN_MIN_BLOCKS)
+select_emit_stream_kernel(const __grid_constant__ CUtensorMap map_w, const EmitStreamParams p)
+{
+    extern __shared__ uint8_t se_smem_raw[];
+    uint8_t *smem = se_smem_raw + ((128u - (smem_u32(se_smem_raw) & 127u)) & 127u);
+    const int lane = threadIdx.x & 31;
+    const uint32_t sel1 = (lane & 1) ? 0x3715u : 0x6240u;
+    const uint32_t sel2 = (lane & 2) ? 0x3276u : 0x5410u;
+    Run<true> run;                                   // down a strip: the lane's columns stay
+    run.set(p, threadIdx.x >> 5);
+    const int64_t c0 = (int64_t)run.line * PN_COLS + lane * 8;
+    const int64_t left = p.cols - c0;
+    const int nvalid = left >= 8 ? 8 : (left > 0 ? (int)left : 0);
+    const uint32_t valid = (1u << nvalid) - 1u;
+    const bool quad_live = (c0 & ~(int64_t)31) < p.cols;
+    float tau[8], sc[8];
+    uint32_t exact_cols = 0u;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        tau[j] = 0.0f;
+        sc[j] = 0.0f;
+        if (j < nvalid) {
+            tau[j] = __uint_as_float(DASS_LD(&p.results[c0 + j].tau32));
+            exact_cols |= (DASS_LD(&p.results[c0 + j].exact) ? 1u : 0u) << j;
+            if (!p.scale_per_row) sc[j] = DASS_LD(&p.scale[c0 + j]);
+        }
+    }
+    UnitRing<true> ring;
+    ring.start(smem, threadIdx.x >> 5, &map_w, p, run, lane);
+
+    for (int f = run.f0; f < run.f1; ++f) {
+        const uint4 *tile = ring.next(&map_w, p, run, lane);
+        if (tile == nullptr) { ring.fail(lane, p.status); return; }
+        const int64_t r0 = (int64_t)f * PN_ROWS;
+        float rs[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) rs[i] = 0.0f;
+        if (p.scale_per_row) {       // the scale vector is padded with zeros to a multiple of 8 and 32-byte aligned
+            const float4 a = DASS_LD_G(reinterpret_cast<const float4 *>(p.scale + r0));
+            const float4 b = DASS_LD_G(reinterpret_cast<const float4 *>(p.scale + r0) + 1);
+            rs[0] = a.x; rs[1] = a.y; rs[2] = a.z; rs[3] = a.w; rs[4] = b.x; rs[5] = b.y; rs[6] = b.z; rs[7] = b.w;
+        }
+#pragma unroll
+        for (int h = 0; h < PN_ROWS / 4; ++h) {
+            const int64_t rh = r0 + 4 * h;
+            if (rh >= p.rows) break;                 // warp-uniform
+            const int nrows = p.rows - rh >= 4 ? 4 : (int)(p.rows - rh);
+            uint4 v[4];
+            uint32_t Z[4][4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                v[i] = tile[(4 * h + i) * p.pitch16 + lane];
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    const uint32_t w = wsel(v[i], k);
+                    const float pe = prod_lo(w, p.scale_per_row ? rs[4 * h + i] : sc[2 * k]);
+                    const float po = prod_hi(w, p.scale_per_row ? rs[4 * h + i] : sc[2 * k + 1]);
+                    Z[i][k] = pruned_lanes(__fsub_rn(pe, tau[2 * k]), __fsub_rn(po, tau[2 * k + 1]));
+                }
+            }
+            const uint32_t rows4 = nrows == 4 ? 0xffffffffu : ((1u << (8 * nrows)) - 1u);
+            uint32_t keep = ~bytes_of_lanes4(Z[0], Z[1], Z[2], Z[3]) & (valid * 0x01010101u) & rows4;
+            if (exact_cols) {                        // rounded products equal to a split threshold: the exact rule decides
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    if (i < nrows) {
+                        const uint32_t kb = emit_exact_row(v[i], (keep >> (8 * i)) & 0xffu, exact_cols, p.results + c0, sc,
+                                                           rs[4 * h + i], p.scale_per_row, (long long)(rh + i));
+                        keep = (keep & ~(0xffu << (8 * i))) | (kb << (8 * i));
+                        uint32_t m[4];
+                        lanes_of_byte(kb, m);
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) Z[i][k] = ~m[k];
+                    }
+                }
+            }
+            const bool row_live = (lane & 3) < nrows;
+            if (p.mask) {
+                const uint32_t word = quad_transpose(keep, sel1, sel2);
+                if (quad_live && row_live) DASS_ST(&p.mask[(rh + (lane & 3)) * p.wpr + (c0 >> 5)], word);
+            }
+            if (p.Wp && nvalid > 0) {
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    if (i < nrows) {
+                        uint4 P;
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) wref(P, k) = wsel(v[i], k) & ~Z[i][k];
+                        store_row8(p.Wp + (rh + i) * p.ld + c0, P, nvalid);
+                    }
+                }
+            }
+        }
+    }
+}
+
 int device_sm_count();   // dass_abi.cu
+cudaError_t unit_grid_setup(UnitGrid &g, CUtensorMap *map, int64_t *grid, const void *W, int64_t rows, int64_t cols, int64_t ld,
+                            bool walk_down);   // prune_nm_bf16.cu
+
+static cudaError_t launch_emit_stream(const void *W, void *Wp, uint32_t *mask, const float *scale, const LineResult *results,
+                                      int64_t rows, int64_t cols, int64_t ld, int scale_per_row, cudaStream_t st)
+{
+    EmitStreamParams p;
+    p.W = static_cast<const uint16_t *>(W);
+    p.Wp = static_cast<uint16_t *>(Wp);
+    p.mask = mask; p.scale = scale; p.results = results;
+    p.ld = ld; p.wpr = (cols + 31) / 32;
+    p.scale_per_row = scale_per_row;
+    CUtensorMap map;
+    int64_t grid = 0;
+    cudaError_t e = unit_grid_setup(p, &map, &grid, W, rows, cols, ld, true);
+    if (e != cudaSuccess) return e;
+    static DeviceMask configured{0ull};
+    e = ensure_dynamic_smem(select_emit_stream_kernel, (int)PN_SMEM_BYTES, configured);
+    if (e != cudaSuccess) return e;
+    select_emit_stream_kernel<<<(unsigned)grid, PN_THREADS, PN_SMEM_BYTES, st>>>(map, p);
+    return cudaGetLastError();
+}
 
 // Dynamic shared memory of the row-line kernel: the cached line and one histogram.
 size_t select_row_smem_bytes(int64_t L, bool bf16)
@@ -1041,10 +1287,6 @@ cudaError_t select_unstructured_launch(const void *W, int64_t rows, int64_t cols
     p.idx_bits = 1;
     while (((int64_t)1 << p.idx_bits) < p.L) ++p.idx_bits;
     p.scale_along_line = (line_is_row == norm_cols) ? 1 : 0;   // the norm index runs along the line
-    {   // four standard deviations of the rank of a sample quantile, in sample positions, plus slack
-        const double q = (double)(p.L - (int64_t)k) / (double)p.L;
-        p.margin = (int)std::ceil(4.0 * std::sqrt((double)SAMPLE * q * (1.0 - q))) + 2;
-    }
     if (line_is_row) {
         if (mask_bits) {   // the kernel writes whole bytes of real columns; the padding of each mask row must read 0
             e = cudaMemsetAsync(mask_bits, 0, (size_t)rows * p.wpr * sizeof(uint32_t), st);
@@ -1063,8 +1305,9 @@ cudaError_t select_unstructured_launch(const void *W, int64_t rows, int64_t cols
     const int64_t want = (q.col_blocks * q.row_blocks + 7) / 8;
     const int64_t cap = (int64_t)device_sm_count() * 8;
     const int grid = (int)(want < cap ? want : cap);
-    if (bf16) select_emit_cols_kernel<true><<<grid, 256, 0, st>>>(q);
-    else select_emit_cols_kernel<false><<<grid, 256, 0, st>>>(q);
+    if (bf16)   // the TMA-fed streaming pass
+        return launch_emit_stream(W, W_pruned, mask_bits, scale_ws, results, rows, cols, ld, norm_cols ? 0 : 1, st);
+    select_emit_cols_kernel<false><<<grid, 256, 0, st>>>(q);
     return cudaGetLastError();
 }
 
