@@ -47,6 +47,8 @@ struct SelectParams {
     uint32_t k;          // survivors per line
     int idx_bits;        // bits of L - 1 (at least 1): width of the index part of the key
     int scale_along_line;   // 1: scale[e] varies along the line; 0: scale[line]
+    uint32_t *line_count;   // row lines: how many lines the streaming kernel left undecided, and which
+    uint32_t *line_list;    // (both null: the radix kernel takes every row)
 };
 
 // out[i] = fl32(norm[i]^alpha) for i < n, 0 for the padding up to npad (a multiple of 8, so that the selection
@@ -280,7 +282,6 @@ constexpr int WIN_SAMPLE = 256;                 // evenly spaced elements of a l
 constexpr int WIN_BELOW = 3;                    // the window: 3 octaves below the octave of the sample's quantile, that octave, 4 above
 constexpr int WIN_SHIFT = 15;                   // 2^26 keys in 2048 bins of 2^15: 256 bins per octave
 constexpr uint32_t WIN_SPAN = 1u << (WIN_SHIFT + HB);
-constexpr int CODE_SHIFT = 11;                  // 16-bit code of a key inside the window: 1 + (key - window start) >> 11, 16 codes per bin
 constexpr int CAND_CAP = 96;                    // elements of the cut's bin that the final ranking takes
 constexpr int64_t FAST_MIN_L = 4096;            // shorter lines go straight to the radix select
 
@@ -460,207 +461,136 @@ __global__ void __launch_bounds__(ROW_THREADS) select_rows_kernel(const SelectPa
     __shared__ uint32_t s_long;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int64_t row = blockIdx.x;
     const int64_t nchunks = p.lpad >> 3;
     const uint32_t idx_top = (uint32_t)((1ull << p.idx_bits) - 1ull);
+    // every row, or the rows the streaming kernel listed as undecided
+    const int64_t n_lines = p.line_list ? (int64_t)DASS_LD(p.line_count) : p.rows;
+    for (int64_t li = blockIdx.x; li < n_lines; li += gridDim.x) {
+        const int64_t row = p.line_list ? (int64_t)DASS_LD(&p.line_list[li]) : li;
+        const float line_scale = p.scale_along_line ? 0.0f : DASS_LD(&p.scale[row]);
+        const elem_t *wrow = static_cast<const elem_t *>(p.W) + row * p.ld;
+        const int64_t nfull = p.L >> 3;                  // chunks whose 8 elements all exist
 
-    const float line_scale = p.scale_along_line ? 0.0f : DASS_LD(&p.scale[row]);
-    const elem_t *wrow = static_cast<const elem_t *>(p.W) + row * p.ld;
-    const int64_t nfull = p.L >> 3;                  // chunks whose 8 elements all exist
+        // ---------------------------------------------------------------- radix select on the line in shared memory
+        {   // rows are 16-byte aligned and padded to whole vectors by the ld rule; what a vector drags in past L is
+            // never used (every consumer checks the index against L)
+            const uint4 *src = reinterpret_cast<const uint4 *>(wrow);
+            uint4 *dst = reinterpret_cast<uint4 *>(line_mem);
+            const int64_t nvec = (p.L + EPV - 1) / EPV;
+            for (int64_t v = tid; v < (int64_t)(p.lpad / EPV); v += ROW_THREADS)
+                dst[v] = v < nvec ? DASS_LD_CS(src + v) : make_uint4(0u, 0u, 0u, 0u);
+        }
+        if (tid == 0) { line_init(st, p.k); s_long = 0u; }
 
-    // ---------------------------------------------------------------- octave window (see the top of the file)
-    // The line is read once from global memory; what stays in shared memory is a 16-bit code per element: 0 below
-    // the window, 0xffff above it, else 1 + (key - window start) >> 11, which orders any two elements that differ in
-    // it.  The window's histogram is filled in the same pass, the cut's bin is searched in the codes, and the
-    // outputs are written from the codes and a second read of the weights; the scale vector, which is twice the
-    // size of a bf16 line, is read once instead of once per pass.
-    __shared__ FastLine fl;
-    __shared__ CandSet cand;
-    if (p.L >= FAST_MIN_L) {                         // the same for every thread
-        uint16_t *codes = reinterpret_cast<uint16_t *>(u_smem);      // [lpad]
-        auto weight_at = [&](int64_t e) {
-            if constexpr (BF16) return __uint_as_float((uint32_t)DASS_LD_G(wrow + e) << 16);
-            else return __uint_as_float(DASS_LD_G(wrow + e));
-        };
-        auto scale_at = [&](int64_t e) { return p.scale_along_line ? DASS_LD_G(p.scale + e) : line_scale; };
-        // the 8 weights of chunk q as stored, and their scales
-        auto load_chunk = [&](int64_t q, Chunk<BF16> &ch, float (&sc)[8]) {
-            const uint4 *src = reinterpret_cast<const uint4 *>(wrow + q * 8);
-            const uint4 v0 = DASS_LD_G(src);
-            ch.w[0] = v0.x; ch.w[1] = v0.y; ch.w[2] = v0.z; ch.w[3] = v0.w;
-            if constexpr (!BF16) {
-                const uint4 v1 = DASS_LD_G(src + 1);         // a row's pitch covers whole 8-element chunks
-                ch.w[4] = v1.x; ch.w[5] = v1.y; ch.w[6] = v1.z; ch.w[7] = v1.w;
-            }
+        // the 8 signed weights and scales of chunk q
+        auto fetch = [&](int64_t q, float (&w)[8], float (&sc)[8]) {
+            Chunk<BF16> ch;
+            chunk_from<BF16>(ch, reinterpret_cast<const uint4 *>(line_mem + q * 8));
+    #pragma unroll
+            for (int j = 0; j < 8; ++j) w[j] = chunk_float<BF16>(ch, j);
             if (p.scale_along_line) {
                 const float4 s0 = DASS_LD_G(reinterpret_cast<const float4 *>(p.scale + q * 8));
                 const float4 s1 = DASS_LD_G(reinterpret_cast<const float4 *>(p.scale + q * 8) + 1);   // the vector is padded to 8
                 sc[0] = s0.x; sc[1] = s0.y; sc[2] = s0.z; sc[3] = s0.w; sc[4] = s1.x; sc[5] = s1.y; sc[6] = s1.z; sc[7] = s1.w;
             } else {
-#pragma unroll
+    #pragma unroll
                 for (int j = 0; j < 8; ++j) sc[j] = line_scale;
             }
         };
-        uint32_t *ehist = hist;                      // [256] exponent counts of the sample, before the bins
-        for (int i = tid; i < 256; i += ROW_THREADS) ehist[i] = 0u;
-        if (tid == 0) fl.ok = 0u;
-        __syncthreads();
-        for (int i = tid; i < WIN_SAMPLE; i += ROW_THREADS) {
-            const int64_t e = ((int64_t)i * p.L) / WIN_SAMPLE;
-            atomicAdd(ehist + (product_key(weight_at(e), scale_at(e)) >> 23), 1u);
-        }
-        __syncthreads();
-        if (warp == 0) window_from_exponents(ehist, fl, win_target(p.k, p.L), lane);
-        __syncthreads();
-        for (int i = tid; i < HBINS; i += ROW_THREADS) hist[i] = 0u;
-        __syncthreads();
-        const uint32_t lo = fl.lo;
-        {   // first pass: codes to shared memory, elements inside the window to the histogram, those above it counted
-            uint32_t above = 0u;
-            auto code_of = [&](float wf, float s) {
-                const uint32_t key = product_key(wf, s);
-                const uint32_t off = key - lo;
-                if (off < WIN_SPAN) {
-                    atomicAdd(hist + (off >> WIN_SHIFT), 1u);
-                    return (off >> CODE_SHIFT) + 1u;
-                }
-                const uint32_t up = key > lo ? 1u : 0u;
-                above += up;
-                return up ? 0xffffu : 0u;
-            };
-            auto code_chunk = [&](int64_t q, const Chunk<BF16> &ch, const float (&sc)[8], int nvalid) {
-                uint32_t cw[4];
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const uint32_t c0 = 2 * i < nvalid ? code_of(chunk_float<BF16>(ch, 2 * i), sc[2 * i]) : 0u;
-                    const uint32_t c1 = 2 * i + 1 < nvalid ? code_of(chunk_float<BF16>(ch, 2 * i + 1), sc[2 * i + 1]) : 0u;
-                    cw[i] = c0 | (c1 << 16);
-                }
-                *reinterpret_cast<uint4 *>(codes + q * 8) = make_uint4(cw[0], cw[1], cw[2], cw[3]);
-            };
-            int64_t q = tid;
-            for (; q + ROW_THREADS < nfull; q += 2 * ROW_THREADS) {      // two chunks of a thread in flight
-                Chunk<BF16> ch0, ch1;
-                float s0[8], s1[8];
-                load_chunk(q, ch0, s0);
-                load_chunk(q + ROW_THREADS, ch1, s1);
-                code_chunk(q, ch0, s0, 8);
-                code_chunk(q + ROW_THREADS, ch1, s1, 8);
+        uint32_t *my_hist = hist + (lane % ROW_COPIES) * HBINS;
+        auto count_pass = [&](auto mode_tag, const Sched &sc, uint32_t t32) {
+            constexpr int MODE = decltype(mode_tag)::value;
+            for (int64_t q = tid; q < nfull; q += ROW_THREADS) {
+                float w[8], s[8];
+                fetch(q, w, s);
+    #pragma unroll
+                for (int j = 0; j < 8; ++j) count_element<MODE>(my_hist, st, t32, w[j], s[j], (uint32_t)(q * 8 + j), sc, idx_top);
             }
-            for (; q < nchunks; q += ROW_THREADS) {
-                Chunk<BF16> ch;
-                float s[8];
-                load_chunk(q, ch, s);
-                const int64_t left = p.L - q * 8;
-                code_chunk(q, ch, s, left >= 8 ? 8 : (int)left);
+            if (tid == 0 && nfull < nchunks) {           // the ragged last chunk
+                float w[8], s[8];
+                fetch(nfull, w, s);
+    #pragma unroll
+                for (int j = 0; j < 8; ++j)
+                    if (nfull * 8 + j < p.L) count_element<MODE>(my_hist, st, t32, w[j], s[j], (uint32_t)(nfull * 8 + j), sc, idx_top);
             }
-#pragma unroll
-            for (int off = 16; off > 0; off >>= 1) above += __shfl_xor_sync(FULL_MASK, above, off);
-            if (lane == 0 && above) atomicAdd(&fl.above, above);
-        }
-        __syncthreads();
-        if (warp == 0) bracket_pick_bin(hist, fl, p.k, lane);
-        __syncthreads();
-        if (fl.ok) {                                 // the same for every thread
-            // the elements of the cut's bin: 16 consecutive codes
-            const uint32_t base2 = (((fl.blo - lo) >> CODE_SHIFT) + 1u) * 0x00010001u;
-            const uint32_t span2 = (1u << (WIN_SHIFT - CODE_SHIFT)) * 0x00010001u;
-            for (int64_t q = tid; q < nchunks; q += ROW_THREADS) {
-                const uint4 c = *reinterpret_cast<const uint4 *>(codes + q * 8);
-                const uint32_t cw[4] = {c.x, c.y, c.z, c.w};
-                uint32_t hit[4], any = 0u;
-#pragma unroll
-                for (int i = 0; i < 4; ++i) { hit[i] = __vcmpltu2(__vsub2(cw[i], base2), span2); any |= hit[i]; }
-                if (any) {
-#pragma unroll
-                    for (int j = 0; j < 8; ++j) {
-                        if ((hit[j >> 1] >> (16 * (j & 1))) & 1u) {
-                            const int64_t e = q * 8 + j;
-                            const float wf = weight_at(e), sv = scale_at(e);
-                            const uint32_t slot = atomicAdd(&fl.ncoll, 1u);
-                            if (slot < (uint32_t)CAND_CAP) {
-                                cand.key[slot] = product_key(wf, sv); cand.idx[slot] = (uint32_t)e; cand.k64[slot] = exact_key(fabsf(wf), sv);
-                            }
-                        }
-                    }
-                }
-            }
-            __syncthreads();
-            if (warp == 0) bracket_rank(cand, fl, lane);
-            __syncthreads();
-        }
-        if (fl.ok) {                                 // the same for every thread: the line is decided, write it out
-            const LineResult res = fl.res;
-            const uint32_t tau2 = (((res.tau32 - lo) >> CODE_SHIFT) + 1u) * 0x00010001u;
-            for (int64_t q = tid; q < nchunks; q += ROW_THREADS) {
-                const uint4 c = *reinterpret_cast<const uint4 *>(codes + q * 8);
-                const uint32_t cw[4] = {c.x, c.y, c.z, c.w};
-                const int64_t e0 = q * 8;
-                Chunk<BF16> ch;
-                if (p.Wp) {
-                    const uint4 *src = reinterpret_cast<const uint4 *>(wrow + e0);
-                    const uint4 v0 = DASS_LD_G(src);
-                    ch.w[0] = v0.x; ch.w[1] = v0.y; ch.w[2] = v0.z; ch.w[3] = v0.w;
-                    if constexpr (!BF16) {
-                        const uint4 v1 = DASS_LD_G(src + 1);
-                        ch.w[4] = v1.x; ch.w[5] = v1.y; ch.w[6] = v1.z; ch.w[7] = v1.w;
-                    }
-                }
-                uint32_t gt[4], tie = 0u;            // per 16-bit half: all ones where the element stays
-#pragma unroll
-                for (int i = 0; i < 4; ++i) { gt[i] = __vcmpgtu2(cw[i], tau2); tie |= __vcmpeq2(cw[i], tau2); }
-                if (tie) {                           // same code as the cut: the full rule decides
-#pragma unroll
-                    for (int j = 0; j < 8; ++j) {
-                        if (((cw[j >> 1] >> (16 * (j & 1))) & 0xffffu) == (tau2 & 0xffffu)) {
-                            const int64_t e = e0 + j;
-                            if (keeps(res, weight_at(e), scale_at(e), e)) gt[j >> 1] |= 0xffffu << (16 * (j & 1));
-                        }
-                    }
-                }
-                if (p.mask) {
-                    const uint32_t b0 = __byte_perm(gt[0], gt[1], 0x6420) & 0x08040201u;
-                    const uint32_t b1 = __byte_perm(gt[2], gt[3], 0x6420) & 0x80402010u;
-                    const uint32_t keep = ((b0 | b1) * 0x01010101u) >> 24;
-                    DASS_ST(&reinterpret_cast<uint8_t *>(p.mask + row * p.wpr)[q], (uint8_t)keep);   // byte q = columns 8q..8q+7
-                }
-                if (p.Wp) {
-                    if constexpr (BF16) {
-#pragma unroll
-                        for (int i = 0; i < 4; ++i) ch.w[i] &= gt[i];
-                    } else {
-#pragma unroll
-                        for (int i = 0; i < 4; ++i) {
-                            ch.w[2 * i] &= (uint32_t)((int32_t)(gt[i] << 16) >> 16);
-                            ch.w[2 * i + 1] &= (uint32_t)((int32_t)gt[i] >> 16);
-                        }
-                    }
-                    const int64_t left = p.L - e0;
-                    chunk_store<BF16>(ch, p.Wp, row * p.ld + e0, left >= 8 ? 8 : (int)left);
-                }
-            }
-            return;
-        }
-        __syncthreads();                             // the codes give way to the line itself
-    }
+        };
 
-    // ---------------------------------------------------------------- radix select on the line in shared memory
-    {   // rows are 16-byte aligned and padded to whole vectors by the ld rule; what a vector drags in past L is
-        // never used (every consumer checks the index against L)
-        const uint4 *src = reinterpret_cast<const uint4 *>(wrow);
-        uint4 *dst = reinterpret_cast<uint4 *>(line_mem);
-        const int64_t nvec = (p.L + EPV - 1) / EPV;
-        for (int64_t v = tid; v < (int64_t)(p.lpad / EPV); v += ROW_THREADS)
-            dst[v] = v < nvec ? DASS_LD_CS(src + v) : make_uint4(0u, 0u, 0u, 0u);
-    }
-    if (tid == 0) { line_init(st, p.k); s_long = 0u; }
+        Sched sc;
+        sched_begin(sc, STAGE_ROUNDED, 31, 0);
+        for (;;) {
+            for (int i = tid; i < ROW_COPIES * HBINS; i += ROW_THREADS) hist[i] = 0u;
+            __syncthreads();
+            const uint32_t t32 = st.tau32;
+            const int mode = count_mode(sc);
+            if (mode == COUNT_ALL) count_pass(std::integral_constant<int, COUNT_ALL>{}, sc, t32);
+            else if (mode == COUNT_ROUNDED) count_pass(std::integral_constant<int, COUNT_ROUNDED>{}, sc, t32);
+            else count_pass(std::integral_constant<int, COUNT_TIED>{}, sc, t32);
+            __syncthreads();
+            if (warp == 0) bucket_step<ROW_COPIES>(hist, st, sc, lane, &s_long);
+            __syncthreads();
+            if (!st.pending) break;
+            const bool was_rounded = sc.stage == STAGE_ROUNDED;
+            if (!sched_next<BF16>(sc, s_long != 0u, p.idx_bits)) break;
+            if (was_rounded && s_long && tid == 0) st.base = 0ull;     // read again only after the next barrier
+        }
 
-    // the 8 signed weights and scales of chunk q
-    auto fetch = [&](int64_t q, float (&w)[8], float (&sc)[8]) {
-        Chunk<BF16> ch;
-        chunk_from<BF16>(ch, reinterpret_cast<const uint4 *>(line_mem + q * 8));
-#pragma unroll
-        for (int j = 0; j < 8; ++j) w[j] = chunk_float<BF16>(ch, j);
+        // ---------------------------------------------------------------- emit in place
+        const LineResult res = line_result(st, idx_top);
+        for (int64_t q = tid; q < nchunks; q += ROW_THREADS) {
+            float a[8], s[8];
+            fetch(q, a, s);
+            uint32_t keep = 0u;
+    #pragma unroll
+            for (int j = 0; j < 8; ++j)
+                if (q * 8 + j < p.L && keeps(res, a[j], s[j], q * 8 + j)) keep |= 1u << j;
+            const int64_t e0 = q * 8;
+            const int64_t left = p.L - e0;
+            const int nvalid = left >= 8 ? 8 : (int)left;
+            if (p.mask) DASS_ST(&reinterpret_cast<uint8_t *>(p.mask + row * p.wpr)[q], (uint8_t)keep);   // byte q = columns 8q..8q+7
+            if (p.Wp) {
+                Chunk<BF16> ch;
+                chunk_from<BF16>(ch, reinterpret_cast<const uint4 *>(line_mem + e0));
+                chunk_apply_mask<BF16>(ch, keep);
+                chunk_store<BF16>(ch, p.Wp, row * p.ld + e0, nvalid);
+            }
+        }
+        __syncthreads();                             // the next line reuses the shared memory
+    }
+}
+
+// ---------------------------------------------------------------- lines that are matrix rows: two streaming passes
+// One CTA per row and nothing cached: the first pass reads the row and fills the window's histogram, one warp finds
+// the bin that holds the cut, and the second pass reads the row again (from L2) and writes the outputs -- every
+// element above that bin stays, every element below it goes, and the handful inside it are set aside, ranked by one
+// warp at the end and patched into the outputs.  A row whose window misses, or whose bin holds too many elements,
+// is put on a list for the radix kernel.
+constexpr int RS_THREADS = 256;
+
+template <bool BF16>
+__global__ void __launch_bounds__(RS_THREADS, 4) select_rows_stream_kernel(const SelectParams p)
+{
+    using elem_t = typename std::conditional<BF16, uint16_t, uint32_t>::type;
+    __shared__ uint32_t hist[HBINS];
+    __shared__ FastLine fl;
+    __shared__ CandSet cand;
+    __shared__ uint32_t cand_raw[CAND_CAP];          // the stored weights of the elements set aside
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int64_t row = blockIdx.x;
+    const int64_t nchunks = p.lpad >> 3;
+    const int64_t nfull = p.L >> 3;                  // chunks whose 8 elements all exist
+    const float line_scale = p.scale_along_line ? 0.0f : DASS_LD(&p.scale[row]);
+    const elem_t *wrow = static_cast<const elem_t *>(p.W) + row * p.ld;
+
+    // the 8 weights of chunk q as stored, and their scales
+    auto load_chunk = [&](int64_t q, Chunk<BF16> &ch, float (&sc)[8]) {
+        const uint4 *src = reinterpret_cast<const uint4 *>(wrow + q * 8);
+        const uint4 v0 = DASS_LD_G(src);
+        ch.w[0] = v0.x; ch.w[1] = v0.y; ch.w[2] = v0.z; ch.w[3] = v0.w;
+        if constexpr (!BF16) {
+            const uint4 v1 = DASS_LD_G(src + 1);             // a row's pitch covers whole 8-element chunks
+            ch.w[4] = v1.x; ch.w[5] = v1.y; ch.w[6] = v1.z; ch.w[7] = v1.w;
+        }
         if (p.scale_along_line) {
             const float4 s0 = DASS_LD_G(reinterpret_cast<const float4 *>(p.scale + q * 8));
             const float4 s1 = DASS_LD_G(reinterpret_cast<const float4 *>(p.scale + q * 8) + 1);   // the vector is padded to 8
@@ -670,61 +600,148 @@ __global__ void __launch_bounds__(ROW_THREADS) select_rows_kernel(const SelectPa
             for (int j = 0; j < 8; ++j) sc[j] = line_scale;
         }
     };
-    uint32_t *my_hist = hist + (lane % ROW_COPIES) * HBINS;
-    auto count_pass = [&](auto mode_tag, const Sched &sc, uint32_t t32) {
-        constexpr int MODE = decltype(mode_tag)::value;
-        for (int64_t q = tid; q < nfull; q += ROW_THREADS) {
-            float w[8], s[8];
-            fetch(q, w, s);
+    // the 8 keys of a chunk: bits of fl32(|w| * scale)
+    auto keys_of = [&](const Chunk<BF16> &ch, const float (&sc)[8], uint32_t (&key)[8]) {
 #pragma unroll
-            for (int j = 0; j < 8; ++j) count_element<MODE>(my_hist, st, t32, w[j], s[j], (uint32_t)(q * 8 + j), sc, idx_top);
+        for (int j = 0; j < 8; ++j) {
+            if constexpr (BF16) key[j] = __float_as_uint((j & 1) ? prod_hi(ch.w[j >> 1], sc[j]) : prod_lo(ch.w[j >> 1], sc[j]));
+            else key[j] = __float_as_uint(fabsf(__uint_as_float(ch.w[j])) * sc[j]);
         }
-        if (tid == 0 && nfull < nchunks) {           // the ragged last chunk
-            float w[8], s[8];
-            fetch(nfull, w, s);
-#pragma unroll
-            for (int j = 0; j < 8; ++j)
-                if (nfull * 8 + j < p.L) count_element<MODE>(my_hist, st, t32, w[j], s[j], (uint32_t)(nfull * 8 + j), sc, idx_top);
+    };
+    // runs f(q, chunk, scales, valid elements) over the row, two chunks of a thread in flight
+    auto sweep = [&](auto &&f) {
+        int64_t q = tid;
+        for (; q + RS_THREADS < nfull; q += 2 * RS_THREADS) {
+            Chunk<BF16> ch0, ch1;
+            float s0[8], s1[8];
+            load_chunk(q, ch0, s0);
+            load_chunk(q + RS_THREADS, ch1, s1);
+            f(q, ch0, s0, 8);
+            f(q + RS_THREADS, ch1, s1, 8);
+        }
+        for (; q < nchunks; q += RS_THREADS) {
+            Chunk<BF16> ch;
+            float sc[8];
+            load_chunk(q, ch, sc);
+            const int64_t left = p.L - q * 8;
+            f(q, ch, sc, left >= 8 ? 8 : (int)left);
         }
     };
 
-    Sched sc;
-    sched_begin(sc, STAGE_ROUNDED, 31, 0);
-    for (;;) {
-        for (int i = tid; i < ROW_COPIES * HBINS; i += ROW_THREADS) hist[i] = 0u;
-        __syncthreads();
-        const uint32_t t32 = st.tau32;
-        const int mode = count_mode(sc);
-        if (mode == COUNT_ALL) count_pass(std::integral_constant<int, COUNT_ALL>{}, sc, t32);
-        else if (mode == COUNT_ROUNDED) count_pass(std::integral_constant<int, COUNT_ROUNDED>{}, sc, t32);
-        else count_pass(std::integral_constant<int, COUNT_TIED>{}, sc, t32);
-        __syncthreads();
-        if (warp == 0) bucket_step<ROW_COPIES>(hist, st, sc, lane, &s_long);
-        __syncthreads();
-        if (!st.pending) break;
-        const bool was_rounded = sc.stage == STAGE_ROUNDED;
-        if (!sched_next<BF16>(sc, s_long != 0u, p.idx_bits)) break;
-        if (was_rounded && s_long && tid == 0) st.base = 0ull;     // read again only after the next barrier
+    // ---------------------------------------------------------------- the window, from a sample's exponents
+    for (int i = tid; i < 256; i += RS_THREADS) hist[i] = 0u;
+    if (tid == 0) fl.ok = 0u;
+    __syncthreads();
+    for (int i = tid; i < WIN_SAMPLE; i += RS_THREADS) {
+        const int64_t e = ((int64_t)i * p.L) / WIN_SAMPLE;
+        float wf;
+        if constexpr (BF16) wf = __uint_as_float((uint32_t)DASS_LD_G(wrow + e) << 16);
+        else wf = __uint_as_float(DASS_LD_G(wrow + e));
+        atomicAdd(hist + (product_key(wf, p.scale_along_line ? DASS_LD_G(p.scale + e) : line_scale) >> 23), 1u);
+    }
+    __syncthreads();
+    if (warp == 0) window_from_exponents(hist, fl, win_target(p.k, p.L), lane);
+    __syncthreads();
+    for (int i = tid; i < HBINS; i += RS_THREADS) hist[i] = 0u;
+    __syncthreads();
+
+    // ---------------------------------------------------------------- first pass: histogram of the window
+    {
+        const uint32_t lo = fl.lo;
+        uint32_t above = 0u;
+        sweep([&](int64_t, const Chunk<BF16> &ch, const float (&sc)[8], int nvalid) {
+            uint32_t key[8];
+            keys_of(ch, sc, key);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                if (j < nvalid) {
+                    const uint32_t off = key[j] - lo;
+                    if (off < WIN_SPAN) atomicAdd(hist + (off >> WIN_SHIFT), 1u);
+                    else above += key[j] > lo ? 1u : 0u;
+                }
+            }
+        });
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) above += __shfl_xor_sync(FULL_MASK, above, off);
+        if (lane == 0 && above) atomicAdd(&fl.above, above);
+    }
+    __syncthreads();
+    if (warp == 0) bracket_pick_bin(hist, fl, p.k, lane);
+    __syncthreads();
+    if (!fl.ok) {                                    // the same for every thread: left to the radix kernel
+        if (tid == 0) DASS_ST(&p.line_list[atomicAdd(p.line_count, 1u)], (uint32_t)row);
+        return;
     }
 
-    // ---------------------------------------------------------------- emit in place
-    const LineResult res = line_result(st, idx_top);
-    for (int64_t q = tid; q < nchunks; q += ROW_THREADS) {
-        float a[8], s[8];
-        fetch(q, a, s);
-        uint32_t keep = 0u;
+    // ---------------------------------------------------------------- second pass: outputs, the cut's bin set aside
+    {
+        const uint32_t blo = fl.blo, bhi = fl.bhi, bw = bhi - blo;
+        sweep([&](int64_t q, Chunk<BF16> &ch, const float (&sc)[8], int nvalid) {
+            uint32_t key[8];
+            keys_of(ch, sc, key);
+            bool some = false;                       // an element of this chunk lies in the cut's bin
 #pragma unroll
-        for (int j = 0; j < 8; ++j)
-            if (q * 8 + j < p.L && keeps(res, a[j], s[j], q * 8 + j)) keep |= 1u << j;
-        const int64_t e0 = q * 8;
-        const int64_t left = p.L - e0;
-        const int nvalid = left >= 8 ? 8 : (int)left;
-        if (p.mask) DASS_ST(&reinterpret_cast<uint8_t *>(p.mask + row * p.wpr)[q], (uint8_t)keep);   // byte q = columns 8q..8q+7
-        if (p.Wp) {
-            Chunk<BF16> ch;
-            chunk_from<BF16>(ch, reinterpret_cast<const uint4 *>(line_mem + e0));
-            chunk_apply_mask<BF16>(ch, keep);
-            chunk_store<BF16>(ch, p.Wp, row * p.ld + e0, nvalid);
+            for (int j = 0; j < 8; ++j) some |= j < nvalid && key[j] - blo < bw;
+            if (some) {
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    if (j < nvalid && key[j] - blo < bw) {
+                        const uint32_t slot = atomicAdd(&fl.ncoll, 1u);
+                        if (slot < (uint32_t)CAND_CAP) {
+                            const float wf = chunk_float<BF16>(ch, j);
+                            cand.key[slot] = key[j]; cand.idx[slot] = (uint32_t)(q * 8 + j); cand.k64[slot] = exact_key(fabsf(wf), sc[j]);
+                            cand_raw[slot] = __float_as_uint(wf);
+                        }
+                    }
+                }
+            }
+            // below bhi: pruned here (the bin's survivors come back at the end)
+            uint32_t keep = 0u;
+            if constexpr (BF16) {
+                uint32_t z[4];
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    z[k] = pn_prmt(key[2 * k] - bhi, key[2 * k + 1] - bhi, 0xFFBBu);   // keys are below 2^31: the sign is the order
+                    ch.w[k] &= ~z[k];
+                }
+                // lane masks to bits: even columns sit in the low lanes, odd ones 16 bits up
+                const uint32_t x = (z[0] & 0x00020001u) | (z[1] & 0x00080004u) | (z[2] & 0x00200010u) | (z[3] & 0x00800040u);
+                keep = ~(x | (x >> 16)) & 0xffu;
+            } else {
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    const uint32_t z = (uint32_t)((int32_t)(key[j] - bhi) >> 31);
+                    ch.w[j] &= ~z;
+                    keep |= ~z & (1u << j);
+                }
+            }
+            keep &= (1u << nvalid) - 1u;
+            if (p.mask) DASS_ST(&reinterpret_cast<uint8_t *>(p.mask + row * p.wpr)[q], (uint8_t)keep);   // byte q = columns 8q..8q+7
+            if (p.Wp) chunk_store<BF16>(ch, p.Wp, row * p.ld + q * 8, nvalid);
+        });
+    }
+    __syncthreads();
+
+    // ---------------------------------------------------------------- the cut's bin: ranked, survivors patched in
+    if (warp == 0) {
+        bracket_rank(cand, fl, lane);
+        __syncwarp();
+        if (fl.ok) {                                 // always: the bin's count was checked and the keys are distinct
+            const LineResult res = fl.res;
+            const int n = (int)fl.ncoll;
+            for (int i = lane; i < n; i += 32) {
+                const uint32_t key = cand.key[i], idx = cand.idx[i];
+                const unsigned long long k64 = cand.k64[i];
+                const bool stays = key > res.tau32 ||
+                                   (key == res.tau32 && (!res.exact || k64 > res.tau64 || (k64 == res.tau64 && (long long)idx <= res.cut)));
+                if (stays) {
+                    if (p.mask) atomicOr(p.mask + row * p.wpr + (idx >> 5), 1u << (idx & 31u));
+                    if (p.Wp) {
+                        if constexpr (BF16) DASS_ST(static_cast<uint16_t *>(p.Wp) + row * p.ld + idx, (uint16_t)(cand_raw[i] >> 16));
+                        else DASS_ST(static_cast<uint32_t *>(p.Wp) + row * p.ld + idx, cand_raw[i]);
+                    }
+                }
+            }
         }
     }
 }
@@ -1244,12 +1261,28 @@ size_t select_row_smem_bytes(int64_t L, bool bf16)
 }
 
 template <bool BF16>
-static cudaError_t launch_rows(const SelectParams &p, cudaStream_t st)
+static cudaError_t launch_rows(SelectParams p, uint32_t *line_count, uint32_t *line_list, cudaStream_t st)
 {
     const size_t smem = select_row_smem_bytes(p.L, BF16);
     cudaError_t e = cudaFuncSetAttribute(select_rows_kernel<BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    select_rows_kernel<BF16><<<(unsigned)p.rows, ROW_THREADS, smem, st>>>(p);
+    if (p.L < FAST_MIN_L) {                          // short lines: the radix kernel alone, one CTA per row
+        p.line_count = nullptr; p.line_list = nullptr;
+        select_rows_kernel<BF16><<<(unsigned)p.rows, ROW_THREADS, smem, st>>>(p);
+        return cudaGetLastError();
+    }
+    // the streaming kernel decides the rows it can and lists the others; the radix kernel works the list off
+    p.line_count = line_count; p.line_list = line_list;
+    e = cudaMemsetAsync(line_count, 0, sizeof(uint32_t), st);
+    if (e != cudaSuccess) return e;
+    select_rows_stream_kernel<BF16><<<(unsigned)p.rows, RS_THREADS, 0, st>>>(p);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    int per_sm = 1;
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, select_rows_kernel<BF16>, ROW_THREADS, smem);
+    if (e != cudaSuccess) return e;
+    const int64_t resident = (int64_t)device_sm_count() * (per_sm > 0 ? per_sm : 1);
+    select_rows_kernel<BF16><<<(unsigned)(p.rows < resident ? p.rows : resident), ROW_THREADS, smem, st>>>(p);
     return cudaGetLastError();
 }
 
@@ -1264,21 +1297,29 @@ static cudaError_t launch_cols(const SelectParams &p, cudaStream_t st)
 }
 
 size_t select_results_bytes(int64_t cols) { return ((size_t)cols * sizeof(LineResult) + 31) / 32 * 32; }
+size_t select_scale_bytes(int64_t n) { return (size_t)((n + 7) / 8 * 8) * sizeof(float); }
+// [per-column results][scale vector padded to 8][count of undecided rows, 32 bytes][their indices]
+size_t select_workspace_bytes(int64_t rows, int64_t cols, bool norm_cols)
+{
+    return select_results_bytes(cols) + select_scale_bytes(norm_cols ? cols : rows) + 32 + (size_t)rows * sizeof(uint32_t);
+}
 
 cudaError_t select_unstructured_launch(const void *W, int64_t rows, int64_t cols, int64_t ld, bool bf16,
                                        const float *norm, bool norm_cols, float alpha, uint32_t k, bool line_is_row,
                                        uint32_t *mask_bits, void *W_pruned, void *workspace, cudaStream_t st)
 {
-    // workspace: [per-column results][scale vector padded to 8]
     LineResult *results = static_cast<LineResult *>(workspace);
     float *scale_ws = reinterpret_cast<float *>(static_cast<unsigned char *>(workspace) + select_results_bytes(cols));
     const int64_t n_norm = norm_cols ? cols : rows;
+    uint32_t *line_count = reinterpret_cast<uint32_t *>(reinterpret_cast<unsigned char *>(scale_ws) + select_scale_bytes(n_norm));
+    uint32_t *line_list = line_count + 8;
     const int64_t n_pad = (n_norm + 7) / 8 * 8;
     scale_vector_kernel<<<(unsigned)((n_pad + 255) / 256), 256, 0, st>>>(norm, n_norm, n_pad, (int)scale_mode_for(alpha), alpha, scale_ws);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     SelectParams p;
     p.W = W; p.Wp = W_pruned; p.mask = mask_bits; p.scale = scale_ws; p.results = results;
+    p.line_count = nullptr; p.line_list = nullptr;
     p.rows = rows; p.cols = cols; p.ld = ld;
     p.wpr = (cols + 31) / 32;
     p.L = line_is_row ? cols : rows;
@@ -1292,7 +1333,7 @@ cudaError_t select_unstructured_launch(const void *W, int64_t rows, int64_t cols
             e = cudaMemsetAsync(mask_bits, 0, (size_t)rows * p.wpr * sizeof(uint32_t), st);
             if (e != cudaSuccess) return e;
         }
-        return bf16 ? launch_rows<true>(p, st) : launch_rows<false>(p, st);
+        return bf16 ? launch_rows<true>(p, line_count, line_list, st) : launch_rows<false>(p, line_count, line_list, st);
     }
     e = bf16 ? launch_cols<true>(p, st) : launch_cols<false>(p, st);
     if (e != cudaSuccess) return e;
@@ -1320,8 +1361,7 @@ extern "C" dass_status dass_select_workspace_bytes(int64_t rows, int64_t cols, d
     if (!bytes) return DASS_ERR_NULL;
     if (norm_axis != DASS_AXIS_ROWS && norm_axis != DASS_AXIS_COLS) return DASS_ERR_DTYPE;
     if (rows < 1 || cols < 1) return DASS_ERR_SHAPE;
-    const int64_t n = norm_axis == DASS_AXIS_ROWS ? rows : cols;
-    *bytes = select_results_bytes(cols) + (size_t)((n + 7) / 8 * 8) * sizeof(float);
+    *bytes = select_workspace_bytes(rows, cols, norm_axis == DASS_AXIS_COLS);
     return DASS_OK;
 }
 
