@@ -47,6 +47,7 @@ struct SelectParams {
     uint32_t k;          // survivors per line
     int idx_bits;        // bits of L - 1 (at least 1): width of the index part of the key
     int scale_along_line;   // 1: scale[e] varies along the line; 0: scale[line]
+    int margin;             // sampled bracket: sample positions on either side of the wanted rank (four standard deviations)
     uint32_t *line_count;   // row lines: how many lines the streaming kernel left undecided, and which
     uint32_t *line_list;    // (both null: the radix kernel takes every row)
 };
@@ -290,6 +291,7 @@ struct FastLine {                // bracket state of one comparison line (shared
     uint32_t blo, bhi;           // the bin of the bracket that holds the cut
     int sh;                      // bin = (key - lo) >> sh
     uint32_t above;              // elements with key >= hi
+    uint32_t below;              // elements with key < lo (streaming kernels: above = L - below - inside)
     uint32_t krem2;              // rank, from the top and 1-based, of the last survivor inside [blo, bhi)
     uint32_t ncoll;              // elements collected from that bin
     uint32_t bucket;             // elements the histogram saw in that bin
@@ -337,19 +339,61 @@ __device__ __forceinline__ void window_from_exponents(const uint32_t *eh, FastLi
         f.lo = (uint32_t)e0 << 23;
         f.hi = f.lo + WIN_SPAN;
         f.sh = WIN_SHIFT;
-        f.above = 0u; f.ncoll = 0u; f.ok = 1u; f.krem2 = 0u; f.bucket = 0u; f.blo = 0u; f.bhi = 0u;
+        f.above = 0u; f.below = 0u; f.ncoll = 0u; f.ok = 1u; f.krem2 = 0u; f.bucket = 0u; f.blo = 0u; f.bhi = 0u;
     }
 }
 
-// Rank, from the top, of the sample key that stands for the line's k-th largest.
-__device__ __forceinline__ uint32_t win_target(uint32_t k, int64_t L)
+// Rank, from the top, of the key that stands for the line's k-th largest in a sample of S.
+__device__ __forceinline__ uint32_t win_target(uint32_t k, int64_t L, int S = WIN_SAMPLE)
 {
-    const int64_t t = ((int64_t)k * WIN_SAMPLE + L - 1) / L;
-    return (uint32_t)(t < 1 ? 1 : (t > WIN_SAMPLE ? WIN_SAMPLE : t));
+    const int64_t t = ((int64_t)k * S + L - 1) / L;
+    return (uint32_t)(t < 1 ? 1 : (t > S ? S : t));
+}
+
+// One warp: narrows a line's window to a bracket [lo, hi) from the fine histogram of a larger sample (FINE_BINS bins
+// of 2^FINE_SHIFT keys from the window's start; n_over = sample keys above the window).  With the sample sorted from
+// the top, the line's cut lies between the sample's (t - m)-th and (t + m)-th key unless the sample is m positions
+// off the expected rank (m is four standard deviations of that rank, set by the host); the bracket is those two
+// keys' fine bins and what lies between.  About 2m/S of the line plus two fine bins falls inside; everything else
+// is only counted.  A miss shows in bracket_pick_bin's counts and sends the line to the radix select.
+constexpr int FINE_SHIFT = 18;                  // 32 fine bins per octave
+constexpr int FINE_BINS = 256;                  // the 8 octaves of the window
+__device__ __forceinline__ void bracket_from_fine(const uint32_t *fh, uint32_t n_over, FastLine &f, int t, int m, int lane)
+{
+    uint32_t c[8], mine = 0u;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) { c[i] = fh[lane * 8 + i]; mine += c[i]; }
+    uint32_t v = mine;                                // becomes the sum over lanes >= this one
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const uint32_t u = __shfl_down_sync(FULL_MASK, v, off);
+        if (lane + off < 32) v += u;
+    }
+    // C(b) = sample keys in fine bin b or higher; walking this lane's bins from the top
+    int cum = (int)(n_over + (v - mine));
+    int b_hi = FINE_BINS, b_lo = 0;                   // min{b : C(b) < t - m} (C(256) = n_over);  max{b : C(b) >= t + m}
+    if (cum < t - m) b_hi = lane * 8 + 8;
+#pragma unroll
+    for (int i = 7; i >= 0; --i) {
+        cum += (int)c[i];
+        const int b = lane * 8 + i;
+        if (cum < t - m) b_hi = b;
+        if (cum >= t + m && b > b_lo) b_lo = b;       // first hit from the top is the largest b
+    }
+    b_hi = __reduce_min_sync(FULL_MASK, b_hi);
+    b_lo = __reduce_max_sync(FULL_MASK, b_lo);
+    if (lane == 0) {
+        const uint32_t wlo = f.lo;
+        f.lo = wlo + ((uint32_t)b_lo << FINE_SHIFT);
+        f.hi = wlo + ((uint32_t)b_hi << FINE_SHIFT);
+        const uint32_t span = f.hi - f.lo - 1u;       // largest offset inside the bracket
+        const int bits = 32 - __clz(span);
+        f.sh = bits > HB ? bits - HB : 0;
+    }
 }
 
 // One warp: the bin of the window's histogram that holds the line's last survivor.
-__device__ __forceinline__ void bracket_pick_bin(const uint32_t *h, FastLine &f, uint32_t k, int lane)
+__device__ __forceinline__ void bracket_pick_bin(const uint32_t *h, FastLine &f, uint32_t k, int lane, int64_t L_if_below = -1)
 {
     const uint32_t *mine_bins = h + lane * 64;
     uint32_t lane_sum = 0u;
@@ -362,7 +406,8 @@ __device__ __forceinline__ void bracket_pick_bin(const uint32_t *h, FastLine &f,
         if (lane + off < 32) v += t;
     }
     const uint32_t total = __shfl_sync(FULL_MASK, v, 0);
-    const uint32_t above_all = f.above;
+    // the elements above the bracket: counted directly, or what is left of the line after those below and inside it
+    const uint32_t above_all = L_if_below < 0 ? f.above : (uint32_t)L_if_below - f.below - total;
     const bool in_range = k > above_all && k - above_all <= total;     // the cut lies inside the bracket
     const uint32_t krem = k - above_all;
     uint32_t above = v - lane_sum;
@@ -565,12 +610,15 @@ __global__ void __launch_bounds__(ROW_THREADS) select_rows_kernel(const SelectPa
 // warp at the end and patched into the outputs.  A row whose window misses, or whose bin holds too many elements,
 // is put on a list for the radix kernel.
 constexpr int RS_THREADS = 256;
+constexpr int RS_SAMPLE = 1024;                 // evenly spaced elements of a row that place its bracket
 
-template <bool BF16>
+// ALONG: the scale varies along the row (one per column) rather than being one number per row.
+template <bool BF16, bool ALONG>
 __global__ void __launch_bounds__(RS_THREADS, 4) select_rows_stream_kernel(const SelectParams p)
 {
     using elem_t = typename std::conditional<BF16, uint16_t, uint32_t>::type;
     __shared__ uint32_t hist[HBINS];
+    __shared__ uint32_t s_over;                      // sample keys above the window
     __shared__ FastLine fl;
     __shared__ CandSet cand;
     __shared__ uint32_t cand_raw[CAND_CAP];          // the stored weights of the elements set aside
@@ -579,8 +627,9 @@ __global__ void __launch_bounds__(RS_THREADS, 4) select_rows_stream_kernel(const
     const int64_t row = blockIdx.x;
     const int64_t nchunks = p.lpad >> 3;
     const int64_t nfull = p.L >> 3;                  // chunks whose 8 elements all exist
-    const float line_scale = p.scale_along_line ? 0.0f : DASS_LD(&p.scale[row]);
+    const float line_scale = ALONG ? 0.0f : DASS_LD(&p.scale[row]);
     const elem_t *wrow = static_cast<const elem_t *>(p.W) + row * p.ld;
+    const uint32_t hist_s = smem_u32(hist);
 
     // the 8 weights of chunk q as stored, and their scales
     auto load_chunk = [&](int64_t q, Chunk<BF16> &ch, float (&sc)[8]) {
@@ -591,7 +640,7 @@ __global__ void __launch_bounds__(RS_THREADS, 4) select_rows_stream_kernel(const
             const uint4 v1 = DASS_LD_G(src + 1);             // a row's pitch covers whole 8-element chunks
             ch.w[4] = v1.x; ch.w[5] = v1.y; ch.w[6] = v1.z; ch.w[7] = v1.w;
         }
-        if (p.scale_along_line) {
+        if constexpr (ALONG) {
             const float4 s0 = DASS_LD_G(reinterpret_cast<const float4 *>(p.scale + q * 8));
             const float4 s1 = DASS_LD_G(reinterpret_cast<const float4 *>(p.scale + q * 8) + 1);   // the vector is padded to 8
             sc[0] = s0.x; sc[1] = s0.y; sc[2] = s0.z; sc[3] = s0.w; sc[4] = s1.x; sc[5] = s1.y; sc[6] = s1.z; sc[7] = s1.w;
@@ -628,45 +677,68 @@ __global__ void __launch_bounds__(RS_THREADS, 4) select_rows_stream_kernel(const
         }
     };
 
-    // ---------------------------------------------------------------- the window, from a sample's exponents
-    for (int i = tid; i < 256; i += RS_THREADS) hist[i] = 0u;
-    if (tid == 0) fl.ok = 0u;
+    // ---------------------------------------------------------------- the bracket, from a sample of the row
+    constexpr int PER_THREAD = RS_SAMPLE / RS_THREADS;
+    uint32_t skey[PER_THREAD];
+    for (int i = tid; i < 256 + FINE_BINS; i += RS_THREADS) hist[i] = 0u;      // exponent counts, then fine bins
+    if (tid == 0) { fl.ok = 0u; s_over = 0u; }
     __syncthreads();
-    for (int i = tid; i < WIN_SAMPLE; i += RS_THREADS) {
-        const int64_t e = ((int64_t)i * p.L) / WIN_SAMPLE;
+#pragma unroll
+    for (int u = 0; u < PER_THREAD; ++u) {
+        const int64_t e = ((int64_t)(tid + u * RS_THREADS) * p.L) / RS_SAMPLE;
         float wf;
         if constexpr (BF16) wf = __uint_as_float((uint32_t)DASS_LD_G(wrow + e) << 16);
         else wf = __uint_as_float(DASS_LD_G(wrow + e));
-        atomicAdd(hist + (product_key(wf, p.scale_along_line ? DASS_LD_G(p.scale + e) : line_scale) >> 23), 1u);
+        float sv = line_scale;
+        if constexpr (ALONG) sv = DASS_LD_G(p.scale + e);
+        skey[u] = product_key(wf, sv);
+    }
+#pragma unroll
+    for (int u = 0; u < PER_THREAD; ++u) atomicAdd(hist + (skey[u] >> 23), 1u);
+    __syncthreads();
+    const int target = (int)win_target(p.k, p.L, RS_SAMPLE);
+    if (warp == 0) window_from_exponents(hist, fl, (uint32_t)target, lane);
+    __syncthreads();
+    {
+        const uint32_t wlo = fl.lo;
+#pragma unroll
+        for (int u = 0; u < PER_THREAD; ++u) {
+            const uint32_t off = skey[u] - wlo;
+            if (off < WIN_SPAN) atomicAdd(hist + 256 + (off >> FINE_SHIFT), 1u);
+            else if (skey[u] > wlo) atomicAdd(&s_over, 1u);
+        }
     }
     __syncthreads();
-    if (warp == 0) window_from_exponents(hist, fl, win_target(p.k, p.L), lane);
+    if (warp == 0) bracket_from_fine(hist + 256, s_over, fl, target, p.margin, lane);
     __syncthreads();
     for (int i = tid; i < HBINS; i += RS_THREADS) hist[i] = 0u;
     __syncthreads();
 
-    // ---------------------------------------------------------------- first pass: histogram of the window
-    {
-        const uint32_t lo = fl.lo;
-        uint32_t above = 0u;
+    // ---------------------------------------------------------------- first pass: histogram of the bracket
+    {   // only the elements inside the bracket touch the histogram (a predicated reduction: the other lanes cost
+        // the shared-memory pipe nothing); those below it are counted, those above it follow from the line's length
+        const uint32_t lo = fl.lo, span = fl.hi - fl.lo;
+        const int sh = fl.sh;
+        uint32_t below = 0u;
         sweep([&](int64_t, const Chunk<BF16> &ch, const float (&sc)[8], int nvalid) {
             uint32_t key[8];
             keys_of(ch, sc, key);
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
                 if (j < nvalid) {
-                    const uint32_t off = key[j] - lo;
-                    if (off < WIN_SPAN) atomicAdd(hist + (off >> WIN_SHIFT), 1u);
-                    else above += key[j] > lo ? 1u : 0u;
+                    const uint32_t off = key[j] - lo;             // keys are below 2^31: the top bit says "below lo"
+                    asm volatile("{\n\t.reg .pred q;\n\tsetp.lt.u32 q, %0, %1;\n\t@q red.shared.add.u32 [%2], 1;\n\t}"
+                                 ::"r"(off), "r"(span), "r"(hist_s + ((off >> sh) << 2)) : "memory");
+                    below += off >> 31;
                 }
             }
         });
 #pragma unroll
-        for (int off = 16; off > 0; off >>= 1) above += __shfl_xor_sync(FULL_MASK, above, off);
-        if (lane == 0 && above) atomicAdd(&fl.above, above);
+        for (int off = 16; off > 0; off >>= 1) below += __shfl_xor_sync(FULL_MASK, below, off);
+        if (lane == 0 && below) atomicAdd(&fl.below, below);
     }
     __syncthreads();
-    if (warp == 0) bracket_pick_bin(hist, fl, p.k, lane);
+    if (warp == 0) bracket_pick_bin(hist, fl, p.k, lane, p.L);
     __syncthreads();
     if (!fl.ok) {                                    // the same for every thread: left to the radix kernel
         if (tid == 0) DASS_ST(&p.line_list[atomicAdd(p.line_count, 1u)], (uint32_t)row);
@@ -1275,7 +1347,8 @@ static cudaError_t launch_rows(SelectParams p, uint32_t *line_count, uint32_t *l
     p.line_count = line_count; p.line_list = line_list;
     e = cudaMemsetAsync(line_count, 0, sizeof(uint32_t), st);
     if (e != cudaSuccess) return e;
-    select_rows_stream_kernel<BF16><<<(unsigned)p.rows, RS_THREADS, 0, st>>>(p);
+    if (p.scale_along_line) select_rows_stream_kernel<BF16, true><<<(unsigned)p.rows, RS_THREADS, 0, st>>>(p);
+    else select_rows_stream_kernel<BF16, false><<<(unsigned)p.rows, RS_THREADS, 0, st>>>(p);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     int per_sm = 1;
@@ -1328,6 +1401,10 @@ cudaError_t select_unstructured_launch(const void *W, int64_t rows, int64_t cols
     p.idx_bits = 1;
     while (((int64_t)1 << p.idx_bits) < p.L) ++p.idx_bits;
     p.scale_along_line = (line_is_row == norm_cols) ? 1 : 0;   // the norm index runs along the line
+    {   // four standard deviations of the rank of a sample quantile, in sample positions, plus slack
+        const double q = (double)(p.L - (int64_t)k) / (double)p.L;
+        p.margin = (int)std::ceil(4.0 * std::sqrt((double)RS_SAMPLE * q * (1.0 - q))) + 2;
+    }
     if (line_is_row) {
         if (mask_bits) {   // the kernel writes whole bytes of real columns; the padding of each mask row must read 0
             e = cudaMemsetAsync(mask_bits, 0, (size_t)rows * p.wpr * sizeof(uint32_t), st);
