@@ -58,7 +58,8 @@ typedef enum {
     DASS_ERR_UNSUPPORTED = 5,  /* a valid request the library has no kernel for */
     DASS_ERR_WORKSPACE = 6,    /* workspace NULL or smaller than the query says */
     DASS_ERR_CUDA = 7,         /* a CUDA runtime / driver call failed */
-    DASS_ERR_TIMEOUT = 8       /* a bounded device-side wait ran out (reported by dass_calib_status) */
+    DASS_ERR_TIMEOUT = 8,      /* a bounded device-side wait ran out (reported by dass_calib_status / dass_prune_status) */
+    DASS_ERR_INTERNAL = 9      /* a consistency check between two passes of a kernel chain failed (dass_prune_status) */
 } dass_status;
 
 typedef enum { DASS_BF16 = 0, DASS_F32 = 1 } dass_dtype;
@@ -193,10 +194,12 @@ dass_status dass_prune_nm(const void *W, int64_t rows, int64_t cols, int64_t ld,
                           const float *norm, dass_axis norm_axis, float alpha,
                           int n_keep, int m, dass_axis group_axis,
                           uint32_t *mask_bits, void *W_pruned, void *values, uint32_t *meta, void *cuda_stream);
-/* The tuned kernels behind dass_prune_nm (bf16, 2:4 and 4:8) receive their tiles through bulk tensor copies and
- * wait for each on a barrier; every such wait is bounded (2 s).  Waits for `cuda_stream`, then returns DASS_OK, or
- * DASS_ERR_TIMEOUT if a wait of any dass_prune_nm call on the current device ran out since the last query (that
- * call's outputs are then incomplete; the context stays usable) and clears the record.  CUDA failure: DASS_ERR_CUDA. */
+/* The tuned kernels behind dass_prune_nm (bf16, 2:4 and 4:8) and behind dass_select_unstructured (bf16, lines that
+ * are columns) receive their tiles through bulk tensor copies and wait for each on a barrier; every such wait is
+ * bounded (2 s).  Waits for `cuda_stream`, then returns DASS_OK, or DASS_ERR_TIMEOUT if a wait of any such call on
+ * the current device ran out since the last query (that call's outputs are then incomplete; the context stays
+ * usable), or DASS_ERR_INTERNAL if the passes of a dass_select_unstructured call disagreed on how many elements lie
+ * at a column's cut (outputs of that call unspecified), and clears the record.  CUDA failure: DASS_ERR_CUDA. */
 dass_status dass_prune_status(void *cuda_stream);
 
 /* Eq. 1's input-feature norms (Wanda; the paper prunes the attention projections with it, Section 4.1 "Sparsity"):
@@ -219,9 +222,11 @@ dass_status dass_feature_sumsq(const void *X, int64_t T, int64_t d, int64_t ldx,
  * Score, scale rounding and order are those of dass_score_nm: exact products, higher score first, lower
  * index first.  sparsity in [0, 1).  mask_bits / W_pruned as for dass_score_nm (at least one; mask_bits is
  * written in full, padding bits 0).  workspace: dass_select_workspace_bytes(...) bytes, 16-byte aligned (holds
- * the rounded norm^alpha vector and the per-column thresholds).  A line that is a matrix row is cached in shared
- * memory: rows of more than about 108 000 bf16 or 54 000 f32 elements are DASS_ERR_UNSUPPORTED; lines that are
- * matrix columns have no such limit (below 2^31 elements).
+ * the rounded norm^alpha vector, the per-column thresholds, the rows left to the slower exact kernel and, per
+ * column, the few elements at its cut that are ranked last: about 1.2 KB per column).  A row that the streaming
+ * kernel cannot decide is cached in shared memory by the exact kernel: rows of more than about 108 000 bf16 or
+ * 54 000 f32 elements are DASS_ERR_UNSUPPORTED; lines that are matrix columns have no such limit (below 2^31
+ * elements).  W_pruned may be W itself (in place).
  * Errors: NULL / DTYPE / SHAPE (sizes, sparsity outside [0,1)) / ALIGN / UNSUPPORTED / WORKSPACE / CUDA. */
 dass_status dass_select_workspace_bytes(int64_t rows, int64_t cols, dass_axis norm_axis, size_t *bytes /* HOST */);
 dass_status dass_select_unstructured(const void *W, int64_t rows, int64_t cols, int64_t ld, dass_dtype dt,

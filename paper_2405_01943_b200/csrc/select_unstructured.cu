@@ -31,7 +31,18 @@ struct LineResult {
     unsigned long long tau64;
     long long cut;
     uint32_t tau32;
-    uint32_t exact;
+    uint32_t exact;      // 0 / 1 as above; LINE_BIN: the line is decided up to one histogram bin, see below
+};
+// A column whose cut is known up to a bin [blo, bhi) of rounded products: every element at or above bhi stays,
+// every element below blo goes, and of the `bucket` elements inside the bin the krem2 largest stay.  The emit pass
+// sets those elements aside in per-column lists and a last small kernel ranks them.  Stored in a LineResult as
+// tau32 = bhi, exact = LINE_BIN, tau64 = blo | krem2 << 32, cut = bucket.
+constexpr uint32_t LINE_BIN = 2u;
+struct CandLists {               // per column: how many elements were set aside, and CAND_CAP slots of each array
+    uint32_t *count;
+    uint32_t *key;               // rounded product
+    uint32_t *idx;               // row
+    uint32_t *raw;               // the stored weight, in the upper 16 bits for bf16
 };
 
 struct SelectParams {
@@ -50,6 +61,7 @@ struct SelectParams {
     int margin;             // sampled bracket: sample positions on either side of the wanted rank (four standard deviations)
     uint32_t *line_count;   // row lines: how many lines the streaming kernel left undecided, and which
     uint32_t *line_list;    // (both null: the radix kernel takes every row)
+    uint32_t *cand_count;   // column lines, bf16: per-column count of the elements the emit pass sets aside (cleared here)
 };
 
 // out[i] = fl32(norm[i]^alpha) for i < n, 0 for the padding up to npad (a multiple of 8, so that the selection
@@ -827,7 +839,8 @@ constexpr int COL_THREADS = 1024;
 constexpr int COL_LINES = 8;
 constexpr int COL_COPIES = 1;                   // histogram copies per column (3 measured slower, as for rows)
 
-template <bool BF16>
+// ALONG: the scale varies along the columns (one per row) rather than being one number per column.
+template <bool BF16, bool ALONG>
 __global__ void __launch_bounds__(COL_THREADS, 1) select_cols_kernel(const SelectParams p)
 {
     using elem_t = typename std::conditional<BF16, uint16_t, uint32_t>::type;
@@ -892,12 +905,15 @@ __global__ void __launch_bounds__(COL_THREADS, 1) select_cols_kernel(const Selec
         }
     };
 
-    // ---------------------------------------------------------------- octave window (see the top of the file)
+    // ---------------------------------------------------------------- sampled bracket (see the top of the file)
+    constexpr bool DEFER = BF16;                     // bf16: the column is published at its bin and the emit pass sets the bin's elements aside
     __shared__ FastLine fl[COL_LINES];
-    __shared__ CandSet cand[COL_LINES];
+    __shared__ CandSet cand[DEFER ? 1 : COL_LINES];
+    __shared__ uint32_t s_over[COL_LINES];           // sample keys above a column's window
     bool any_pending = true;
     if (tid < COL_LINES) fl[tid].ok = 0u;
     if (p.L >= FAST_MIN_L) {                         // the same for every thread
+        const uint32_t hist_s = smem_u32(hist);
         // loads one row of the strip (the vector loads of count_pass)
         auto load_row = [&](int64_t r, Chunk<BF16> &ch) {
             const uint4 *src = reinterpret_cast<const uint4 *>(strip + r * p.ld);
@@ -923,7 +939,7 @@ __global__ void __launch_bounds__(COL_THREADS, 1) select_cols_kernel(const Selec
                     row_scale[u] = 0.0f;
                     if (r < p.L) {
                         load_row(r, ch[u]);
-                        if (p.scale_along_line) row_scale[u] = DASS_LD_G(p.scale + r);
+                        if constexpr (ALONG) row_scale[u] = DASS_LD_G(p.scale + r);
                     }
                 }
 #pragma unroll
@@ -932,53 +948,88 @@ __global__ void __launch_bounds__(COL_THREADS, 1) select_cols_kernel(const Selec
                     if (r < p.L) {
 #pragma unroll
                         for (int j = 0; j < COL_LINES; ++j)
-                            f(j, chunk_float<BF16>(ch[u], j), p.scale_along_line ? row_scale[u] : col_scale[j], r);
+                            f(j, chunk_float<BF16>(ch[u], j), ALONG ? row_scale[u] : col_scale[j], r);
                     }
                 }
             }
         };
         uint32_t *ehist = hist;                      // [COL_LINES][256] exponent counts of the sample, before the bins
-        for (int i = tid; i < COL_LINES * 256; i += COL_THREADS) ehist[i] = 0u;
+        uint32_t *fhist = hist + COL_LINES * 256;    // [COL_LINES][FINE_BINS] the sample inside each column's window
+        for (int i = tid; i < COL_LINES * (256 + FINE_BINS); i += COL_THREADS) hist[i] = 0u;
+        if (tid < COL_LINES) s_over[tid] = 0u;
         __syncthreads();
-        if (tid < WIN_SAMPLE) {
-            const int64_t r = ((int64_t)tid * p.L) / WIN_SAMPLE;
+        uint32_t skey[COL_LINES];                    // the sample: one row per thread, all of the strip's columns
+        {
+            const int64_t r = ((int64_t)tid * p.L) / COL_THREADS;
             Chunk<BF16> ch;
             load_row(r, ch);
-            const float rs = p.scale_along_line ? DASS_LD_G(p.scale + r) : 0.0f;
-#pragma unroll
-            for (int j = 0; j < COL_LINES; ++j)
-                atomicAdd(ehist + j * 256 + (product_key(chunk_float<BF16>(ch, j), p.scale_along_line ? rs : col_scale[j]) >> 23), 1u);
-        }
-        __syncthreads();
-        if (warp < nl) window_from_exponents(ehist + warp * 256, fl[warp], win_target(p.k, p.L), lane);
-        __syncthreads();
-        for (int i = tid; i < COL_LINES * HBINS; i += COL_THREADS) hist[i] = 0u;
-        __syncthreads();
-        {   // first pass: elements above a column's window are counted, those inside go to its histogram
-            uint32_t lo[COL_LINES], above[COL_LINES];
+            float rs = 0.0f;
+            if constexpr (ALONG) rs = DASS_LD_G(p.scale + r);
 #pragma unroll
             for (int j = 0; j < COL_LINES; ++j) {
-                lo[j] = j < nl ? fl[j].lo : 0u;      // a column past the matrix edge fills bins nobody reads
-                above[j] = 0u;
+                skey[j] = product_key(chunk_float<BF16>(ch, j), ALONG ? rs : col_scale[j]);
+                // a warp's keys share a few exponents: one update per distinct exponent
+                const uint32_t e = skey[j] >> 23;
+                const uint32_t same = __match_any_sync(FULL_MASK, e);
+                if (lane == __ffs(same) - 1) atomicAdd(ehist + j * 256 + e, (uint32_t)__popc(same));
+            }
+        }
+        __syncthreads();
+        const int target = (int)win_target(p.k, p.L, COL_THREADS);
+        if (warp < nl) window_from_exponents(ehist + warp * 256, fl[warp], (uint32_t)target, lane);
+        __syncthreads();
+#pragma unroll
+        for (int j = 0; j < COL_LINES; ++j) {
+            if (j < nl) {
+                const uint32_t wlo = fl[j].lo, off = skey[j] - wlo;
+                if (off < WIN_SPAN) atomicAdd(fhist + j * FINE_BINS + (off >> FINE_SHIFT), 1u);
+                else if (skey[j] > wlo) atomicAdd(&s_over[j], 1u);
+            }
+        }
+        __syncthreads();
+        if (warp < nl) bracket_from_fine(fhist + warp * FINE_BINS, s_over[warp], fl[warp], target, p.margin, lane);
+        __syncthreads();
+        int sh = 0;                                  // one bin width for the strip: the widest bracket's
+#pragma unroll
+        for (int j = 0; j < COL_LINES; ++j) sh = (j < nl && fl[j].sh > sh) ? fl[j].sh : sh;
+        for (int i = tid; i < COL_LINES * HBINS; i += COL_THREADS) hist[i] = 0u;
+        __syncthreads();
+        if (tid < nl) fl[tid].sh = sh;
+        {   // first pass: the elements inside a column's bracket go to its histogram (predicated: the other lanes cost
+            // the shared-memory pipe nothing), those below it are counted, those above it follow from the length
+            uint32_t lo[COL_LINES], span[COL_LINES], below[COL_LINES];
+#pragma unroll
+            for (int j = 0; j < COL_LINES; ++j) {
+                lo[j] = j < nl ? fl[j].lo : 0u;      // a column past the matrix edge has an empty bracket
+                span[j] = j < nl ? fl[j].hi - fl[j].lo : 0u;
+                below[j] = 0u;
             }
             sweep([&](int j, float wf, float sc_, int64_t) {
-                const uint32_t key = product_key(wf, sc_);
-                const uint32_t off = key - lo[j];
-                if (off < WIN_SPAN) atomicAdd(hist + j * HBINS + (off >> WIN_SHIFT), 1u);
-                else above[j] += key > lo[j] ? 1u : 0u;
+                const uint32_t off = product_key(wf, sc_) - lo[j];        // keys are below 2^31: the top bit says "below lo"
+                asm volatile("{\n\t.reg .pred q;\n\tsetp.lt.u32 q, %0, %1;\n\t@q red.shared.add.u32 [%2], 1;\n\t}"
+                             ::"r"(off), "r"(span[j]), "r"(hist_s + (uint32_t)(j * HBINS * 4) + ((off >> sh) << 2)) : "memory");
+                below[j] += off >> 31;
             });
 #pragma unroll
             for (int j = 0; j < COL_LINES; ++j) {
-                uint32_t a = above[j];
+                uint32_t a = below[j];
 #pragma unroll
                 for (int off = 16; off > 0; off >>= 1) a += __shfl_xor_sync(FULL_MASK, a, off);
-                if (lane == 0 && a && j < nl) atomicAdd(&fl[j].above, a);
+                if (lane == 0 && a && j < nl) atomicAdd(&fl[j].below, a);
             }
         }
         __syncthreads();
-        if (warp < nl) bracket_pick_bin(hist + warp * HBINS, fl[warp], p.k, lane);
+        if (warp < nl) bracket_pick_bin(hist + warp * HBINS, fl[warp], p.k, lane, p.L);
         __syncthreads();
-        {   // second pass: the elements of each column's bin are collected
+        if constexpr (DEFER) {
+            if (tid < nl && fl[tid].ok) {            // published at the bin; nothing set aside yet
+                LineResult r;
+                r.tau32 = fl[tid].bhi; r.exact = LINE_BIN;
+                r.tau64 = (unsigned long long)fl[tid].blo | ((unsigned long long)fl[tid].krem2 << 32);
+                r.cut = (long long)fl[tid].bucket;
+                fl[tid].res = r;
+            }
+        } else {   // second pass: the elements of each column's bin are collected and ranked here
             uint32_t blo[COL_LINES], bw[COL_LINES];
             uint32_t some = 0u;
 #pragma unroll
@@ -1034,7 +1085,10 @@ __global__ void __launch_bounds__(COL_THREADS, 1) select_cols_kernel(const Selec
         if (!sched_next<BF16>(sc, s_long != 0u, p.idx_bits)) break;
         if (was_rounded && s_long && tid < COL_LINES) st[tid].base = 0ull;   // read again only after the next barrier
     }
-    if (tid < nl) DASS_ST(&p.results[c0 + tid], fl[tid].ok ? fl[tid].res : line_result(st[tid], idx_top));
+    if (tid < nl) {
+        DASS_ST(&p.results[c0 + tid], fl[tid].ok ? fl[tid].res : line_result(st[tid], idx_top));
+        if (p.cand_count) DASS_ST(&p.cand_count[c0 + tid], 0u);
+    }
 }
 
 // ---------------------------------------------------------------- column lines: streaming emit
@@ -1183,9 +1237,31 @@ struct EmitStreamParams : UnitGrid {
     uint32_t *mask;      // nullable
     const float *scale;
     const LineResult *results;
+    CandLists cand;
     int64_t ld, wpr;
     int scale_per_row;
 };
+
+// Rare path of the emit pass: the elements of one row of a lane's tile that lie in their column's undecided bin are
+// appended to that column's list (they were written as pruned; the ranking kernel brings the survivors back).
+__device__ __noinline__ void emit_set_aside(uint4 row, uint32_t in_bin, const float *sc8, float row_scale,
+                                            int scale_per_row, long long r, long long c0, CandLists cl)
+{
+    for (int j = 0; j < 8; ++j) {
+        if (!((in_bin >> j) & 1u)) continue;
+        const uint32_t w = wsel(row, j >> 1);
+        const uint32_t raw = (j & 1) ? (w & 0xffff0000u) : (w << 16);
+        const float s = scale_per_row ? row_scale : sc8[j];
+        const uint32_t key = __float_as_uint(fabsf(__uint_as_float(raw)) * s);
+        const uint32_t slot = atomicAdd(cl.count + c0 + j, 1u);
+        if (slot < (uint32_t)CAND_CAP) {
+            const size_t at = (size_t)(c0 + j) * CAND_CAP + slot;
+            DASS_ST(&cl.key[at], key);
+            DASS_ST(&cl.idx[at], (uint32_t)r);
+            DASS_ST(&cl.raw[at], raw);
+        }
+    }
+}
 
 // Keep byte of one row of a lane's tile when some of its columns need the exact rule (rare).
 __device__ __noinline__ uint32_t emit_exact_row(uint4 row, uint32_t keep, uint32_t exact_cols, const LineResult *res8,
@@ -1220,15 +1296,21 @@ select_emit_stream_kernel(const __grid_constant__ CUtensorMap map_w, const EmitS
     const int nvalid = left >= 8 ? 8 : (left > 0 ? (int)left : 0);
     const uint32_t valid = (1u << nvalid) - 1u;
     const bool quad_live = (c0 & ~(int64_t)31) < p.cols;
-    float tau[8], sc[8];
-    uint32_t exact_cols = 0u;
+    float tau[8], tlo[8], sc[8];                     // tlo: start of the column's undecided bin (none: infinity)
+    uint32_t exact_cols = 0u, bin_cols = 0u;
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
         tau[j] = 0.0f;
+        tlo[j] = __uint_as_float(0x7f800000u);
         sc[j] = 0.0f;
         if (j < nvalid) {
             tau[j] = __uint_as_float(DASS_LD(&p.results[c0 + j].tau32));
-            exact_cols |= (DASS_LD(&p.results[c0 + j].exact) ? 1u : 0u) << j;
+            const uint32_t mode = DASS_LD(&p.results[c0 + j].exact);
+            exact_cols |= (mode == 1u ? 1u : 0u) << j;
+            if (mode == LINE_BIN) {
+                bin_cols |= 1u << j;
+                tlo[j] = __uint_as_float((uint32_t)DASS_LD(&p.results[c0 + j].tau64));
+            }
             if (!p.scale_per_row) sc[j] = DASS_LD(&p.scale[c0 + j]);
         }
     }
@@ -1254,19 +1336,30 @@ select_emit_stream_kernel(const __grid_constant__ CUtensorMap map_w, const EmitS
             const int nrows = p.rows - rh >= 4 ? 4 : (int)(p.rows - rh);
             uint4 v[4];
             uint32_t Z[4][4];
+            uint32_t aside[4];                       // per row: lanes below the threshold but not below the bin's start
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
                 v[i] = tile[(4 * h + i) * p.pitch16 + lane];
+                aside[i] = 0u;
 #pragma unroll
                 for (int k = 0; k < 4; ++k) {
                     const uint32_t w = wsel(v[i], k);
                     const float pe = prod_lo(w, p.scale_per_row ? rs[4 * h + i] : sc[2 * k]);
                     const float po = prod_hi(w, p.scale_per_row ? rs[4 * h + i] : sc[2 * k + 1]);
                     Z[i][k] = pruned_lanes(__fsub_rn(pe, tau[2 * k]), __fsub_rn(po, tau[2 * k + 1]));
+                    aside[i] |= Z[i][k] & ~pruned_lanes(__fsub_rn(pe, tlo[2 * k]), __fsub_rn(po, tlo[2 * k + 1])) & (0x00010001u << (2 * k));
                 }
             }
             const uint32_t rows4 = nrows == 4 ? 0xffffffffu : ((1u << (8 * nrows)) - 1u);
             uint32_t keep = ~bytes_of_lanes4(Z[0], Z[1], Z[2], Z[3]) & (valid * 0x01010101u) & rows4;
+            if (aside[0] | aside[1] | aside[2] | aside[3]) {     // elements of undecided bins: set aside for the ranking
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const uint32_t in_bin = (aside[i] | (aside[i] >> 15)) & valid & bin_cols;   // bit j = column j
+                    if (i < nrows && in_bin)
+                        emit_set_aside(v[i], in_bin, sc, rs[4 * h + i], p.scale_per_row, (long long)(rh + i), c0, p.cand);
+                }
+            }
             if (exact_cols) {                        // rounded products equal to a split threshold: the exact rule decides
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
@@ -1301,17 +1394,93 @@ select_emit_stream_kernel(const __grid_constant__ CUtensorMap map_w, const EmitS
     }
 }
 
+// ---------------------------------------------------------------- column lines: the undecided bins
+// One warp per column that the selection left at a bin: the elements the emit pass set aside are ranked by the full
+// key (rounded product, exact product, lower row first), the column's rule is completed, and the survivors are put
+// back into the mask and the pruned copy.
+constexpr int FIX_WARPS = 8;
+struct FixParams {
+    LineResult *results;
+    CandLists cand;
+    const float *scale;
+    uint16_t *Wp;        // nullable
+    uint32_t *mask;      // nullable
+    int64_t cols, ld, wpr;
+    int scale_per_row;
+    int *status;
+};
+
+__global__ void __launch_bounds__(FIX_WARPS * 32) select_fix_cols_kernel(const FixParams p)
+{
+    __shared__ CandSet cand[FIX_WARPS];
+    __shared__ FastLine fl[FIX_WARPS];
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    const int64_t col = (int64_t)blockIdx.x * FIX_WARPS + w;
+    if (col >= p.cols) return;
+    const LineResult r = DASS_LD(&p.results[col]);
+    if (r.exact != LINE_BIN) return;                 // warp-uniform
+    const uint32_t n = DASS_LD(&p.cand.count[col]);
+    const uint32_t bucket = (uint32_t)r.cut;
+    if (n != bucket || n > (uint32_t)CAND_CAP) {     // the two passes disagree: cannot happen, is reported
+        if (lane == 0) atomicMax(p.status, (int)DASS_ERR_INTERNAL);
+        return;
+    }
+    const float col_scale = p.scale_per_row ? 0.0f : DASS_LD(&p.scale[col]);
+    uint32_t raw[(CAND_CAP + 31) / 32];
+#pragma unroll
+    for (int t = 0; t < (CAND_CAP + 31) / 32; ++t) {
+        const int i = t * 32 + lane;
+        raw[t] = 0u;
+        if (i < (int)n) {
+            const size_t at = (size_t)col * CAND_CAP + i;
+            const uint32_t row = DASS_LD(&p.cand.idx[at]);
+            raw[t] = DASS_LD(&p.cand.raw[at]);
+            const float s = p.scale_per_row ? DASS_LD_G(p.scale + row) : col_scale;
+            cand[w].key[i] = DASS_LD(&p.cand.key[at]);
+            cand[w].idx[i] = row;
+            cand[w].k64[i] = exact_key(fabsf(__uint_as_float(raw[t])), s);
+        }
+    }
+    if (lane == 0) { fl[w].ncoll = n; fl[w].bucket = bucket; fl[w].krem2 = (uint32_t)(r.tau64 >> 32); fl[w].ok = 1u; }
+    __syncwarp();
+    bracket_rank(cand[w], fl[w], lane);
+    __syncwarp();
+    if (!fl[w].ok) {
+        if (lane == 0) atomicMax(p.status, (int)DASS_ERR_INTERNAL);
+        return;
+    }
+    const LineResult res = fl[w].res;
+#pragma unroll
+    for (int t = 0; t < (CAND_CAP + 31) / 32; ++t) {
+        const int i = t * 32 + lane;
+        if (i < (int)n) {
+            const uint32_t key = cand[w].key[i], row = cand[w].idx[i];
+            const unsigned long long k64 = cand[w].k64[i];
+            const bool stays = key > res.tau32 ||
+                               (key == res.tau32 && (!res.exact || k64 > res.tau64 || (k64 == res.tau64 && (long long)row <= res.cut)));
+            if (stays) {
+                if (p.mask) atomicOr(p.mask + (int64_t)row * p.wpr + (col >> 5), 1u << (col & 31));
+                if (p.Wp) DASS_ST(p.Wp + (int64_t)row * p.ld + col, (uint16_t)(raw[t] >> 16));
+            }
+        }
+    }
+    if (lane == 0) DASS_ST(&p.results[col], res);    // the column's completed rule
+}
+
 int device_sm_count();   // dass_abi.cu
 cudaError_t unit_grid_setup(UnitGrid &g, CUtensorMap *map, int64_t *grid, const void *W, int64_t rows, int64_t cols, int64_t ld,
                             bool walk_down);   // prune_nm_bf16.cu
 
-static cudaError_t launch_emit_stream(const void *W, void *Wp, uint32_t *mask, const float *scale, const LineResult *results,
-                                      int64_t rows, int64_t cols, int64_t ld, int scale_per_row, cudaStream_t st)
+int *stage_b_status_word();   // prune_nm_bf16.cu
+
+static cudaError_t launch_emit_stream(const void *W, void *Wp, uint32_t *mask, const float *scale, LineResult *results,
+                                      const CandLists &cand, int64_t rows, int64_t cols, int64_t ld, int scale_per_row,
+                                      cudaStream_t st)
 {
     EmitStreamParams p;
     p.W = static_cast<const uint16_t *>(W);
     p.Wp = static_cast<uint16_t *>(Wp);
-    p.mask = mask; p.scale = scale; p.results = results;
+    p.mask = mask; p.scale = scale; p.results = results; p.cand = cand;
     p.ld = ld; p.wpr = (cols + 31) / 32;
     p.scale_per_row = scale_per_row;
     CUtensorMap map;
@@ -1322,6 +1491,15 @@ static cudaError_t launch_emit_stream(const void *W, void *Wp, uint32_t *mask, c
     e = ensure_dynamic_smem(select_emit_stream_kernel, (int)PN_SMEM_BYTES, configured);
     if (e != cudaSuccess) return e;
     select_emit_stream_kernel<<<(unsigned)grid, PN_THREADS, PN_SMEM_BYTES, st>>>(map, p);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    FixParams f;
+    f.results = results; f.cand = cand; f.scale = scale;
+    f.Wp = static_cast<uint16_t *>(Wp); f.mask = mask;
+    f.cols = cols; f.ld = ld; f.wpr = p.wpr;
+    f.scale_per_row = scale_per_row;
+    f.status = p.status;
+    select_fix_cols_kernel<<<(unsigned)((cols + FIX_WARPS - 1) / FIX_WARPS), FIX_WARPS * 32, 0, st>>>(f);
     return cudaGetLastError();
 }
 
@@ -1359,22 +1537,30 @@ static cudaError_t launch_rows(SelectParams p, uint32_t *line_count, uint32_t *l
     return cudaGetLastError();
 }
 
+template <bool BF16, bool ALONG>
+static cudaError_t launch_cols_as(const SelectParams &p, cudaStream_t st)
+{
+    static_assert(COL_THREADS == RS_SAMPLE, "one sample margin serves both line directions");
+    const size_t smem = (size_t)COL_LINES * COL_COPIES * HBINS * sizeof(uint32_t);
+    cudaError_t e = cudaFuncSetAttribute(select_cols_kernel<BF16, ALONG>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    select_cols_kernel<BF16, ALONG><<<(unsigned)((p.cols + COL_LINES - 1) / COL_LINES), COL_THREADS, smem, st>>>(p);
+    return cudaGetLastError();
+}
 template <bool BF16>
 static cudaError_t launch_cols(const SelectParams &p, cudaStream_t st)
 {
-    const size_t smem = (size_t)COL_LINES * COL_COPIES * HBINS * sizeof(uint32_t);
-    cudaError_t e = cudaFuncSetAttribute(select_cols_kernel<BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-    select_cols_kernel<BF16><<<(unsigned)((p.cols + COL_LINES - 1) / COL_LINES), COL_THREADS, smem, st>>>(p);
-    return cudaGetLastError();
+    return p.scale_along_line ? launch_cols_as<BF16, true>(p, st) : launch_cols_as<BF16, false>(p, st);
 }
 
 size_t select_results_bytes(int64_t cols) { return ((size_t)cols * sizeof(LineResult) + 31) / 32 * 32; }
 size_t select_scale_bytes(int64_t n) { return (size_t)((n + 7) / 8 * 8) * sizeof(float); }
 // [per-column results][scale vector padded to 8][count of undecided rows, 32 bytes][their indices]
+// [per column: count of elements set aside][their keys][rows][stored weights]
 size_t select_workspace_bytes(int64_t rows, int64_t cols, bool norm_cols)
 {
-    return select_results_bytes(cols) + select_scale_bytes(norm_cols ? cols : rows) + 32 + (size_t)rows * sizeof(uint32_t);
+    return select_results_bytes(cols) + select_scale_bytes(norm_cols ? cols : rows) + 32 + (size_t)((rows + 7) / 8 * 8) * sizeof(uint32_t) +
+           (size_t)((cols + 7) / 8 * 8) * sizeof(uint32_t) * (1 + 3 * CAND_CAP);
 }
 
 cudaError_t select_unstructured_launch(const void *W, int64_t rows, int64_t cols, int64_t ld, bool bf16,
@@ -1386,6 +1572,12 @@ cudaError_t select_unstructured_launch(const void *W, int64_t rows, int64_t cols
     const int64_t n_norm = norm_cols ? cols : rows;
     uint32_t *line_count = reinterpret_cast<uint32_t *>(reinterpret_cast<unsigned char *>(scale_ws) + select_scale_bytes(n_norm));
     uint32_t *line_list = line_count + 8;
+    const size_t cols8 = (size_t)((cols + 7) / 8 * 8);
+    CandLists cand;
+    cand.count = line_list + (rows + 7) / 8 * 8;
+    cand.key = cand.count + cols8;
+    cand.idx = cand.key + cols8 * CAND_CAP;
+    cand.raw = cand.idx + cols8 * CAND_CAP;
     const int64_t n_pad = (n_norm + 7) / 8 * 8;
     scale_vector_kernel<<<(unsigned)((n_pad + 255) / 256), 256, 0, st>>>(norm, n_norm, n_pad, (int)scale_mode_for(alpha), alpha, scale_ws);
     cudaError_t e = cudaGetLastError();
@@ -1393,6 +1585,7 @@ cudaError_t select_unstructured_launch(const void *W, int64_t rows, int64_t cols
     SelectParams p;
     p.W = W; p.Wp = W_pruned; p.mask = mask_bits; p.scale = scale_ws; p.results = results;
     p.line_count = nullptr; p.line_list = nullptr;
+    p.cand_count = (!line_is_row && bf16) ? cand.count : nullptr;
     p.rows = rows; p.cols = cols; p.ld = ld;
     p.wpr = (cols + 31) / 32;
     p.L = line_is_row ? cols : rows;
@@ -1424,7 +1617,7 @@ cudaError_t select_unstructured_launch(const void *W, int64_t rows, int64_t cols
     const int64_t cap = (int64_t)device_sm_count() * 8;
     const int grid = (int)(want < cap ? want : cap);
     if (bf16)   // the TMA-fed streaming pass
-        return launch_emit_stream(W, W_pruned, mask_bits, scale_ws, results, rows, cols, ld, norm_cols ? 0 : 1, st);
+        return launch_emit_stream(W, W_pruned, mask_bits, scale_ws, results, cand, rows, cols, ld, norm_cols ? 0 : 1, st);
     select_emit_cols_kernel<false><<<grid, 256, 0, st>>>(q);
     return cudaGetLastError();
 }
@@ -1459,15 +1652,15 @@ extern "C" dass_status dass_select_unstructured(const void *W, int64_t rows, int
     if (ld % (bf16 ? 8 : 4) != 0) return DASS_ERR_ALIGN;
     if ((reinterpret_cast<uintptr_t>(W) & 15u) || (W_pruned && (reinterpret_cast<uintptr_t>(W_pruned) & 15u)) ||
         (reinterpret_cast<uintptr_t>(norm) & 3u) || (reinterpret_cast<uintptr_t>(mask_bits) & 3u)) return DASS_ERR_ALIGN;
+    const bool line_is_row = compare_axis == DASS_AXIS_COLS;         // the index that varies inside a line
+    const int64_t L = line_is_row ? cols : rows;
+    if (L >= (int64_t)1 << 31) return DASS_ERR_UNSUPPORTED;
+    if (line_is_row && select_row_smem_bytes(L, bf16) > (size_t)220 * 1024) return DASS_ERR_UNSUPPORTED;   // a row line is cached in shared memory
     size_t need = 0;
     const dass_status qs = dass_select_workspace_bytes(rows, cols, norm_axis, &need);
     if (qs != DASS_OK) return qs;
     if (!workspace || workspace_bytes < need) return DASS_ERR_WORKSPACE;
     if (reinterpret_cast<uintptr_t>(workspace) & 15u) return DASS_ERR_ALIGN;
-    const bool line_is_row = compare_axis == DASS_AXIS_COLS;         // the index that varies inside a line
-    const int64_t L = line_is_row ? cols : rows;
-    if (L >= (int64_t)1 << 31) return DASS_ERR_UNSUPPORTED;
-    if (line_is_row && select_row_smem_bytes(L, bf16) > (size_t)220 * 1024) return DASS_ERR_UNSUPPORTED;   // a row line is cached in shared memory
     const int64_t n_prune = (int64_t)std::floor(sparsity * (double)L);
     const uint32_t k = (uint32_t)(L - n_prune);
     DASS_BOUNDS_SCOPE(bs);
