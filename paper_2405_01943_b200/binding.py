@@ -349,7 +349,8 @@ def prune_nm(W: torch.Tensor, norm: torch.Tensor, norm_axis: int, alpha: float, 
 
 
 def prune_status(stream: Optional[torch.cuda.Stream] = None) -> None:
-    """Waits for the stream and raises if a bounded wait inside a prune_nm kernel ran out since the last query."""
+    """Waits for the stream and raises if, since the last query, a bounded wait inside a prune_nm or
+    select_unstructured kernel ran out or the passes of a select_unstructured call disagreed."""
     _check(load().dass_prune_status(_stream(stream)), "dass_prune_status")
 
 

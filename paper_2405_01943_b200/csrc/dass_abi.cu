@@ -111,6 +111,7 @@ const char *dass_status_string(dass_status s)
     case DASS_ERR_WORKSPACE: return "workspace too small";
     case DASS_ERR_CUDA: return "CUDA error";
     case DASS_ERR_TIMEOUT: return "device-side wait timed out";
+    case DASS_ERR_INTERNAL: return "passes of a kernel chain disagree";
     }
     return "unknown status";
 }
@@ -261,7 +262,7 @@ dass_status dass_prune_status(void *cuda_stream)
 {
     int value = 0;
     if (prune_status_read(&value, static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) return DASS_ERR_CUDA;
-    return value == 0 ? DASS_OK : DASS_ERR_TIMEOUT;
+    return value == DASS_ERR_INTERNAL ? DASS_ERR_INTERNAL : (value == 0 ? DASS_OK : DASS_ERR_TIMEOUT);
 }
 
 dass_status dass_compress_nm(const void *W, const uint32_t *mask_bits,

@@ -250,7 +250,7 @@ struct UnitRing {
     // After a failed wait: record it and give the copies still in flight one more bounded chance to land.
     __device__ __forceinline__ void fail(int lane, int *status)
     {
-        if (lane == 0 && status) atomicExch(status, (int)DASS_ERR_TIMEOUT);
+        if (lane == 0 && status) atomicMax(status, (int)DASS_ERR_TIMEOUT);
 #pragma unroll
         for (int s = 0; s < PN_STAGES; ++s) {
             slot_wait(bars + 8u * s, 0u);

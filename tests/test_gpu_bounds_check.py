@@ -81,13 +81,14 @@ def test_stage_b_entry_points(check_lib, dtype, axis):
 
 @pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32], ids=["bf16", "f32"])
 def test_unstructured_selection_and_feature_norms(check_lib, dtype):
-    for rows, cols in ((72, 344), (2104, 264), (40, 2600)):       # short lines, long column lines (sampled bracket), long row lines
+    for rows, cols in ((72, 344), (4104, 264), (40, 4200)):       # short lines, long column lines and long row lines (streaming kernels)
         W = _rand((rows, cols), dtype)
         for axis in (AXIS_ROWS, AXIS_COLS):
             norm = (torch.rand(rows if axis == AXIS_ROWS else cols, device=DEV) * 10 + 0.1).float()
             for sparsity in (0.5, 0.0, 0.73):
                 binding.select_unstructured(W, norm, axis, 0.5, sparsity, axis)
             binding.select_unstructured(W, norm, axis, 0.0, 0.5, axis)          # ties everywhere
+            binding.prune_status()
             _clean()
     X = _rand((1030, 200), dtype, 1.0)
     binding.feature_sumsq(X)

@@ -59,6 +59,92 @@ def test_small_shapes_bit_exact(dtype, norm_axis, compare_axis, ties):
             _check(W, norm, norm_axis, alpha, s, compare_axis)
 
 
+# ---------------------------------------------------------------- lines long enough for the streaming kernels
+# (4096 elements and more: sampled bracket, one histogram sweep, the cut's bin ranked at the end; lines those
+# kernels cannot decide go to the radix select)
+def _long_case(kind, rows, cols, dtype, gen, line_axis):
+    """A matrix whose comparison lines run along `line_axis` (0: columns are the lines, 1: rows are)."""
+    L = rows if line_axis == 0 else cols
+    n_lines = cols if line_axis == 0 else rows
+    w = torch.randn((rows, cols), generator=gen, device=DEV) * 0.02
+    lines = torch.arange(n_lines, device=DEV)
+    along = torch.arange(L, device=DEV)
+
+    def put(sel_lines, values):                      # values: [L, len(sel_lines)] along the line
+        if line_axis == 0:
+            w[:, sel_lines] = values
+        else:
+            w[sel_lines, :] = values.t()
+
+    if kind == "ties":                               # a handful of magnitudes: the cut's bin overflows everywhere
+        vals = torch.tensor([0.0, -0.0, 0.25, -0.25, 0.5, 1.0, -1.0, 2.0], device=DEV)
+        w = vals[torch.randint(0, len(vals), (rows, cols), generator=gen, device=DEV)]
+    elif kind == "mixed":                            # every third line tied, the others random
+        sel = lines[::3]
+        vals = torch.tensor([0.125, -0.125, 0.5, 3.0], device=DEV)
+        put(sel, vals[torch.randint(0, len(vals), (L, len(sel)), generator=gen, device=DEV)])
+    elif kind == "zeros":                            # two thirds of every other line are zero: the cut sits at zero
+        sel = lines[::2]
+        v = torch.randn((L, len(sel)), generator=gen, device=DEV) * 0.02
+        v[torch.rand((L, len(sel)), generator=gen, device=DEV) < 0.66] = 0.0
+        put(sel, v)
+    elif kind == "outliers":                         # a few huge and a few tiny magnitudes in every line
+        big = torch.randint(0, L, (16,), generator=gen, device=DEV)
+        tiny = torch.randint(0, L, (64,), generator=gen, device=DEV)
+        if line_axis == 0:
+            w[big, :] *= 1e6
+            w[tiny, :] *= 1e-12
+        else:
+            w[:, big] *= 1e6
+            w[:, tiny] *= 1e-12
+    elif kind == "spread":                           # magnitudes over 24 octaves: the window must follow the quantile
+        e = torch.randint(-12, 12, (rows, cols), generator=gen, device=DEV).float()
+        w = w * torch.exp2(e)
+    ld = (cols + 7) // 8 * 8
+    base = torch.full((rows, ld), 7.0, dtype=dtype, device=DEV)
+    base[:, :cols] = w.to(dtype)
+    return base[:, :cols]
+
+
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32], ids=["bf16", "f32"])
+@pytest.mark.parametrize("line_axis", [0, 1], ids=["column-lines", "row-lines"])
+@pytest.mark.parametrize("kind", ["random", "ties", "mixed", "zeros", "outliers", "spread"])
+def test_long_lines_bit_exact(dtype, line_axis, kind):
+    gen = torch.Generator(device=DEV)
+    gen.manual_seed(101 + 7 * line_axis + len(kind))
+    compare_axis = AXIS_ROWS if line_axis == 0 else AXIS_COLS
+    # ragged everywhere: 4099 / 4233 elements per line, 27 / 21 lines (not multiples of 8 or 32)
+    rows, cols = (4099, 27) if line_axis == 0 else (21, 4233)
+    for norm_axis in (AXIS_ROWS, AXIS_COLS):         # the scale varies along the line, or is one number per line
+        for s, alpha in [(0.5, 0.5), (0.07, 1.0), (0.97, 1.0), (0.0, 0.5), (0.5, 0.0)]:
+            W = _long_case(kind, rows, cols, dtype, gen, line_axis)
+            norm = _norm(rows if norm_axis == AXIS_ROWS else cols, gen, ties=(kind == "ties"))
+            _check(W, norm, norm_axis, alpha, s, compare_axis)
+    binding.prune_status()                           # raises if a bounded wait ran out or the passes disagreed
+
+
+@pytest.mark.parametrize("line_axis", [0, 1], ids=["column-lines", "row-lines"])
+def test_long_lines_in_place(line_axis):
+    """W_pruned may be W itself: the streaming passes read every element before they overwrite it, and the elements
+    of the cut's bin are put back from what was set aside."""
+    gen = torch.Generator(device=DEV)
+    gen.manual_seed(55 + line_axis)
+    compare_axis = AXIS_ROWS if line_axis == 0 else AXIS_COLS
+    rows, cols = (8200, 40) if line_axis == 0 else (24, 8200)
+    norm_axis = compare_axis
+    for kind in ("random", "mixed"):
+        W = _long_case(kind, rows, cols, torch.bfloat16, gen, line_axis)
+        norm = _norm(rows if norm_axis == AXIS_ROWS else cols, gen)
+        Wn = to_np32(W)
+        want = oracle.select_unstructured(Wn, to_np32(norm), norm_axis, 1.0, 0.5, compare_axis)
+        mask_bits, pruned = binding.select_unstructured(W, norm, norm_axis, 1.0, 0.5, compare_axis, W_pruned=W)
+        torch.cuda.synchronize()
+        assert pruned.data_ptr() == W.data_ptr()
+        assert np.array_equal(u32(mask_bits), oracle.pack_mask(want))
+        assert np.array_equal(bits_of(W), bits_like(np.where(want == 1, Wn, np.float32(0.0)), W.dtype))
+    binding.prune_status()
+
+
 def test_tiny_config_input_and_output_balanced():
     cfg = synth.CONFIGS["tiny"]
     Wg, Wu, Wd = synth.make_weights(cfg, DEV)
