@@ -18,12 +18,22 @@
 // kernel publishes (tau32, exact, tau64, cut) per column and select_emit_cols_kernel applies them in a streaming
 // pass with coalesced rows.
 #include <cmath>
+#include <cstring>
 #include <type_traits>
 
 #include "stream_units.cuh"
 
 namespace dass {
 
+// f(integral_constant<int, 0>) ... f(integral_constant<int, N - 1>)
+template <int N, typename F>
+__device__ __forceinline__ void static_for(F &&f)
+{
+    if constexpr (N > 0) {
+        static_for<N - 1>(f);
+        f(std::integral_constant<int, N - 1>{});
+    }
+}
 
 // What the selection found for one line; enough to decide every element of the line locally:
 // keep iff p > tau32, or p == tau32 and (not exact, or k64 > tau64, or k64 == tau64 and index <= cut).
@@ -62,6 +72,7 @@ struct SelectParams {
     uint32_t *line_count;   // row lines: how many lines the streaming kernel left undecided, and which
     uint32_t *line_list;    // (both null: the radix kernel takes every row)
     uint32_t *cand_count;   // column lines, bf16: per-column count of the elements the emit pass sets aside (cleared here)
+    int *status;            // device status word for bounded waits that ran out
 };
 
 // out[i] = fl32(norm[i]^alpha) for i < n, 0 for the padding up to npad (a multiple of 8, so that the selection
@@ -835,14 +846,26 @@ __global__ void __launch_bounds__(RS_THREADS, 4) select_rows_stream_kernel(const
 // every pass reads it again with one vector load per row and thread, and one CTA per SM keeps the strips in
 // flight (148 x 0.46 MB on the 70B-shaped matrix) inside L2, so only the first pass reads DRAM.  The kernel
 // publishes (tau32, exact, tau64, cut) per column; select_emit_cols_kernel applies them with coalesced rows.
-constexpr int COL_THREADS = 1024;
+constexpr int COL_THREADS = 512;                // two CTAs per SM: one sweeps while the other samples, picks its bins or waits
+constexpr int COL_SAMPLE = 1024;                // evenly spaced rows of a strip that place its columns' brackets
 constexpr int COL_LINES = 8;
 constexpr int COL_COPIES = 1;                   // histogram copies per column (3 measured slower, as for rows)
 
 // ALONG: the scale varies along the columns (one per row) rather than being one number per column.
-template <bool BF16, bool ALONG>
-__global__ void __launch_bounds__(COL_THREADS, 1) select_cols_kernel(const SelectParams p)
+// TMA (bf16, at least 8 columns): the sweep of the sampled bracket receives the strip through bulk tensor copies --
+// SR_STAGE_ROWS rows of 16 bytes per stage, one stage in flight while the other is worked on -- instead of one 16-byte load per thread from 1024
+// different cache lines per warp instruction pair, which kept the load/store pipe busier than the arithmetic.
+constexpr int HSTRIDE = HBINS + 32;                      // a column's bins of the bracket sweep, then one idle word per lane
+constexpr int SR_STAGES = 2;
+constexpr int SR_BOX_ROWS = 256;                         // rows of one bulk copy (a box dimension is at most 256)
+constexpr int SR_STAGE_ROWS = 1024;                      // rows of one stage: SR_RPT per thread
+constexpr int SR_RPT = SR_STAGE_ROWS / COL_THREADS;
+constexpr uint32_t SR_STAGE_BYTES = SR_STAGE_ROWS * 16u;
+
+template <bool BF16, bool ALONG, bool TMA>
+__global__ void __launch_bounds__(COL_THREADS, 2) select_cols_kernel(const __grid_constant__ CUtensorMap map_w, const SelectParams p)
 {
+    static_assert(!TMA || BF16, "the bulk-copy sweep is written for bf16 strips");
     using elem_t = typename std::conditional<BF16, uint16_t, uint32_t>::type;
     extern __shared__ __align__(16) unsigned char u_smem[];
     uint32_t *hist = reinterpret_cast<uint32_t *>(u_smem);       // [COL_LINES][COL_COPIES][HBINS]
@@ -911,9 +934,30 @@ __global__ void __launch_bounds__(COL_THREADS, 1) select_cols_kernel(const Selec
     __shared__ CandSet cand[DEFER ? 1 : COL_LINES];
     __shared__ uint32_t s_over[COL_LINES];           // sample keys above a column's window
     bool any_pending = true;
-    if (tid < COL_LINES) fl[tid].ok = 0u;
+    if (tid < COL_LINES) { fl[tid].ok = 0u; fl[tid].lo = 0u; fl[tid].hi = 0u; }     // past the matrix edge: an empty bracket
     if (p.L >= FAST_MIN_L) {                         // the same for every thread
         const uint32_t hist_s = smem_u32(hist);
+        // the ring of the bulk-copy sweep, behind the histograms (128-byte aligned), and its barriers
+        uint8_t *ring_mem = u_smem + (size_t)COL_LINES * HSTRIDE * sizeof(uint32_t);
+        ring_mem += (128u - (smem_u32(ring_mem) & 127u)) & 127u;
+        const uint32_t ring_s = smem_u32(ring_mem), bars_s = ring_s + SR_STAGES * SR_STAGE_BYTES;
+        const int n_it = (int)((p.L + SR_STAGE_ROWS - 1) / SR_STAGE_ROWS);
+        auto ring_issue = [&](int it) {              // one thread: the rows from it * SR_STAGE_ROWS into stage it % SR_STAGES
+            const uint32_t bar = bars_s + 8u * (uint32_t)(it % SR_STAGES);
+            const uint32_t dst = ring_s + (uint32_t)(it % SR_STAGES) * SR_STAGE_BYTES;
+            mbar_arrive_expect_tx(bar, SR_STAGE_BYTES);
+#pragma unroll
+            for (int b = 0; b < SR_STAGE_ROWS / SR_BOX_ROWS; ++b)
+                tma_load_2d(dst + (uint32_t)(b * SR_BOX_ROWS * 16), &map_w, bar, (int)c0, it * SR_STAGE_ROWS + b * SR_BOX_ROWS);
+        };
+        if constexpr (TMA) {                         // the first stages travel while the sample is taken
+            if (tid == 0) {
+#pragma unroll
+                for (int s_ = 0; s_ < SR_STAGES; ++s_) mbar_init(bars_s + 8u * s_, 1);
+                asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+                for (int it = 0; it < SR_STAGES - 1 && it < n_it; ++it) ring_issue(it);
+            }
+        }
         // loads one row of the strip (the vector loads of count_pass)
         auto load_row = [&](int64_t r, Chunk<BF16> &ch) {
             const uint4 *src = reinterpret_cast<const uint4 *>(strip + r * p.ld);
@@ -958,41 +1002,51 @@ __global__ void __launch_bounds__(COL_THREADS, 1) select_cols_kernel(const Selec
         for (int i = tid; i < COL_LINES * (256 + FINE_BINS); i += COL_THREADS) hist[i] = 0u;
         if (tid < COL_LINES) s_over[tid] = 0u;
         __syncthreads();
-        uint32_t skey[COL_LINES];                    // the sample: one row per thread, all of the strip's columns
-        {
-            const int64_t r = ((int64_t)tid * p.L) / COL_THREADS;
+        constexpr int SPT = COL_SAMPLE / COL_THREADS;
+        uint32_t skey[SPT][COL_LINES];               // the sample: SPT rows per thread, all of the strip's columns
+#pragma unroll
+        for (int u = 0; u < SPT; ++u) {
+            const int64_t r = ((int64_t)(tid + u * COL_THREADS) * p.L) / COL_SAMPLE;
             Chunk<BF16> ch;
             load_row(r, ch);
             float rs = 0.0f;
             if constexpr (ALONG) rs = DASS_LD_G(p.scale + r);
 #pragma unroll
+            for (int j = 0; j < COL_LINES; ++j) skey[u][j] = product_key(chunk_float<BF16>(ch, j), ALONG ? rs : col_scale[j]);
+        }
+#pragma unroll
+        for (int u = 0; u < SPT; ++u) {
+#pragma unroll
             for (int j = 0; j < COL_LINES; ++j) {
-                skey[j] = product_key(chunk_float<BF16>(ch, j), ALONG ? rs : col_scale[j]);
                 // a warp's keys share a few exponents: one update per distinct exponent
-                const uint32_t e = skey[j] >> 23;
+                const uint32_t e = skey[u][j] >> 23;
                 const uint32_t same = __match_any_sync(FULL_MASK, e);
                 if (lane == __ffs(same) - 1) atomicAdd(ehist + j * 256 + e, (uint32_t)__popc(same));
             }
         }
         __syncthreads();
-        const int target = (int)win_target(p.k, p.L, COL_THREADS);
+        const int target = (int)win_target(p.k, p.L, COL_SAMPLE);
         if (warp < nl) window_from_exponents(ehist + warp * 256, fl[warp], (uint32_t)target, lane);
         __syncthreads();
 #pragma unroll
-        for (int j = 0; j < COL_LINES; ++j) {
-            if (j < nl) {
-                const uint32_t wlo = fl[j].lo, off = skey[j] - wlo;
-                if (off < WIN_SPAN) atomicAdd(fhist + j * FINE_BINS + (off >> FINE_SHIFT), 1u);
-                else if (skey[j] > wlo) atomicAdd(&s_over[j], 1u);
+        for (int u = 0; u < SPT; ++u) {
+#pragma unroll
+            for (int j = 0; j < COL_LINES; ++j) {
+                if (j < nl) {
+                    const uint32_t wlo = fl[j].lo, off = skey[u][j] - wlo;
+                    if (off < WIN_SPAN) atomicAdd(fhist + j * FINE_BINS + (off >> FINE_SHIFT), 1u);
+                    else if (skey[u][j] > wlo) atomicAdd(&s_over[j], 1u);
+                }
             }
         }
         __syncthreads();
         if (warp < nl) bracket_from_fine(fhist + warp * FINE_BINS, s_over[warp], fl[warp], target, p.margin, lane);
         __syncthreads();
+        bool lost = false;                           // a bounded wait of the bulk-copy sweep ran out
         int sh = 0;                                  // one bin width for the strip: the widest bracket's
 #pragma unroll
         for (int j = 0; j < COL_LINES; ++j) sh = (j < nl && fl[j].sh > sh) ? fl[j].sh : sh;
-        for (int i = tid; i < COL_LINES * HBINS; i += COL_THREADS) hist[i] = 0u;
+        for (int i = tid; i < COL_LINES * HSTRIDE; i += COL_THREADS) hist[i] = 0u;
         __syncthreads();
         if (tid < nl) fl[tid].sh = sh;
         {   // first pass: the elements inside a column's bracket go to its histogram (predicated: the other lanes cost
@@ -1000,16 +1054,64 @@ __global__ void __launch_bounds__(COL_THREADS, 1) select_cols_kernel(const Selec
             uint32_t lo[COL_LINES], span[COL_LINES], below[COL_LINES];
 #pragma unroll
             for (int j = 0; j < COL_LINES; ++j) {
-                lo[j] = j < nl ? fl[j].lo : 0u;      // a column past the matrix edge has an empty bracket
-                span[j] = j < nl ? fl[j].hi - fl[j].lo : 0u;
+                lo[j] = fl[j].lo;                    // (a column past the matrix edge has an empty bracket)
+                span[j] = fl[j].hi - fl[j].lo;
                 below[j] = 0u;
             }
-            sweep([&](int j, float wf, float sc_, int64_t) {
-                const uint32_t off = product_key(wf, sc_) - lo[j];        // keys are below 2^31: the top bit says "below lo"
-                asm volatile("{\n\t.reg .pred q;\n\tsetp.lt.u32 q, %0, %1;\n\t@q red.shared.add.u32 [%2], 1;\n\t}"
-                             ::"r"(off), "r"(span[j]), "r"(hist_s + (uint32_t)(j * HBINS * 4) + ((off >> sh) << 2)) : "memory");
+            // every lane updates a counter: its element's bin inside the bracket, else a word of its own behind the column's
+            // bins that nobody reads
+            const uint32_t idle_rel = (uint32_t)(HBINS + lane) * 4u;
+            auto count_key = [&](auto jc, uint32_t key) {                 // jc: the column, a compile-time constant
+                constexpr int J = decltype(jc)::value;
+                const uint32_t off = key - lo[J];                         // keys are below 2^31: the top bit says "below lo"
+                const uint32_t rel = off < span[J] ? (off >> sh) << 2 : idle_rel;
+                asm volatile("red.shared.add.u32 [%0+%1], 1;" ::"r"(hist_s + rel), "n"(J * HSTRIDE * 4) : "memory");
+                below[J] += off >> 31;
+            };
+            auto visit = [&](int j, float wf, float sc_, int64_t) {
+                const uint32_t off = product_key(wf, sc_) - lo[j];
+                const uint32_t rel = off < span[j] ? (off >> sh) << 2 : idle_rel;
+                asm volatile("red.shared.add.u32 [%0], 1;" ::"r"(hist_s + (uint32_t)(j * HSTRIDE * 4) + rel) : "memory");
                 below[j] += off >> 31;
-            });
+            };
+            if constexpr (TMA) {
+                for (int it = 0; it < n_it; ++it) {
+                    // the stage read one iteration ago is free (every thread passed that iteration's barrier)
+                    if (tid == 0 && it + SR_STAGES - 1 < n_it) ring_issue(it + SR_STAGES - 1);
+                    const int64_t r0 = (int64_t)it * SR_STAGE_ROWS + tid;
+                    float rs[SR_RPT];
+#pragma unroll
+                    for (int u = 0; u < SR_RPT; ++u) {
+                        rs[u] = 0.0f;
+                        if constexpr (ALONG) rs[u] = r0 + u * COL_THREADS < p.L ? DASS_LD_G(p.scale + r0 + u * COL_THREADS) : 0.0f;
+                    }
+                    const bool ok = slot_wait(bars_s + 8u * (uint32_t)(it % SR_STAGES), (uint32_t)((it / SR_STAGES) & 1));
+                    uint4 v[SR_RPT];
+#pragma unroll
+                    for (int u = 0; u < SR_RPT; ++u)
+                        v[u] = *reinterpret_cast<const uint4 *>(ring_mem + (size_t)(it % SR_STAGES) * SR_STAGE_BYTES + (size_t)(u * COL_THREADS + tid) * 16);
+                    if (__syncthreads_or(ok ? 0 : 1)) { lost = true; break; }
+#pragma unroll
+                    for (int u = 0; u < SR_RPT; ++u) {
+                        if (r0 + u * COL_THREADS < p.L) {    // rows past the end arrive as zeros and are not counted
+                            const uint32_t a[4] = {v[u].x & 0x7fff7fffu, v[u].y & 0x7fff7fffu, v[u].z & 0x7fff7fffu, v[u].w & 0x7fff7fffu};   // |w|, in pairs
+                            static_for<COL_LINES>([&](auto jc) {
+                                constexpr int J = decltype(jc)::value;
+                                const float wa = __uint_as_float((J & 1) ? (a[J >> 1] & 0xffff0000u) : (a[J >> 1] << 16));
+                                count_key(jc, __float_as_uint(__fmul_rn(wa, ALONG ? rs[u] : col_scale[J])));
+                            });
+                        }
+                    }
+                }
+                if (lost) {                          // recorded; the copies in flight get one more bounded chance to land,
+                    if (tid == 0) {                  // and the radix select (plain loads) decides the strip
+                        if (p.status) atomicMax(p.status, (int)DASS_ERR_TIMEOUT);
+                        for (int s_ = 0; s_ < SR_STAGES; ++s_) { slot_wait(bars_s + 8u * s_, 0u); slot_wait(bars_s + 8u * s_, 1u); }
+                    }
+                }
+            } else {
+                sweep(visit);
+            }
 #pragma unroll
             for (int j = 0; j < COL_LINES; ++j) {
                 uint32_t a = below[j];
@@ -1019,8 +1121,12 @@ __global__ void __launch_bounds__(COL_THREADS, 1) select_cols_kernel(const Selec
             }
         }
         __syncthreads();
-        if (warp < nl) bracket_pick_bin(hist + warp * HBINS, fl[warp], p.k, lane, p.L);
+        if (warp < nl) bracket_pick_bin(hist + warp * HSTRIDE, fl[warp], p.k, lane, p.L);
         __syncthreads();
+        if (lost) {                                  // the same for every thread: the counts are incomplete
+            if (tid < nl) fl[tid].ok = 0u;
+            __syncthreads();
+        }
         if constexpr (DEFER) {
             if (tid < nl && fl[tid].ok) {            // published at the bin; nothing set aside yet
                 LineResult r;
@@ -1537,20 +1643,34 @@ static cudaError_t launch_rows(SelectParams p, uint32_t *line_count, uint32_t *l
     return cudaGetLastError();
 }
 
-template <bool BF16, bool ALONG>
+bool tile_map_bf16(CUtensorMap *map, const void *ptr, int64_t rows, int64_t cols, int64_t ld, int box_cols, int box_rows);   // calib_tc.cu
+
+template <bool BF16, bool ALONG, bool TMA>
 static cudaError_t launch_cols_as(const SelectParams &p, cudaStream_t st)
 {
-    static_assert(COL_THREADS == RS_SAMPLE, "one sample margin serves both line directions");
-    const size_t smem = (size_t)COL_LINES * COL_COPIES * HBINS * sizeof(uint32_t);
-    cudaError_t e = cudaFuncSetAttribute(select_cols_kernel<BF16, ALONG>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    static_assert(COL_SAMPLE == RS_SAMPLE, "one sample margin serves both line directions");
+    CUtensorMap map;
+    memset(&map, 0, sizeof(map));
+    static_assert(COL_COPIES == 1, "the bracket sweep lays its histograms out with stride HSTRIDE");
+    size_t smem = (size_t)COL_LINES * HSTRIDE * sizeof(uint32_t);
+    if (TMA) {
+        if (!tile_map_bf16(&map, p.W, p.rows, p.cols, p.ld, COL_LINES, SR_BOX_ROWS)) return cudaErrorInvalidValue;
+        smem += 128 + SR_STAGES * SR_STAGE_BYTES + SR_STAGES * 8;
+    }
+    cudaError_t e = cudaFuncSetAttribute(select_cols_kernel<BF16, ALONG, TMA>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    select_cols_kernel<BF16, ALONG><<<(unsigned)((p.cols + COL_LINES - 1) / COL_LINES), COL_THREADS, smem, st>>>(p);
+    select_cols_kernel<BF16, ALONG, TMA><<<(unsigned)((p.cols + COL_LINES - 1) / COL_LINES), COL_THREADS, smem, st>>>(map, p);
     return cudaGetLastError();
 }
 template <bool BF16>
 static cudaError_t launch_cols(const SelectParams &p, cudaStream_t st)
 {
-    return p.scale_along_line ? launch_cols_as<BF16, true>(p, st) : launch_cols_as<BF16, false>(p, st);
+    // bulk copies need whole boxes of 8 columns x 256 rows inside the matrix, and the sweep they feed runs on long lines only
+    const bool tma = BF16 && p.cols >= COL_LINES && p.L >= FAST_MIN_L && p.rows < 0x7fffffffll - SR_STAGE_ROWS;
+    if constexpr (BF16) {
+        if (tma) return p.scale_along_line ? launch_cols_as<true, true, true>(p, st) : launch_cols_as<true, false, true>(p, st);
+    }
+    return p.scale_along_line ? launch_cols_as<BF16, true, false>(p, st) : launch_cols_as<BF16, false, false>(p, st);
 }
 
 size_t select_results_bytes(int64_t cols) { return ((size_t)cols * sizeof(LineResult) + 31) / 32 * 32; }
@@ -1586,6 +1706,7 @@ cudaError_t select_unstructured_launch(const void *W, int64_t rows, int64_t cols
     p.W = W; p.Wp = W_pruned; p.mask = mask_bits; p.scale = scale_ws; p.results = results;
     p.line_count = nullptr; p.line_list = nullptr;
     p.cand_count = (!line_is_row && bf16) ? cand.count : nullptr;
+    p.status = stage_b_status_word();
     p.rows = rows; p.cols = cols; p.ld = ld;
     p.wpr = (cols + 31) / 32;
     p.L = line_is_row ? cols : rows;
