@@ -412,6 +412,7 @@ __device__ __forceinline__ void bracket_from_fine(const uint32_t *fh, uint32_t n
         const uint32_t span = f.hi - f.lo - 1u;       // largest offset inside the bracket
         const int bits = 32 - __clz(span);
         f.sh = bits > HB ? bits - HB : 0;
+        f.hi = f.lo + ((uint32_t)HBINS << f.sh);      // widened to the whole histogram: "inside" is "bin below HBINS"
     }
 }
 
@@ -640,7 +641,7 @@ template <bool BF16, bool ALONG>
 __global__ void __launch_bounds__(RS_THREADS, 4) select_rows_stream_kernel(const SelectParams p)
 {
     using elem_t = typename std::conditional<BF16, uint16_t, uint32_t>::type;
-    __shared__ uint32_t hist[HBINS];
+    __shared__ uint32_t hist[HBINS + 32];            // the bins, then one idle word per lane
     __shared__ uint32_t s_over;                      // sample keys above the window
     __shared__ FastLine fl;
     __shared__ CandSet cand;
@@ -738,9 +739,10 @@ __global__ void __launch_bounds__(RS_THREADS, 4) select_rows_stream_kernel(const
     __syncthreads();
 
     // ---------------------------------------------------------------- first pass: histogram of the bracket
-    {   // only the elements inside the bracket touch the histogram (a predicated reduction: the other lanes cost
-        // the shared-memory pipe nothing); those below it are counted, those above it follow from the line's length
-        const uint32_t lo = fl.lo, span = fl.hi - fl.lo;
+    {   // every lane updates a counter: its element's bin inside the bracket (which spans all HBINS bins), else a word of
+        // its own behind the bins that nobody reads; the elements below the bracket are counted, those above it follow
+        // from the line's length
+        const uint32_t lo = fl.lo, idle_bin = (uint32_t)(HBINS + lane);
         const int sh = fl.sh;
         uint32_t below = 0u;
         sweep([&](int64_t, const Chunk<BF16> &ch, const float (&sc)[8], int nvalid) {
@@ -750,9 +752,8 @@ __global__ void __launch_bounds__(RS_THREADS, 4) select_rows_stream_kernel(const
             for (int j = 0; j < 8; ++j) {
                 if (j < nvalid) {
                     const uint32_t off = key[j] - lo;             // keys are below 2^31: the top bit says "below lo"
-                    asm volatile("{\n\t.reg .pred q;\n\tsetp.lt.u32 q, %0, %1;\n\t@q red.shared.add.u32 [%2], 1;\n\t}"
-                                 ::"r"(off), "r"(span), "r"(hist_s + ((off >> sh) << 2)) : "memory");
-                    below += off >> 31;
+                    asm volatile("red.shared.add.u32 [%0], 1;" ::"r"(hist_s + (min(off >> sh, idle_bin) << 2)) : "memory");
+                    below = __umulhi(off, 2u) + below;
                 }
             }
         });
@@ -1048,31 +1049,28 @@ __global__ void __launch_bounds__(COL_THREADS, 2) select_cols_kernel(const __gri
         for (int j = 0; j < COL_LINES; ++j) sh = (j < nl && fl[j].sh > sh) ? fl[j].sh : sh;
         for (int i = tid; i < COL_LINES * HSTRIDE; i += COL_THREADS) hist[i] = 0u;
         __syncthreads();
-        if (tid < nl) fl[tid].sh = sh;
+        if (tid < nl) { fl[tid].sh = sh; fl[tid].hi = fl[tid].lo + ((uint32_t)HBINS << sh); }
         {   // first pass: the elements inside a column's bracket go to its histogram (predicated: the other lanes cost
             // the shared-memory pipe nothing), those below it are counted, those above it follow from the length
-            uint32_t lo[COL_LINES], span[COL_LINES], below[COL_LINES];
+            uint32_t lo[COL_LINES], below[COL_LINES];
 #pragma unroll
             for (int j = 0; j < COL_LINES; ++j) {
-                lo[j] = fl[j].lo;                    // (a column past the matrix edge has an empty bracket)
-                span[j] = fl[j].hi - fl[j].lo;
+                lo[j] = fl[j].lo;                    // (a column past the matrix edge fills bins nobody reads)
                 below[j] = 0u;
             }
-            // every lane updates a counter: its element's bin inside the bracket, else a word of its own behind the column's
-            // bins that nobody reads
-            const uint32_t idle_rel = (uint32_t)(HBINS + lane) * 4u;
+            // every lane updates a counter: its element's bin inside the bracket (the bracket spans all HBINS bins), else a
+            // word of its own behind the column's bins that nobody reads
+            const uint32_t idle_bin = (uint32_t)(HBINS + lane);
             auto count_key = [&](auto jc, uint32_t key) {                 // jc: the column, a compile-time constant
                 constexpr int J = decltype(jc)::value;
                 const uint32_t off = key - lo[J];                         // keys are below 2^31: the top bit says "below lo"
-                const uint32_t rel = off < span[J] ? (off >> sh) << 2 : idle_rel;
-                asm volatile("red.shared.add.u32 [%0+%1], 1;" ::"r"(hist_s + rel), "n"(J * HSTRIDE * 4) : "memory");
-                below[J] += off >> 31;
+                asm volatile("red.shared.add.u32 [%0+%1], 1;" ::"r"(hist_s + (min(off >> sh, idle_bin) << 2)), "n"(J * HSTRIDE * 4) : "memory");
+                below[J] = __umulhi(off, 2u) + below[J];
             };
             auto visit = [&](int j, float wf, float sc_, int64_t) {
                 const uint32_t off = product_key(wf, sc_) - lo[j];
-                const uint32_t rel = off < span[j] ? (off >> sh) << 2 : idle_rel;
-                asm volatile("red.shared.add.u32 [%0], 1;" ::"r"(hist_s + (uint32_t)(j * HSTRIDE * 4) + rel) : "memory");
-                below[j] += off >> 31;
+                asm volatile("red.shared.add.u32 [%0], 1;" ::"r"(hist_s + (uint32_t)(j * HSTRIDE * 4) + (min(off >> sh, idle_bin) << 2)) : "memory");
+                below[j] = __umulhi(off, 2u) + below[j];
             };
             if constexpr (TMA) {
                 for (int it = 0; it < n_it; ++it) {
