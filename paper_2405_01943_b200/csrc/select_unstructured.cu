@@ -1335,6 +1335,8 @@ __global__ void __launch_bounds__(256, 4) select_emit_cols_kernel(const EmitPara
 // stay the same for the whole run, and "product < threshold" is read off the sign of a float difference that one
 // byte permute turns into the pruned-lane mask of a word.  Columns whose threshold the exact stage had to split
 // (rounded products tie across the cut) take a scalar fix-up for the elements equal to the threshold.
+constexpr int SE_MIN_BLOCKS = 5;                 // CTAs per SM the emit kernel is built for
+constexpr int SE_STAGES = 2;                     // ring slots per warp (a third slot would cost the fifth CTA its shared memory)
 struct EmitStreamParams : UnitGrid {
     const uint16_t *W;
     uint16_t *Wp;        // nullable
@@ -1385,7 +1387,9 @@ __device__ __noinline__ uint32_t emit_exact_row(uint4 row, uint32_t keep, uint32
     return keep;
 }
 
-__global__ void __launch_bounds__(PN_THREADS, PN_MIN_BLOCKS)
+// PER_ROW: the scale belongs to the row (it varies down a column) rather than to the column.
+template <bool PER_ROW>
+__global__ void __launch_bounds__(PN_THREADS, SE_MIN_BLOCKS)
 select_emit_stream_kernel(const __grid_constant__ CUtensorMap map_w, const EmitStreamParams p)
 {
     extern __shared__ uint8_t se_smem_raw[];
@@ -1415,10 +1419,10 @@ select_emit_stream_kernel(const __grid_constant__ CUtensorMap map_w, const EmitS
                 bin_cols |= 1u << j;
                 tlo[j] = __uint_as_float((uint32_t)DASS_LD(&p.results[c0 + j].tau64));
             }
-            if (!p.scale_per_row) sc[j] = DASS_LD(&p.scale[c0 + j]);
+            if (!PER_ROW) sc[j] = DASS_LD(&p.scale[c0 + j]);
         }
     }
-    UnitRing<true> ring;
+    UnitRing<true, SE_STAGES> ring;
     ring.start(smem, threadIdx.x >> 5, &map_w, p, run, lane);
 
     for (int f = run.f0; f < run.f1; ++f) {
@@ -1428,7 +1432,7 @@ select_emit_stream_kernel(const __grid_constant__ CUtensorMap map_w, const EmitS
         float rs[8];
 #pragma unroll
         for (int i = 0; i < 8; ++i) rs[i] = 0.0f;
-        if (p.scale_per_row) {       // the scale vector is padded with zeros to a multiple of 8 and 32-byte aligned
+        if constexpr (PER_ROW) {     // the scale vector is padded with zeros to a multiple of 8 and 32-byte aligned
             const float4 a = DASS_LD_G(reinterpret_cast<const float4 *>(p.scale + r0));
             const float4 b = DASS_LD_G(reinterpret_cast<const float4 *>(p.scale + r0) + 1);
             rs[0] = a.x; rs[1] = a.y; rs[2] = a.z; rs[3] = a.w; rs[4] = b.x; rs[5] = b.y; rs[6] = b.z; rs[7] = b.w;
@@ -1448,8 +1452,8 @@ select_emit_stream_kernel(const __grid_constant__ CUtensorMap map_w, const EmitS
 #pragma unroll
                 for (int k = 0; k < 4; ++k) {
                     const uint32_t w = wsel(v[i], k);
-                    const float pe = prod_lo(w, p.scale_per_row ? rs[4 * h + i] : sc[2 * k]);
-                    const float po = prod_hi(w, p.scale_per_row ? rs[4 * h + i] : sc[2 * k + 1]);
+                    const float pe = prod_lo(w, PER_ROW ? rs[4 * h + i] : sc[2 * k]);
+                    const float po = prod_hi(w, PER_ROW ? rs[4 * h + i] : sc[2 * k + 1]);
                     Z[i][k] = pruned_lanes(__fsub_rn(pe, tau[2 * k]), __fsub_rn(po, tau[2 * k + 1]));
                     aside[i] |= Z[i][k] & ~pruned_lanes(__fsub_rn(pe, tlo[2 * k]), __fsub_rn(po, tlo[2 * k + 1])) & (0x00010001u << (2 * k));
                 }
@@ -1592,9 +1596,12 @@ static cudaError_t launch_emit_stream(const void *W, void *Wp, uint32_t *mask, c
     cudaError_t e = unit_grid_setup(p, &map, &grid, W, rows, cols, ld, true);
     if (e != cudaSuccess) return e;
     static DeviceMask configured{0ull};
-    e = ensure_dynamic_smem(select_emit_stream_kernel, (int)PN_SMEM_BYTES, configured);
+    static DeviceMask configured_col{0ull};
+    e = scale_per_row ? ensure_dynamic_smem(select_emit_stream_kernel<true>, (int)pn_smem_bytes(SE_STAGES), configured)
+                      : ensure_dynamic_smem(select_emit_stream_kernel<false>, (int)pn_smem_bytes(SE_STAGES), configured_col);
     if (e != cudaSuccess) return e;
-    select_emit_stream_kernel<<<(unsigned)grid, PN_THREADS, PN_SMEM_BYTES, st>>>(map, p);
+    if (scale_per_row) select_emit_stream_kernel<true><<<(unsigned)grid, PN_THREADS, pn_smem_bytes(SE_STAGES), st>>>(map, p);
+    else select_emit_stream_kernel<false><<<(unsigned)grid, PN_THREADS, pn_smem_bytes(SE_STAGES), st>>>(map, p);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     FixParams f;

@@ -157,7 +157,8 @@ __device__ __forceinline__ void store_row8(uint16_t *dst, const uint4 &v, int n,
 constexpr int PN_STAGES = 3;
 constexpr uint32_t PN_SLOT_BYTES = PN_ROWS * PN_COLS * 2;           // 4 KB: one full box
 constexpr uint32_t PN_WARPS = PN_THREADS / 32;
-constexpr uint32_t PN_SMEM_BYTES = PN_WARPS * PN_STAGES * PN_SLOT_BYTES + PN_WARPS * PN_STAGES * 8 + 128;
+constexpr uint32_t pn_smem_bytes(int stages) { return PN_WARPS * stages * PN_SLOT_BYTES + PN_WARPS * stages * 8 + 128; }
+constexpr uint32_t PN_SMEM_BYTES = pn_smem_bytes(PN_STAGES);
 constexpr unsigned long long PN_WAIT_NS = 2000000000ull;            // a wait gives up after 2 s
 
 template <bool NORM_COLS>
@@ -202,8 +203,8 @@ __device__ __forceinline__ bool slot_wait(uint32_t bar, uint32_t parity)
     return false;
 }
 
-// The TMA-fed ring of a warp: PN_STAGES slots of one box each, one mbarrier per slot.
-template <bool NORM_COLS>
+// The TMA-fed ring of a warp: STAGES slots of one box each, one mbarrier per slot.
+template <bool NORM_COLS, int STAGES = PN_STAGES>
 struct UnitRing {
     uint32_t slots, bars;            // shared-memory addresses of this warp's slots and barriers
     const uint8_t *generic;          // generic pointer to slot 0
@@ -223,28 +224,28 @@ struct UnitRing {
     __device__ __forceinline__ void start(uint8_t *smem_aligned, int warp_in_cta, const CUtensorMap *map, const UnitGrid &p,
                                           const Run<NORM_COLS> &run, int lane)
     {
-        generic = smem_aligned + warp_in_cta * PN_STAGES * PN_SLOT_BYTES;
+        generic = smem_aligned + warp_in_cta * STAGES * PN_SLOT_BYTES;
         slots = smem_u32(generic);
-        bars = smem_u32(smem_aligned + PN_WARPS * PN_STAGES * PN_SLOT_BYTES) + warp_in_cta * PN_STAGES * 8;
+        bars = smem_u32(smem_aligned + PN_WARPS * STAGES * PN_SLOT_BYTES) + warp_in_cta * STAGES * 8;
         if (lane == 0) {
 #pragma unroll
-            for (int s = 0; s < PN_STAGES; ++s) mbar_init(bars + 8u * s, 1);
+            for (int s = 0; s < STAGES; ++s) mbar_init(bars + 8u * s, 1);
             asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         }
         __syncwarp();
         f_pre = run.f0;
 #pragma unroll
-        for (int s = 0; s < PN_STAGES - 1; ++s) issue(map, p, run, s, lane);
+        for (int s = 0; s < STAGES - 1; ++s) issue(map, p, run, s, lane);
     }
     // Refills the slot consumed one iteration ago, then waits for the current unit.  Returns its tile (16-byte
     // vectors, row pitch p.pitch16) or nullptr when the wait ran out.
     __device__ __forceinline__ const uint4 *next(const CUtensorMap *map, const UnitGrid &p, const Run<NORM_COLS> &run, int lane)
     {
         __syncwarp();                  // every lane is done reading the slot that is refilled now
-        issue(map, p, run, slot == 0 ? PN_STAGES - 1 : slot - 1, lane);
+        issue(map, p, run, slot == 0 ? STAGES - 1 : slot - 1, lane);
         const bool ok = slot_wait(bars + 8u * slot, phase);
         const uint4 *tile = reinterpret_cast<const uint4 *>(generic + slot * PN_SLOT_BYTES);
-        if (++slot == PN_STAGES) { slot = 0; phase ^= 1u; }
+        if (++slot == STAGES) { slot = 0; phase ^= 1u; }
         return ok ? tile : nullptr;
     }
     // After a failed wait: record it and give the copies still in flight one more bounded chance to land.
@@ -252,7 +253,7 @@ struct UnitRing {
     {
         if (lane == 0 && status) atomicMax(status, (int)DASS_ERR_TIMEOUT);
 #pragma unroll
-        for (int s = 0; s < PN_STAGES; ++s) {
+        for (int s = 0; s < STAGES; ++s) {
             slot_wait(bars + 8u * s, 0u);
             slot_wait(bars + 8u * s, 1u);
         }
