@@ -223,7 +223,7 @@ dass_status dass_feature_sumsq(const void *X, int64_t T, int64_t d, int64_t ldx,
  * index first.  sparsity in [0, 1).  mask_bits / W_pruned as for dass_score_nm (at least one; mask_bits is
  * written in full, padding bits 0).  workspace: dass_select_workspace_bytes(...) bytes, 16-byte aligned (holds
  * the rounded norm^alpha vector, the per-column thresholds, the rows left to the slower exact kernel and, per
- * column, the few elements at its cut that are ranked last: about 1.2 KB per column).  A row that the streaming
+ * column, the few elements at its cut that are ranked last: about 1.9 KB per column).  A row that the streaming
  * kernel cannot decide is cached in shared memory by the exact kernel: rows of more than about 108 000 bf16 or
  * 54 000 f32 elements are DASS_ERR_UNSUPPORTED; lines that are matrix columns have no such limit (below 2^31
  * elements).  W_pruned may be W itself (in place).

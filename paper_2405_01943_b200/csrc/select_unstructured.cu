@@ -306,13 +306,14 @@ constexpr int WIN_SAMPLE = 256;                 // evenly spaced elements of a l
 constexpr int WIN_BELOW = 3;                    // the window: 3 octaves below the octave of the sample's quantile, that octave, 4 above
 constexpr int WIN_SHIFT = 15;                   // 2^26 keys in 2048 bins of 2^15: 256 bins per octave
 constexpr uint32_t WIN_SPAN = 1u << (WIN_SHIFT + HB);
-constexpr int CAND_CAP = 96;                    // elements of the cut's bin that the final ranking takes
+constexpr int CAND_CAP = 160;                   // elements of the cut's bin that the final ranking takes (equal scales: ~100 equal bf16 magnitudes)
 constexpr int64_t FAST_MIN_L = 4096;            // shorter lines go straight to the radix select
 
 struct FastLine {                // bracket state of one comparison line (shared memory)
     uint32_t lo, hi;             // candidates: lo <= key < hi (key = bits of the rounded product, sign cleared)
     uint32_t blo, bhi;           // the bin of the bracket that holds the cut
-    int sh;                      // bin = (key - lo) >> sh
+    uint32_t mul;                // bin = floor((key - lo) * mul / 2^32): bins of an odd width, so that keys a power of two apart
+                                 // (equal scales: bf16 magnitudes) spread over the shared-memory banks
     uint32_t above;              // elements with key >= hi
     uint32_t below;              // elements with key < lo (streaming kernels: above = L - below - inside)
     uint32_t krem2;              // rank, from the top and 1-based, of the last survivor inside [blo, bhi)
@@ -361,7 +362,7 @@ __device__ __forceinline__ void window_from_exponents(const uint32_t *eh, FastLi
         const int e0 = e > WIN_BELOW ? e - WIN_BELOW : 0;
         f.lo = (uint32_t)e0 << 23;
         f.hi = f.lo + WIN_SPAN;
-        f.sh = WIN_SHIFT;
+        f.mul = 0u;
         f.above = 0u; f.below = 0u; f.ncoll = 0u; f.ok = 1u; f.krem2 = 0u; f.bucket = 0u; f.blo = 0u; f.bhi = 0u;
     }
 }
@@ -379,6 +380,18 @@ __device__ __forceinline__ uint32_t win_target(uint32_t k, int64_t L, int S = WI
 // off the expected rank (m is four standard deviations of that rank, set by the host); the bracket is those two
 // keys' fine bins and what lies between.  About 2m/S of the line plus two fine bins falls inside; everything else
 // is only counted.  A miss shows in bracket_pick_bin's counts and sends the line to the radix select.
+// Bins of the bracket's histogram: bin = floor(offset * mul / 2^32) with mul = floor(2^32 / width), width odd and wide
+// enough for HBINS bins to cover `span`.  Bin d holds the offsets [bin_start(d), bin_start(d + 1)).
+__device__ __forceinline__ uint32_t bin_multiplier(uint32_t span)
+{
+    const uint32_t width = ((span + (uint32_t)HBINS - 1u) / (uint32_t)HBINS) | 1u;
+    return (uint32_t)(0x100000000ull / (width < 3u ? 3u : width));
+}
+__device__ __forceinline__ uint32_t bin_start(uint32_t d, uint32_t mul)
+{
+    return (uint32_t)((((unsigned long long)d << 32) + mul - 1u) / mul);
+}
+
 constexpr int FINE_SHIFT = 18;                  // 32 fine bins per octave
 constexpr int FINE_BINS = 256;                  // the 8 octaves of the window
 __device__ __forceinline__ void bracket_from_fine(const uint32_t *fh, uint32_t n_over, FastLine &f, int t, int m, int lane)
@@ -409,10 +422,8 @@ __device__ __forceinline__ void bracket_from_fine(const uint32_t *fh, uint32_t n
         const uint32_t wlo = f.lo;
         f.lo = wlo + ((uint32_t)b_lo << FINE_SHIFT);
         f.hi = wlo + ((uint32_t)b_hi << FINE_SHIFT);
-        const uint32_t span = f.hi - f.lo - 1u;       // largest offset inside the bracket
-        const int bits = 32 - __clz(span);
-        f.sh = bits > HB ? bits - HB : 0;
-        f.hi = f.lo + ((uint32_t)HBINS << f.sh);      // widened to the whole histogram: "inside" is "bin below HBINS"
+        f.mul = bin_multiplier(f.hi - f.lo);
+        f.hi = f.lo + bin_start((uint32_t)HBINS, f.mul);   // widened to the whole histogram: "inside" is "bin below HBINS"
     }
 }
 
@@ -453,8 +464,8 @@ __device__ __forceinline__ void bracket_pick_bin(const uint32_t *h, FastLine &f,
         if (!in_range || who == 0u || bucket > (uint32_t)CAND_CAP) {
             f.ok = 0u;
         } else {
-            f.blo = f.lo + (digit << f.sh);
-            const uint32_t end = f.blo + (1u << f.sh);
+            f.blo = f.lo + bin_start(digit, f.mul);
+            const uint32_t end = f.lo + bin_start(digit + 1u, f.mul);
             f.bhi = end < f.hi ? end : f.hi;
             f.krem2 = krem - greater;
             f.bucket = bucket;
@@ -743,7 +754,7 @@ __global__ void __launch_bounds__(RS_THREADS, 4) select_rows_stream_kernel(const
         // its own behind the bins that nobody reads; the elements below the bracket are counted, those above it follow
         // from the line's length
         const uint32_t lo = fl.lo, idle_bin = (uint32_t)(HBINS + lane);
-        const int sh = fl.sh;
+        const uint32_t mul = fl.mul;
         uint32_t below = 0u;
         sweep([&](int64_t, const Chunk<BF16> &ch, const float (&sc)[8], int nvalid) {
             uint32_t key[8];
@@ -752,7 +763,7 @@ __global__ void __launch_bounds__(RS_THREADS, 4) select_rows_stream_kernel(const
             for (int j = 0; j < 8; ++j) {
                 if (j < nvalid) {
                     const uint32_t off = key[j] - lo;             // keys are below 2^31: the top bit says "below lo"
-                    asm volatile("red.shared.add.u32 [%0], 1;" ::"r"(hist_s + (min(off >> sh, idle_bin) << 2)) : "memory");
+                    asm volatile("red.shared.add.u32 [%0], 1;" ::"r"(hist_s + (min(__umulhi(off, mul), idle_bin) << 2)) : "memory");
                     below = __umulhi(off, 2u) + below;
                 }
             }
@@ -1044,12 +1055,12 @@ __global__ void __launch_bounds__(COL_THREADS, 2) select_cols_kernel(const __gri
         if (warp < nl) bracket_from_fine(fhist + warp * FINE_BINS, s_over[warp], fl[warp], target, p.margin, lane);
         __syncthreads();
         bool lost = false;                           // a bounded wait of the bulk-copy sweep ran out
-        int sh = 0;                                  // one bin width for the strip: the widest bracket's
+        uint32_t mul = 0xffffffffu;                  // one bin width for the strip: the widest bracket's
 #pragma unroll
-        for (int j = 0; j < COL_LINES; ++j) sh = (j < nl && fl[j].sh > sh) ? fl[j].sh : sh;
+        for (int j = 0; j < COL_LINES; ++j) mul = (j < nl && fl[j].mul < mul) ? fl[j].mul : mul;
         for (int i = tid; i < COL_LINES * HSTRIDE; i += COL_THREADS) hist[i] = 0u;
         __syncthreads();
-        if (tid < nl) { fl[tid].sh = sh; fl[tid].hi = fl[tid].lo + ((uint32_t)HBINS << sh); }
+        if (tid < nl) { fl[tid].mul = mul; fl[tid].hi = fl[tid].lo + bin_start((uint32_t)HBINS, mul); }
         {   // first pass: the elements inside a column's bracket go to its histogram (predicated: the other lanes cost
             // the shared-memory pipe nothing), those below it are counted, those above it follow from the length
             uint32_t lo[COL_LINES], below[COL_LINES];
@@ -1064,12 +1075,12 @@ __global__ void __launch_bounds__(COL_THREADS, 2) select_cols_kernel(const __gri
             auto count_key = [&](auto jc, uint32_t key) {                 // jc: the column, a compile-time constant
                 constexpr int J = decltype(jc)::value;
                 const uint32_t off = key - lo[J];                         // keys are below 2^31: the top bit says "below lo"
-                asm volatile("red.shared.add.u32 [%0+%1], 1;" ::"r"(hist_s + (min(off >> sh, idle_bin) << 2)), "n"(J * HSTRIDE * 4) : "memory");
+                asm volatile("red.shared.add.u32 [%0+%1], 1;" ::"r"(hist_s + (min(__umulhi(off, mul), idle_bin) << 2)), "n"(J * HSTRIDE * 4) : "memory");
                 below[J] = __umulhi(off, 2u) + below[J];
             };
             auto visit = [&](int j, float wf, float sc_, int64_t) {
                 const uint32_t off = product_key(wf, sc_) - lo[j];
-                asm volatile("red.shared.add.u32 [%0], 1;" ::"r"(hist_s + (uint32_t)(j * HSTRIDE * 4) + (min(off >> sh, idle_bin) << 2)) : "memory");
+                asm volatile("red.shared.add.u32 [%0], 1;" ::"r"(hist_s + (uint32_t)(j * HSTRIDE * 4) + (min(__umulhi(off, mul), idle_bin) << 2)) : "memory");
                 below[j] = __umulhi(off, 2u) + below[j];
             };
             if constexpr (TMA) {
@@ -1350,14 +1361,15 @@ struct EmitStreamParams : UnitGrid {
 
 // Rare path of the emit pass: the elements of one row of a lane's tile that lie in their column's undecided bin are
 // appended to that column's list (they were written as pruned; the ranking kernel brings the survivors back).
-__device__ __noinline__ void emit_set_aside(uint4 row, uint32_t in_bin, const float *sc8, float row_scale,
+__device__ __noinline__ void emit_set_aside(uint4 row, uint32_t in_bin, const float *col_scales, float row_scale,
                                             int scale_per_row, long long r, long long c0, CandLists cl)
 {
-    for (int j = 0; j < 8; ++j) {
-        if (!((in_bin >> j) & 1u)) continue;
+    while (in_bin) {
+        const int j = __ffs((int)in_bin) - 1;
+        in_bin &= in_bin - 1u;
         const uint32_t w = wsel(row, j >> 1);
         const uint32_t raw = (j & 1) ? (w & 0xffff0000u) : (w << 16);
-        const float s = scale_per_row ? row_scale : sc8[j];
+        const float s = scale_per_row ? row_scale : DASS_LD(&col_scales[c0 + j]);
         const uint32_t key = __float_as_uint(fabsf(__uint_as_float(raw)) * s);
         const uint32_t slot = atomicAdd(cl.count + c0 + j, 1u);
         if (slot < (uint32_t)CAND_CAP) {
@@ -1371,13 +1383,14 @@ __device__ __noinline__ void emit_set_aside(uint4 row, uint32_t in_bin, const fl
 
 // Keep byte of one row of a lane's tile when some of its columns need the exact rule (rare).
 __device__ __noinline__ uint32_t emit_exact_row(uint4 row, uint32_t keep, uint32_t exact_cols, const LineResult *res8,
-                                                const float *sc8, float row_scale, int scale_per_row, long long r)
+                                                const float *col_scales8, float row_scale, int scale_per_row, long long r)
 {
-    for (int j = 0; j < 8; ++j) {
-        if (!((exact_cols >> j) & 1u)) continue;
+    while (exact_cols) {
+        const int j = __ffs((int)exact_cols) - 1;
+        exact_cols &= exact_cols - 1u;
         const uint32_t w = wsel(row, j >> 1);
         const float a = fabsf(__uint_as_float((j & 1) ? (w & 0xffff0000u) : (w << 16)));
-        const float s = scale_per_row ? row_scale : sc8[j];
+        const float s = scale_per_row ? row_scale : DASS_LD(&col_scales8[j]);
         const LineResult t = DASS_LD(res8 + j);
         if (__float_as_uint(__fmul_rn(a, s)) != t.tau32) continue;          // only products equal to the threshold
         const unsigned long long k64 = (unsigned long long)__double_as_longlong((double)a * (double)s);
@@ -1465,15 +1478,15 @@ select_emit_stream_kernel(const __grid_constant__ CUtensorMap map_w, const EmitS
                 for (int i = 0; i < 4; ++i) {
                     const uint32_t in_bin = (aside[i] | (aside[i] >> 15)) & valid & bin_cols;   // bit j = column j
                     if (i < nrows && in_bin)
-                        emit_set_aside(v[i], in_bin, sc, rs[4 * h + i], p.scale_per_row, (long long)(rh + i), c0, p.cand);
+                        emit_set_aside(v[i], in_bin, p.scale, rs[4 * h + i], PER_ROW ? 1 : 0, (long long)(rh + i), c0, p.cand);
                 }
             }
             if (exact_cols) {                        // rounded products equal to a split threshold: the exact rule decides
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
                     if (i < nrows) {
-                        const uint32_t kb = emit_exact_row(v[i], (keep >> (8 * i)) & 0xffu, exact_cols, p.results + c0, sc,
-                                                           rs[4 * h + i], p.scale_per_row, (long long)(rh + i));
+                        const uint32_t kb = emit_exact_row(v[i], (keep >> (8 * i)) & 0xffu, exact_cols, p.results + c0, p.scale + c0,
+                                                           rs[4 * h + i], PER_ROW ? 1 : 0, (long long)(rh + i));
                         keep = (keep & ~(0xffu << (8 * i))) | (kb << (8 * i));
                         uint32_t m[4];
                         lanes_of_byte(kb, m);
