@@ -186,6 +186,27 @@ def test_full_size_70b_sampled_lines():
     assert np.array_equal(bits_of(pruned[torch.from_numpy(rws).to(DEV)]), bits_like(want_pruned, Wd.dtype))
 
 
+def test_full_matrices_7b_shape_every_line():
+    """Whole LLaMA2-7B-shaped matrices against the oracle, every line and every element: gate with columns as the
+    lines (Eq. 4, alpha = 0.5, and alpha = 0 where equal magnitudes tie in every column), down with rows as the lines
+    (Eq. 5).  Masks, pruned copies and the count of survivors per line."""
+    cfg = synth.CONFIGS["llama2_7b"]
+    Wg, _, Wd = synth.make_weights(cfg, DEV)
+    gen = torch.Generator(device=DEV)
+    gen.manual_seed(9)
+    norm = (torch.randn(cfg.I, generator=gen, device=DEV).abs() * 40 + 0.5).float().contiguous()
+    norm32 = to_np32(norm)
+    for W, axis, alpha, s in ((Wg, AXIS_ROWS, 0.5, 0.5), (Wg, AXIS_ROWS, 0.0, 0.5), (Wd, AXIS_COLS, 1.0, 0.5)):
+        mask_bits, pruned = binding.select_unstructured(W, norm, axis, alpha, s, axis)
+        binding.prune_status()
+        Wn = to_np32(W)
+        want = oracle.select_unstructured(Wn, norm32, axis, alpha, s, axis)
+        assert np.array_equal(u32(mask_bits), oracle.pack_mask(want)), "mask words differ"
+        assert np.array_equal(bits_of(pruned), bits_like(np.where(want == 1, Wn, np.float32(0.0)), W.dtype)), "pruned weights differ"
+        L = W.shape[0] if axis == AXIS_ROWS else W.shape[1]
+        assert np.all(want.sum(0 if axis == AXIS_ROWS else 1) == L - int(np.floor(s * L)))
+
+
 def test_argument_errors():
     lib = binding.load()
     F = 0x10000
