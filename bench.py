@@ -74,15 +74,16 @@ def _git_blob_sha(path):
 
 
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per launch, from ncu captures summarised under profiles/.
-# Each entry names its summary and the git blob id of the kernel source it was captured from; when the source has
+# Each entry names its summary and the git blob ids of the kernel sources it was captured from; when a source has
 # changed since, the number is withheld (reported as null) instead of going stale.
 NCU_DRAM_BYTES = {
     "llama2_70b": {
         "calib": {"bytes": 4 * (29.607549696e9 + 15.025152e6), "profile": "profiles/calib_tc2_kernel_llama2_70b_T65536_dram.md",
-                  "source": "paper_2405_01943_b200/csrc/calib_tc2.cu", "blob": "729748d82f305308578b4f36418f5fcceedbd567",
+                  "sources": {"paper_2405_01943_b200/csrc/calib_tc2.cu": "729748d82f305308578b4f36418f5fcceedbd567"},
                   "how": "one launch at T = 65536 (one group of 16 interleaved bands) x 4: the full launch repeats that group four times"},
-        "prune": {"bytes": (2 * (470.0 + 706.4) + 470.0 + 708.5) * 1e6, "profile": "profiles/prune_bf16_kernels_llama2_70b_matrices.md",
-                  "source": "paper_2405_01943_b200/csrc/prune_nm_bf16.cu", "blob": "fcc444888ad6e9461fd7ad586f333d7f33683726",
+        "prune": {"bytes": (1176.3 + 1176.6 + 1178.0) * 1e6, "profile": "profiles/prune_bf16_kernels_llama2_70b_matrices.md",
+                  "sources": {"paper_2405_01943_b200/csrc/prune_nm_bf16.cu": "589f5434a8fb3dc0205c8543aba82e894d24f928",
+                              "paper_2405_01943_b200/csrc/stream_units.cuh": "09bbd579b7cb40f0fd99356d6d5c9bcdee68fc45"},
                   "how": "the three launches of one step (gate, up, down) on the full-size matrices"},
     },
 }
@@ -92,9 +93,10 @@ def ncu_traffic(cfg_name, key):
     rec = NCU_DRAM_BYTES.get(cfg_name, {}).get(key)
     if rec is None:
         return None, None
-    if _git_blob_sha(rec["source"]) != rec["blob"]:
-        return None, {"withheld": f"{rec['source']} changed since {rec['profile']} was captured"}
-    return rec["bytes"], {"profile": rec["profile"], "source": rec["source"], "blob": rec["blob"], "how": rec["how"]}
+    changed = [src for src, blob in rec["sources"].items() if _git_blob_sha(src) != blob]
+    if changed:
+        return None, {"withheld": f"{', '.join(changed)} changed since {rec['profile']} was captured"}
+    return rec["bytes"], {"profile": rec["profile"], "sources": rec["sources"], "how": rec["how"]}
 
 
 def roofline_b(kernel, algorithmic_bytes, in_step_ms, isolated_ms, peaks, peak_src, traffic, provenance):
@@ -504,7 +506,8 @@ def unstructured_leg(path, pool, alpha, iters, peaks, sparsity=0.5):
     return {"sparsity": sparsity, "ms_x3": ms, "achieved": gbs, "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"],
             "frac_of_nominal": gbs / NOMINAL["hbm_gbs"],
             "alpha0_ms_x3": ms_a0, "alpha0_frac": nbytes / (ms_a0 * 1e-3) / 1e9 / peaks["hbm_gbs"],
-            "kernels": "select_cols_kernel + select_emit_cols_kernel (gate, up), select_rows_kernel (down)",
+            "kernels": "select_cols_kernel + select_emit_stream_kernel + select_fix_cols_kernel (gate, up), "
+                       "select_rows_stream_kernel + select_rows_kernel for the rows it leaves (down)",
             "algorithmic_bytes_per_step": nbytes, "timed": "alone, back to back, after the step loop"}
 
 
