@@ -1,4 +1,6 @@
-// Stage (b) for bf16 weights: Eq. 4 / Eq. 5 score and N:M selection, tuned to stay under the HBM roofline.
+// Stage (b) for bf16 weights: Eq. 4 / Eq. 5 score and N:M selection (mask and pruned copy), tuned to stay under the
+// HBM roofline.  The patterns with n_keep = m / 2 (2:4, 4:8) are served by the one-pass kernels of prune_nm_bf16.cu;
+// these kernels serve the other bf16 patterns (1:4, 3:4, 1:8 ... 7:8).
 //
 // Same tiling as the generic kernels in score_nm.cu (a lane owns 8 consecutive columns = one 16-byte
 // vector; a warp row is one contiguous 512-byte segment), but the selection is done with 32-bit

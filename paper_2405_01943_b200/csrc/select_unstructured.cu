@@ -1,22 +1,26 @@
 // Unstructured DaSS selection at a sparsity ratio s (Section 3, "Pruning Granularity"): in every comparison
 // line -- a column of Wg / Wu (all neurons at one input: input-balanced) or a row of Wd (output-balanced) --
-// the floor(s * L) weights with the lowest Eq. 4 / Eq. 5 score are pruned.  No sort: an exact radix select.
+// the floor(s * L) weights with the lowest Eq. 4 / Eq. 5 score are pruned.  No sort.
 //
 // The order of the oracle, "higher score first, lower index first", is the order of a three-part key: the
-// rounded product fl32(|w| * scale), then the exact double product, then the index counted from the top.  Its
-// k-th largest value per line is found 11 bits at a time with shared-memory histograms, and a line stops as soon
-// as the bucket at the cut holds exactly the survivors still wanted (after two or three passes on real data;
-// exact products and indices are consulted only where rounded products tie across the cut).
-// In front of that sits, for lines that are matrix columns, a sampled bracket, which decides almost every line of
-// real data without the conflict-heavy first histogram pass: 512 evenly spaced elements of the line are sorted, the two sample values that enclose the
-// wanted rank with a margin of four standard deviations bracket the cut, one pass counts the elements above the
-// bracket and histograms the few per cent inside it (evenly spread over the bins: no hot bins), a second pass
-// collects the handful of elements of the bin that holds the cut, and one warp ranks those by the full key.  A line
-// whose bracket misses, or whose bin holds many equal products, takes the radix select instead.
-// Lines that are matrix rows: one CTA per row, the row cached in shared memory, outputs written by the same CTA.
-// Lines that are matrix columns: one CTA per strip of 8 adjacent columns, re-read from L2 on every pass; the
-// kernel publishes (tau32, exact, tau64, cut) per column and select_emit_cols_kernel applies them in a streaming
-// pass with coalesced rows.
+// rounded product fl32(|w| * scale), then the exact double product, then the index counted from the top.
+//
+// Lines of FAST_MIN_L elements and more are decided by two streaming sweeps: 1024 evenly spaced elements of the line
+// give, through two small histograms (no sort), a bracket of rounded products that holds the cut unless the sample is
+// four standard deviations off; the first sweep reduces every element into a 2048-bin histogram of the bracket (those
+// outside land on idle words) and counts the elements below it; one warp finds the bin that holds the cut; the second
+// sweep writes the outputs -- above the bin stays, below it goes -- and sets the bin's few elements aside; one warp
+// ranks those by the full key and puts the survivors back.  A line whose bracket misses, or whose bin holds more than
+// CAND_CAP elements, is decided by the radix select: the k-th largest key is found 11 bits at a time with
+// shared-memory histograms, and a line stops as soon as the bucket at the cut holds exactly the survivors still
+// wanted (exact products and indices are consulted only where rounded products tie across the cut).
+//
+// Lines that are matrix rows: select_rows_stream_kernel (both sweeps, two rows per CTA), then select_rows_kernel
+// (radix select, the row cached in shared memory) for the rows the first kernel listed, or for every row when the
+// lines are short.  Lines that are matrix columns: select_cols_kernel (one CTA per strip of 8 adjacent columns: sample,
+// first sweep, bin; radix select inside the kernel where needed) publishes a LineResult per column, a streaming
+// kernel with coalesced rows emits (select_emit_stream_kernel for bf16, select_emit_cols_kernel for f32), and
+// select_fix_cols_kernel ranks what the emit pass set aside.
 #include <cmath>
 #include <cstring>
 #include <type_traits>
@@ -902,10 +906,10 @@ __global__ void __launch_bounds__(RS_THREADS, 4) select_rows_stream_kernel(const
 }
 
 // ---------------------------------------------------------------- lines that are matrix columns
-// One CTA per strip of 8 adjacent columns (16 bytes of every row for bf16, 32 for f32).  The strip is not cached:
-// every pass reads it again with one vector load per row and thread, and one CTA per SM keeps the strips in
-// flight (148 x 0.46 MB on the 70B-shaped matrix) inside L2, so only the first pass reads DRAM.  The kernel
-// publishes (tau32, exact, tau64, cut) per column; select_emit_cols_kernel applies them with coalesced rows.
+// One CTA per strip of 8 adjacent columns (16 bytes of every row for bf16, 32 for f32).  The strip is not cached: the
+// sweep of the sampled bracket reads it once (bf16: through bulk tensor copies), and every pass of the radix select,
+// where a column needs it, reads it again with one vector load per row and thread (mostly from L2).  The kernel
+// publishes a LineResult per column: the bin that holds the cut (bf16), or the exact rule (tau32, exact, tau64, cut).
 constexpr int COL_THREADS = 512;                // two CTAs per SM: one sweeps while the other samples, picks its bins or waits
 constexpr int COL_SAMPLE = 1024;                // evenly spaced rows of a strip that place its columns' brackets
 constexpr int COL_LINES = 8;
