@@ -384,11 +384,15 @@ __device__ __forceinline__ uint32_t win_target(uint32_t k, int64_t L, int S = WI
 // off the expected rank (m is four standard deviations of that rank, set by the host); the bracket is those two
 // keys' fine bins and what lies between.  About 2m/S of the line plus two fine bins falls inside; everything else
 // is only counted.  A miss shows in bracket_pick_bin's counts and sends the line to the radix select.
-// Bins of the bracket's histogram: bin = floor(offset * mul / 2^32) with mul = floor(2^32 / width), width odd and wide
-// enough for HBINS bins to cover `span`.  Bin d holds the offsets [bin_start(d), bin_start(d + 1)).
+// Bins of the bracket's histogram: BBINS of them (about a sixth of a line falls inside the bracket: 9 elements per bin
+// for a line of 28672, and equal bf16 magnitudes lie 2^16 keys apart, many bin widths), bin = floor(offset * mul / 2^32)
+// with mul = floor(2^32 / width), width odd and wide enough for BBINS bins to cover `span`.  Bin d holds the offsets
+// [bin_start(d), bin_start(d + 1)).
+constexpr int BBINS = 1024;
+constexpr int64_t FAST_MAX_L = 1 << 18;         // longer lines would crowd the bins: radix select
 __device__ __forceinline__ uint32_t bin_multiplier(uint32_t span)
 {
-    const uint32_t width = ((span + (uint32_t)HBINS - 1u) / (uint32_t)HBINS) | 1u;
+    const uint32_t width = ((span + (uint32_t)BBINS - 1u) / (uint32_t)BBINS) | 1u;
     return (uint32_t)(0x100000000ull / (width < 3u ? 3u : width));
 }
 __device__ __forceinline__ uint32_t bin_start(uint32_t d, uint32_t mul)
@@ -427,17 +431,18 @@ __device__ __forceinline__ void bracket_from_fine(const uint32_t *fh, uint32_t n
         f.lo = wlo + ((uint32_t)b_lo << FINE_SHIFT);
         f.hi = wlo + ((uint32_t)b_hi << FINE_SHIFT);
         f.mul = bin_multiplier(f.hi - f.lo);
-        f.hi = f.lo + bin_start((uint32_t)HBINS, f.mul);   // widened to the whole histogram: "inside" is "bin below HBINS"
+        f.hi = f.lo + bin_start((uint32_t)BBINS, f.mul);   // widened to the whole histogram: "inside" is "bin below BBINS"
     }
 }
 
 // One warp: the bin of the window's histogram that holds the line's last survivor.
 __device__ __forceinline__ void bracket_pick_bin(const uint32_t *h, FastLine &f, uint32_t k, int lane, int64_t L_if_below = -1)
 {
-    const uint32_t *mine_bins = h + lane * 64;
+    constexpr int PER_LANE = BBINS / 32;
+    const uint32_t *mine_bins = h + lane * PER_LANE;
     uint32_t lane_sum = 0u;
 #pragma unroll 4
-    for (int i = 0; i < 64; ++i) lane_sum += mine_bins[(i + lane) & 63];
+    for (int i = 0; i < PER_LANE; ++i) lane_sum += mine_bins[(i + lane) & (PER_LANE - 1)];
     uint32_t v = lane_sum;                            // becomes the sum over lanes >= this one
 #pragma unroll
     for (int off = 1; off < 32; off <<= 1) {
@@ -453,9 +458,9 @@ __device__ __forceinline__ void bracket_pick_bin(const uint32_t *h, FastLine &f,
     const bool mine = in_range && above < krem && krem <= above + lane_sum;
     uint32_t d = 0u, g = 0u, bc = 0u;
     if (mine) {
-        for (int i = 63; i >= 0; --i) {
+        for (int i = PER_LANE - 1; i >= 0; --i) {
             const uint32_t c = mine_bins[i];
-            if (krem <= above + c) { d = (uint32_t)(lane * 64 + i); g = above; bc = c; break; }
+            if (krem <= above + c) { d = (uint32_t)(lane * PER_LANE + i); g = above; bc = c; break; }
             above += c;
         }
     }
@@ -652,7 +657,7 @@ __global__ void __launch_bounds__(ROW_THREADS) select_rows_kernel(const SelectPa
 constexpr int RS_THREADS = 256;
 constexpr int RS_ROWS = 2;
 constexpr int RS_SAMPLE = 1024;                 // evenly spaced elements of a row that place its bracket
-constexpr int RS_HSTRIDE = HBINS + 32;          // a row's bins, then one idle word per lane
+constexpr int RS_HSTRIDE = BBINS + 32;          // a row's bins, then one idle word per lane (the sample's 256 + 256 counters fit in front)
 
 // ALONG: the scale varies along the row (one per column) rather than being one number per row.
 template <bool BF16, bool ALONG>
@@ -775,13 +780,13 @@ __global__ void __launch_bounds__(RS_THREADS, 4) select_rows_stream_kernel(const
     __syncthreads();
 
     // ---------------------------------------------------------------- first pass: histograms of the brackets
-    {   // every lane updates a counter: its element's bin inside the bracket (which spans all HBINS bins), else a word of
+    {   // every lane updates a counter: its element's bin inside the bracket (which spans all BBINS bins), else a word of
         // its own behind the bins that nobody reads; the elements below the bracket are counted, those above it follow
         // from the line's length
         uint32_t lo[RS_ROWS], mul[RS_ROWS], below[RS_ROWS];
 #pragma unroll
         for (int r = 0; r < RS_ROWS; ++r) { lo[r] = fl[r < nr ? r : 0].lo; mul[r] = fl[r < nr ? r : 0].mul; below[r] = 0u; }
-        const uint32_t idle_bin = (uint32_t)(HBINS + lane);
+        const uint32_t idle_bin = (uint32_t)(BBINS + lane);
         sweep([&](int64_t, const Chunk<BF16> (&ch)[RS_ROWS], const float (&sc)[8], int nvalid) {
 #pragma unroll
             for (int r = 0; r < RS_ROWS; ++r) {
@@ -919,10 +924,10 @@ constexpr int COL_COPIES = 1;                   // histogram copies per column (
 // TMA (bf16, at least 8 columns): the sweep of the sampled bracket receives the strip through bulk tensor copies --
 // SR_STAGE_ROWS rows of 16 bytes per stage, one stage in flight while the other is worked on -- instead of one 16-byte load per thread from 1024
 // different cache lines per warp instruction pair, which kept the load/store pipe busier than the arithmetic.
-constexpr int HSTRIDE = HBINS + 32;                      // a column's bins of the bracket sweep, then one idle word per lane
+constexpr int HSTRIDE = BBINS + 32;                      // a column's bins of the bracket sweep, then one idle word per lane
 constexpr int SR_STAGES = 2;
 constexpr int SR_BOX_ROWS = 256;                         // rows of one bulk copy (a box dimension is at most 256)
-constexpr int SR_STAGE_ROWS = 1024;                      // rows of one stage: SR_RPT per thread
+constexpr int SR_STAGE_ROWS = 2048;                      // rows of one stage: SR_RPT per thread
 constexpr int SR_RPT = SR_STAGE_ROWS / COL_THREADS;
 constexpr uint32_t SR_STAGE_BYTES = SR_STAGE_ROWS * 16u;
 
@@ -999,7 +1004,7 @@ __global__ void __launch_bounds__(COL_THREADS, 2) select_cols_kernel(const __gri
     __shared__ uint32_t s_over[COL_LINES];           // sample keys above a column's window
     bool any_pending = true;
     if (tid < COL_LINES) { fl[tid].ok = 0u; fl[tid].lo = 0u; fl[tid].hi = 0u; }     // past the matrix edge: an empty bracket
-    if (p.L >= FAST_MIN_L) {                         // the same for every thread
+    if (p.L >= FAST_MIN_L && p.L <= FAST_MAX_L) {    // the same for every thread
         const uint32_t hist_s = smem_u32(hist);
         // the ring of the bulk-copy sweep, behind the histograms (128-byte aligned), and its barriers
         uint8_t *ring_mem = u_smem + (size_t)COL_LINES * HSTRIDE * sizeof(uint32_t);
@@ -1112,7 +1117,7 @@ __global__ void __launch_bounds__(COL_THREADS, 2) select_cols_kernel(const __gri
         for (int j = 0; j < COL_LINES; ++j) mul = (j < nl && fl[j].mul < mul) ? fl[j].mul : mul;
         for (int i = tid; i < COL_LINES * HSTRIDE; i += COL_THREADS) hist[i] = 0u;
         __syncthreads();
-        if (tid < nl) { fl[tid].mul = mul; fl[tid].hi = fl[tid].lo + bin_start((uint32_t)HBINS, mul); }
+        if (tid < nl) { fl[tid].mul = mul; fl[tid].hi = fl[tid].lo + bin_start((uint32_t)BBINS, mul); }
         {   // first pass: the elements inside a column's bracket go to its histogram (predicated: the other lanes cost
             // the shared-memory pipe nothing), those below it are counted, those above it follow from the length
             uint32_t lo[COL_LINES], below[COL_LINES];
@@ -1121,9 +1126,9 @@ __global__ void __launch_bounds__(COL_THREADS, 2) select_cols_kernel(const __gri
                 lo[j] = fl[j].lo;                    // (a column past the matrix edge fills bins nobody reads)
                 below[j] = 0u;
             }
-            // every lane updates a counter: its element's bin inside the bracket (the bracket spans all HBINS bins), else a
+            // every lane updates a counter: its element's bin inside the bracket (the bracket spans all BBINS bins), else a
             // word of its own behind the column's bins that nobody reads
-            const uint32_t idle_bin = (uint32_t)(HBINS + lane);
+            const uint32_t idle_bin = (uint32_t)(BBINS + lane);
             auto count_key = [&](auto jc, uint32_t key) {                 // jc: the column, a compile-time constant
                 constexpr int J = decltype(jc)::value;
                 const uint32_t off = key - lo[J];                         // keys are below 2^31: the top bit says "below lo"
@@ -1184,9 +1189,15 @@ __global__ void __launch_bounds__(COL_THREADS, 2) select_cols_kernel(const __gri
         __syncthreads();
         if (warp < nl) bracket_pick_bin(hist + warp * HSTRIDE, fl[warp], p.k, lane, p.L);
         __syncthreads();
-        if (lost) {                                  // the same for every thread: the counts are incomplete
-            if (tid < nl) fl[tid].ok = 0u;
-            __syncthreads();
+        if (lost) {   // the same for every thread: the counts are incomplete, and copies may still land in the ring,
+                      // which the radix select would use as its histograms: the strip is given up (every element stays)
+            if (tid < nl) {
+                LineResult r;
+                r.tau32 = 0u; r.exact = 0u; r.tau64 = 0ull; r.cut = 0ll;
+                DASS_ST(&p.results[c0 + tid], r);
+                if (p.cand_count) DASS_ST(&p.cand_count[c0 + tid], 0u);
+            }
+            return;
         }
         if constexpr (DEFER) {
             if (tid < nl && fl[tid].ok) {            // published at the bin; nothing set aside yet
@@ -1692,7 +1703,7 @@ static cudaError_t launch_rows(SelectParams p, uint32_t *line_count, uint32_t *l
     const size_t smem = select_row_smem_bytes(p.L, BF16);
     cudaError_t e = cudaFuncSetAttribute(select_rows_kernel<BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    if (p.L < FAST_MIN_L) {                          // short lines: the radix kernel alone, one CTA per row
+    if (p.L < FAST_MIN_L || p.L > FAST_MAX_L) {      // short or very long lines: the radix kernel alone, one CTA per row
         p.line_count = nullptr; p.line_list = nullptr;
         select_rows_kernel<BF16><<<(unsigned)p.rows, ROW_THREADS, smem, st>>>(p);
         return cudaGetLastError();
@@ -1728,6 +1739,9 @@ static cudaError_t launch_cols_as(const SelectParams &p, cudaStream_t st)
         if (!tile_map_bf16(&map, p.W, p.rows, p.cols, p.ld, COL_LINES, SR_BOX_ROWS)) return cudaErrorInvalidValue;
         smem += 128 + SR_STAGES * SR_STAGE_BYTES + SR_STAGES * 8;
     }
+    // the radix select lays its 2048-bin histograms over the same bytes (the bracket's bins and the ring are idle by then)
+    const size_t radix_smem = (size_t)COL_LINES * COL_COPIES * HBINS * sizeof(uint32_t);
+    smem = smem < radix_smem ? radix_smem : smem;
     cudaError_t e = cudaFuncSetAttribute(select_cols_kernel<BF16, ALONG, TMA>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     select_cols_kernel<BF16, ALONG, TMA><<<(unsigned)((p.cols + COL_LINES - 1) / COL_LINES), COL_THREADS, smem, st>>>(map, p);
@@ -1737,7 +1751,7 @@ template <bool BF16>
 static cudaError_t launch_cols(const SelectParams &p, cudaStream_t st)
 {
     // bulk copies need whole boxes of 8 columns x 256 rows inside the matrix, and the sweep they feed runs on long lines only
-    const bool tma = BF16 && p.cols >= COL_LINES && p.L >= FAST_MIN_L && p.rows < 0x7fffffffll - SR_STAGE_ROWS;
+    const bool tma = BF16 && p.cols >= COL_LINES && p.L >= FAST_MIN_L && p.L <= FAST_MAX_L;
     if constexpr (BF16) {
         if (tma) return p.scale_along_line ? launch_cols_as<true, true, true>(p, st) : launch_cols_as<true, false, true>(p, st);
     }
