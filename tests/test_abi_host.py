@@ -34,8 +34,8 @@ def test_header_symbols_are_exported(lib):
 
 def test_status_strings_and_version(lib):
     assert binding.status_string(0) == "ok"
-    seen = {binding.status_string(c) for c in range(9)}
-    assert len(seen) == 9
+    seen = {binding.status_string(c) for c in range(10)}
+    assert len(seen) == 10
     assert binding.status_string(1234) == "unknown status"
     assert binding.version() >= 100
 
@@ -49,6 +49,25 @@ def test_workspace_query_validation(lib):
     assert lib.dass_calib_workspace_bytes(128, 256, 688, 7, ctypes.byref(out)) == 4        # DTYPE
     assert lib.dass_calib_workspace_bytes(262144, 8192, 28672, binding.BF16, ctypes.byref(out)) == 0
     assert out.value < (1 << 30)
+
+
+def test_select_workspace_query(lib):
+    """The selection's scratch holds a result per column, the rounded scale vector, the list of rows left to the exact
+    kernel and, per column, a counter and the slots of the elements ranked last."""
+    out = ctypes.c_size_t(0)
+    f = lib.dass_select_workspace_bytes
+    assert f(8192, 28672, binding.AXIS_COLS, None) == 1                                   # NULL
+    assert f(0, 64, binding.AXIS_COLS, ctypes.byref(out)) == 2                            # SHAPE
+    assert f(64, 64, 5, ctypes.byref(out)) == 4                                           # bad axis
+    sizes = {}
+    for rows, cols, axis in ((8192, 28672, binding.AXIS_COLS), (28672, 8192, binding.AXIS_ROWS), (1, 8, binding.AXIS_ROWS)):
+        assert f(rows, cols, axis, ctypes.byref(out)) == 0
+        sizes[(rows, cols)] = out.value
+        n_norm = rows if axis == binding.AXIS_ROWS else cols
+        floor = 24 * cols + 4 * n_norm + 4 * rows + 4 * cols      # results, scale, row list, per-column counters
+        assert out.value >= floor
+        assert out.value <= floor + 4096 + cols * 3 * 4 * 256     # the ranked slots: a few hundred 12-byte entries per column at most
+    assert sizes[(8192, 28672)] > sizes[(28672, 8192)] > sizes[(1, 8)]
 
 
 def test_calib_workspace_of_short_batches_stays_within_the_static_scratch(lib):

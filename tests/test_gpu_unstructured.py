@@ -186,6 +186,19 @@ def test_full_size_70b_sampled_lines():
     assert np.array_equal(bits_of(pruned[torch.from_numpy(rws).to(DEV)]), bits_like(want_pruned, Wd.dtype))
 
 
+def test_column_lines_at_and_beyond_the_streaming_limit():
+    """Columns of 2^18 rows still take the streaming kernels (128 stages of the bulk-copy ring per strip); one row more
+    and the radix select decides them.  Both against the oracle, every element; 11 columns (a ragged last strip)."""
+    gen = torch.Generator(device=DEV)
+    gen.manual_seed(77)
+    for rows in (1 << 18, (1 << 18) + 1):
+        cols = 11
+        W = _long_case("random", rows, cols, torch.bfloat16, gen, 0)
+        norm = _norm(rows, gen)
+        _check(W, norm, AXIS_ROWS, 0.5, 0.5, AXIS_ROWS)
+    binding.prune_status()
+
+
 def test_full_matrices_7b_shape_every_line():
     """Whole LLaMA2-7B-shaped matrices against the oracle, every line and every element: gate with columns as the
     lines (Eq. 4, alpha = 0.5, and alpha = 0 where equal magnitudes tie in every column), down with rows as the lines
