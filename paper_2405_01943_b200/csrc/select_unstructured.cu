@@ -1160,11 +1160,11 @@ __global__ void __launch_bounds__(COL_THREADS, 2) select_cols_kernel(const __gri
 #pragma unroll
                     for (int u = 0; u < SR_RPT; ++u) {
                         if (r0 + u * COL_THREADS < p.L) {    // rows past the end arrive as zeros and are not counted
-                            const uint32_t a[4] = {v[u].x & 0x7fff7fffu, v[u].y & 0x7fff7fffu, v[u].z & 0x7fff7fffu, v[u].w & 0x7fff7fffu};   // |w|, in pairs
+                            const uint32_t w4[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
                             static_for<COL_LINES>([&](auto jc) {
                                 constexpr int J = decltype(jc)::value;
-                                const float wa = __uint_as_float((J & 1) ? (a[J >> 1] & 0xffff0000u) : (a[J >> 1] << 16));
-                                count_key(jc, __float_as_uint(__fmul_rn(wa, ALONG ? rs[u] : col_scale[J])));
+                                const float sv = ALONG ? rs[u] : col_scale[J];
+                                count_key(jc, __float_as_uint((J & 1) ? prod_hi(w4[J >> 1], sv) : prod_lo(w4[J >> 1], sv)));
                             });
                         }
                     }
