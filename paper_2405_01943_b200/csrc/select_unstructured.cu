@@ -305,11 +305,9 @@ __device__ __forceinline__ bool keeps(const LineResult &res, float a, float s, l
     return k64 > res.tau64 || (k64 == res.tau64 && idx <= res.cut);
 }
 
-// ---------------------------------------------------------------- octave window in front of the radix select
-constexpr int WIN_SAMPLE = 256;                 // evenly spaced elements of a line whose exponents place its window
+// ---------------------------------------------------------------- sampled bracket in front of the radix select
 constexpr int WIN_BELOW = 3;                    // the window: 3 octaves below the octave of the sample's quantile, that octave, 4 above
-constexpr int WIN_SHIFT = 15;                   // 2^26 keys in 2048 bins of 2^15: 256 bins per octave
-constexpr uint32_t WIN_SPAN = 1u << (WIN_SHIFT + HB);
+constexpr uint32_t WIN_SPAN = 1u << 26;         // 8 octaves of keys
 constexpr int CAND_CAP = 160;                   // elements of the cut's bin that the final ranking takes (equal scales: ~100 equal bf16 magnitudes)
 constexpr int64_t FAST_MIN_L = 4096;            // shorter lines go straight to the radix select
 
@@ -372,7 +370,7 @@ __device__ __forceinline__ void window_from_exponents(const uint32_t *eh, FastLi
 }
 
 // Rank, from the top, of the key that stands for the line's k-th largest in a sample of S.
-__device__ __forceinline__ uint32_t win_target(uint32_t k, int64_t L, int S = WIN_SAMPLE)
+__device__ __forceinline__ uint32_t win_target(uint32_t k, int64_t L, int S)
 {
     const int64_t t = ((int64_t)k * S + L - 1) / L;
     return (uint32_t)(t < 1 ? 1 : (t > S ? S : t));
