@@ -56,8 +56,10 @@ class LayerPruner:
         return b.norm_finalize(self.sumsq, self.norm)
 
     def check(self) -> None:
-        """Raises if a bounded device-side wait of the calibration kernel gave up (synchronises the stream)."""
+        """Raises if a bounded device-side wait of the calibration kernel or of a stage-(b) kernel gave up, or the passes
+        of an unstructured selection disagreed (synchronises the stream)."""
         b.calib_status(self.calib_ws)
+        b.prune_status()
 
     # ------------------------------------------------------------------ stage (b)
     def score_nm(self, Wg: torch.Tensor, Wu: torch.Tensor, Wd: torch.Tensor, alpha: float = 0.5) -> None:

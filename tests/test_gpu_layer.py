@@ -60,6 +60,30 @@ def test_prune_unstructured_and_batched_calibration():
     assert np.max(np.abs(to_np32(pruner.norm) - norm_one_call) / norm_one_call) <= 1e-6
 
 
+def test_prune_unstructured_with_long_lines_through_the_layer_calls():
+    """A layer whose comparison lines have 4608 elements (the streaming selection kernels): calibration, then the
+    paper's 50 % unstructured setting on all three matrices, against the oracle fed the GPU's norms; then the same
+    weights through forward_pruned()."""
+    cfg, X, Wg, Wu, Wd = _layer("llama2_7b", d=384, I=4608, T=300)
+    pruner = LayerPruner(cfg.T, cfg.d, cfg.I, X.dtype, act=cfg.act, device=DEV, compressed=False)
+    out = pruner.prune(X, Wg, Wu, Wd, alpha=0.5, sparsity=0.5)
+    pruner.check()
+    ref_norm = oracle.norm_from_sumsq(oracle.calib_sumsq(to_np32(X), to_np32(Wg), to_np32(Wu), ORACLE_ACT[cfg.act]))
+    norm = to_np32(pruner.norm)
+    assert np.max(np.abs(norm - ref_norm) / ref_norm) <= 2e-3
+    for pname, W, axis, alpha in (("gate", Wg, AXIS_ROWS, 0.5), ("up", Wu, AXIS_ROWS, 0.5), ("down", Wd, AXIS_COLS, 1.0)):
+        want = oracle.select_unstructured(to_np32(W), norm, axis, alpha, 0.5, axis)
+        assert np.array_equal(u32(out[pname]["mask"]), oracle.pack_mask(want)), pname
+        assert np.array_equal(bits_of(out[pname]["pruned"]), bits_like(np.where(want == 1, to_np32(W), np.float32(0.0)), W.dtype)), pname
+    Z = pruner.forward_pruned(X)
+    pruner.check()
+    Z_ref, _ = oracle.mlp_forward(to_np32(X), to_np32(out["gate"]["pruned"]), to_np32(out["up"]["pruned"]),
+                                  to_np32(out["down"]["pruned"]), ORACLE_ACT[cfg.act], True, want_h=True)
+    z = to_np32(Z).astype(np.float64)
+    err = np.sqrt(np.mean((z - Z_ref) ** 2)) / (np.sqrt(np.mean(Z_ref ** 2)) + 1e-30)
+    assert err <= 6e-3                                          # the bound test_gpu_forward.py derives for bf16
+
+
 def test_forward_of_the_pruned_layer_matches_oracle_forward_of_the_same_weights():
     """prune() then forward_pruned(): the oracle's forward pass of the very weights the GPU pruned (bf16 rounding
     of the intermediate on both sides), in one pass and in token chunks."""
