@@ -22,7 +22,7 @@ class LayerPruner:
     """Holds the output and scratch buffers of one layer shape, so that pruning a stack of layers allocates once."""
 
     def __init__(self, T: int, d: int, I: int, dtype: torch.dtype, act: str = "silu", n_keep: int = 2, m: int = 4,
-                 device="cuda", compressed: bool = True):
+                 device="cuda", compressed: bool = True, overlap_projections: bool = True):
         self.T, self.d, self.I, self.dtype = int(T), int(d), int(I), dtype
         self.act = b.ACT_BY_NAME[act]
         self.n_keep, self.m, self.device = int(n_keep), int(m), torch.device(device)
@@ -41,6 +41,9 @@ class LayerPruner:
                 o["meta"] = torch.empty(mshape, dtype=torch.int32, device=self.device)
             self.out[name] = o
         self.compressed = compressed
+        # The three projections are independent once the norms exist: up and down are launched on two side streams, so
+        # that one kernel's last CTAs drain while the next one's first CTAs start (the tail of a 40-200 us launch).
+        self._side = [torch.cuda.Stream(device=self.device) for _ in range(2)] if overlap_projections else None
         self._select_ws: Optional[Dict[str, torch.Tensor]] = None
         self._forward_ws: Optional[torch.Tensor] = None
 
@@ -71,12 +74,24 @@ class LayerPruner:
 
     def prune_nm(self, Wg: torch.Tensor, Wu: torch.Tensor, Wd: torch.Tensor, alpha: float = 0.5) -> None:
         """score_nm and compress_nm in one pass per projection: each weight is read once for all of its outputs."""
-        for name, W in zip(_PROJECTIONS, (Wg, Wu, Wd)):
+        cur = torch.cuda.current_stream(self.device)
+        fork = None
+        if self._side is not None:
+            fork = torch.cuda.Event()
+            fork.record(cur)                         # everything the projections read (the norms, the weights) is ordered before it
+        for i, (name, W) in enumerate(zip(_PROJECTIONS, (Wg, Wu, Wd))):
             _, _, axis = self.geometry[name]
             o = self.out[name]
+            stream = cur if (fork is None or i == 0) else self._side[i - 1]
+            if stream is not cur:
+                stream.wait_event(fork)
             b.prune_nm(W, self.norm, axis, alpha if name != "down" else 1.0, self.n_keep, self.m, axis,
                        mask_bits=o["mask"], W_pruned=o["pruned"], values=o.get("values"), meta=o.get("meta"),
-                       want_compressed=self.compressed)
+                       want_compressed=self.compressed, stream=stream)
+            if stream is not cur:
+                join = torch.cuda.Event()
+                join.record(stream)
+                cur.wait_event(join)                 # later work on the caller's stream sees all three projections done
 
     def compress_nm(self, Wg: torch.Tensor, Wu: torch.Tensor, Wd: torch.Tensor) -> None:
         for name, W in zip(_PROJECTIONS, (Wg, Wu, Wd)):
