@@ -234,6 +234,7 @@ select_emit_stream_kernel(const __grid_constant__ CUtensorMap map_w, const EmitS
             if (!PER_ROW) sc[j] = DASS_LD(&p.scale[c0 + j]);
         }
     }
+    const bool cols_full = __all_sync(FULL_MASK, nvalid == 8);     // the warp's 256 columns all exist
     UnitRing<true, SE_STAGES> ring;
     ring.start(smem, threadIdx.x >> 5, &map_w, p, run, lane);
 
@@ -249,11 +250,11 @@ select_emit_stream_kernel(const __grid_constant__ CUtensorMap map_w, const EmitS
             const float4 b = DASS_LD_G(reinterpret_cast<const float4 *>(p.scale + r0) + 1);
             rs[0] = a.x; rs[1] = a.y; rs[2] = a.z; rs[3] = a.w; rs[4] = b.x; rs[5] = b.y; rs[6] = b.z; rs[7] = b.w;
         }
-#pragma unroll
-        for (int h = 0; h < PN_ROWS / 4; ++h) {
+        // four rows of the tile; FULL: all four rows and all of the warp's columns lie inside the matrix
+        auto four_rows = [&](auto full_tag, int h) {
+            constexpr bool FULL = decltype(full_tag)::value;
             const int64_t rh = r0 + 4 * h;
-            if (rh >= p.rows) break;                 // warp-uniform
-            const int nrows = p.rows - rh >= 4 ? 4 : (int)(p.rows - rh);
+            const int nrows = FULL ? 4 : (p.rows - rh >= 4 ? 4 : (int)(p.rows - rh));
             uint4 v[4];
             uint32_t Z[4][4];
             uint32_t aside[4];                       // per row: lanes below the threshold but not below the bin's start
@@ -270,12 +271,12 @@ select_emit_stream_kernel(const __grid_constant__ CUtensorMap map_w, const EmitS
                     aside[i] |= Z[i][k] & ~pruned_lanes(__fsub_rn(pe, tlo[2 * k]), __fsub_rn(po, tlo[2 * k + 1])) & (0x00010001u << (2 * k));
                 }
             }
-            const uint32_t rows4 = nrows == 4 ? 0xffffffffu : ((1u << (8 * nrows)) - 1u);
-            uint32_t keep = ~bytes_of_lanes4(Z[0], Z[1], Z[2], Z[3]) & (valid * 0x01010101u) & rows4;
+            uint32_t keep = ~bytes_of_lanes4(Z[0], Z[1], Z[2], Z[3]);
+            if constexpr (!FULL) keep &= (valid * 0x01010101u) & (nrows == 4 ? 0xffffffffu : ((1u << (8 * nrows)) - 1u));
             if (aside[0] | aside[1] | aside[2] | aside[3]) {     // elements of undecided bins: set aside for the ranking
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
-                    const uint32_t in_bin = (aside[i] | (aside[i] >> 15)) & valid & bin_cols;   // bit j = column j
+                    const uint32_t in_bin = (aside[i] | (aside[i] >> 15)) & (FULL ? 0xffu : valid) & bin_cols;   // bit j = column j
                     if (i < nrows && in_bin)
                         emit_set_aside(v[i], in_bin, p.scale, rs[4 * h + i], PER_ROW ? 1 : 0, (long long)(rh + i), c0, p.cand);
                 }
@@ -294,22 +295,30 @@ select_emit_stream_kernel(const __grid_constant__ CUtensorMap map_w, const EmitS
                     }
                 }
             }
-            const bool row_live = (lane & 3) < nrows;
+            const bool row_live = FULL || (lane & 3) < nrows;
             if (p.mask) {
                 const uint32_t word = quad_transpose(keep, sel1, sel2);
-                if (quad_live && row_live) DASS_ST(&p.mask[(rh + (lane & 3)) * p.wpr + (c0 >> 5)], word);
+                if ((FULL || quad_live) && row_live) DASS_ST(&p.mask[(rh + (lane & 3)) * p.wpr + (c0 >> 5)], word);
             }
-            if (p.Wp && nvalid > 0) {
+            if (p.Wp && (FULL || nvalid > 0)) {
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
                     if (i < nrows) {
                         uint4 P;
 #pragma unroll
                         for (int k = 0; k < 4; ++k) wref(P, k) = wsel(v[i], k) & ~Z[i][k];
-                        store_row8(p.Wp + (rh + i) * p.ld + c0, P, nvalid);
+                        store_row8(p.Wp + (rh + i) * p.ld + c0, P, FULL ? 8 : nvalid);
                     }
                 }
             }
+        };
+        if (cols_full && r0 + PN_ROWS <= p.rows) {   // warp-uniform: the common tile
+#pragma unroll
+            for (int h = 0; h < PN_ROWS / 4; ++h) four_rows(std::true_type{}, h);
+        } else {
+#pragma unroll
+            for (int h = 0; h < PN_ROWS / 4; ++h)
+                if (r0 + 4 * h < p.rows) four_rows(std::false_type{}, h);
         }
     }
 }
