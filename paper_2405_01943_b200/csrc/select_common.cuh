@@ -56,7 +56,7 @@ struct SelectParams {
     uint32_t k;          // survivors per line
     int idx_bits;        // bits of L - 1 (at least 1): width of the index part of the key
     int scale_along_line;   // 1: scale[e] varies along the line; 0: scale[line]
-    int margin;             // sampled bracket: sample positions on either side of the wanted rank (four standard deviations)
+    int margin;             // sampled bracket: sample positions on either side of the wanted rank (five standard deviations)
     uint32_t *line_count;   // row lines: how many lines the streaming kernel left undecided, and which
     uint32_t *line_list;    // (both null: the radix kernel takes every row)
     uint32_t *cand_count;   // column lines, bf16: per-column count of the elements the emit pass sets aside (cleared here)
@@ -354,10 +354,10 @@ __device__ __forceinline__ uint32_t win_target(uint32_t k, int64_t L, int S)
 // One warp: narrows a line's window to a bracket [lo, hi) from the fine histogram of a larger sample (FINE_BINS bins
 // of 2^FINE_SHIFT keys from the window's start; n_over = sample keys above the window).  With the sample sorted from
 // the top, the line's cut lies between the sample's (t - m)-th and (t + m)-th key unless the sample is m positions
-// off the expected rank (m is four standard deviations of that rank, set by the host); the bracket is those two
+// off the expected rank (m is five standard deviations of that rank, set by the host); the bracket is those two
 // keys' fine bins and what lies between.  About 2m/S of the line plus two fine bins falls inside; everything else
 // is only counted.  A miss shows in bracket_pick_bin's counts and sends the line to the radix select.
-// Bins of the bracket's histogram: BBINS of them (about a sixth of a line falls inside the bracket: 9 elements per bin
+// Bins of the bracket's histogram: BBINS of them (about a fifth of a line falls inside the bracket: 5 elements per bin
 // for a line of 28672, and equal bf16 magnitudes lie 2^16 keys apart, many bin widths), bin = floor(offset * mul / 2^32)
 // with mul = floor(2^32 / width), width odd and wide enough for BBINS bins to cover `span`.  Bin d holds the offsets
 // [bin_start(d), bin_start(d + 1)).

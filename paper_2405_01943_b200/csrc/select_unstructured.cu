@@ -7,7 +7,7 @@
 //
 // Lines of FAST_MIN_L elements and more are decided by two streaming sweeps: 1024 evenly spaced elements of the line
 // give, through two small histograms (no sort), a bracket of rounded products that holds the cut unless the sample is
-// four standard deviations off; the first sweep reduces every element into a 2048-bin histogram of the bracket (those
+// five standard deviations off; the first sweep reduces every element into a 1024-bin histogram of the bracket (those
 // outside land on idle words) and counts the elements below it; one warp finds the bin that holds the cut; the second
 // sweep writes the outputs -- above the bin stays, below it goes -- and sets the bin's few elements aside; one warp
 // ranks those by the full key and puts the survivors back.  A line whose bracket misses, or whose bin holds more than
@@ -78,9 +78,12 @@ cudaError_t select_unstructured_launch(const void *W, int64_t rows, int64_t cols
     p.idx_bits = 1;
     while (((int64_t)1 << p.idx_bits) < p.L) ++p.idx_bits;
     p.scale_along_line = (line_is_row == norm_cols) ? 1 : 0;   // the norm index runs along the line
-    {   // four standard deviations of the rank of a sample quantile, in sample positions, plus slack
+    {   // five standard deviations of the rank of a sample quantile, in sample positions, plus slack: a line in
+        // two million misses (a column that misses sends its whole strip of eight through the radix select, which
+        // can lengthen the launch by a CTA's radix passes; the wider bracket costs nothing, every element is reduced
+        // into a counter either way)
         const double q = (double)(p.L - (int64_t)k) / (double)p.L;
-        p.margin = (int)std::ceil(4.0 * std::sqrt((double)SELECT_SAMPLE * q * (1.0 - q))) + 2;
+        p.margin = (int)std::ceil(5.0 * std::sqrt((double)SELECT_SAMPLE * q * (1.0 - q))) + 2;
     }
     if (line_is_row) {
         if (mask_bits) {   // the kernel writes whole bytes of real columns; the padding of each mask row must read 0
